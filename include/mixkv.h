@@ -1,0 +1,146 @@
+/*
+ * mixkv.h -- C ABI of the B200 (sm_100a) MixKV prefill KV-cache compression library.
+ *
+ * The library implements one step of LVLM / LLM inference: at the end of prefill, for
+ * one transformer layer, score every cached key of every KV head, keep the best B per
+ * head and copy the kept K/V rows into a compact cache (MixKV, arxiv 2510.20707,
+ * Sec. 3.1 "KV Cache Compression", Sec. 3.2-3.3, Algorithm 1).
+ *
+ * Conventions shared by every entry point
+ * ---------------------------------------
+ *  - All tensor pointers are DEVICE pointers unless the name ends in `_host`.
+ *    bf16 tensors must be 16-byte aligned, fp32 / int32 tensors 4-byte aligned.
+ *  - The caller owns every buffer, including the workspace.  The library allocates no
+ *    device memory, keeps no global state between calls and never synchronises the
+ *    stream: every call only enqueues kernels on `stream` (a cudaStream_t passed as
+ *    void*; NULL is the default stream).
+ *  - Shapes.  H = kv_heads, G = gqa_ratio, d = head_dim (128), W = window.
+ *      K, V      [H, Ltot, d] bf16, row-major.  Ltot = L for one sequence, else
+ *                cu_seqlens_host[batch]; sequence b owns rows cu[b] .. cu[b+1]-1.
+ *      Qwin      [batch, H*G, W, d] bf16: the last W prompt queries (post-RoPE) of every
+ *                query head; query head q attends KV head q / G.  Window row j sits at
+ *                sequence position P + j (P = L - W) and sees keys 0 .. P + j.
+ *      scores    [H, Ptot] fp32, Ptot = Ltot - batch*W: the P_b = L_b - W candidate
+ *                (non-window) positions of sequence b start at column cu[b] - b*W.
+ *      rbar      [batch, H] fp32.
+ *  - cu_seqlens_host: HOST pointer to batch+1 ascending int32 offsets, read during the
+ *    call (not retained).  NULL means one sequence of length L (batch must be 1).
+ *  - Return value: 0 on success, a negative mixkv_status otherwise; on error nothing has
+ *    been enqueued.  Conditions only the device can see (a bounded wait inside a kernel
+ *    expired) are written to *status_dev (device int32, optional, must be zeroed by the
+ *    caller) as MIXKV_ERR_TIMEOUT; kernels never trap.
+ *  - Limits: head_dim == 128; 16 <= G*W <= 240 and G*W % 16 == 0; batch <= 64;
+ *    every sequence needs L_b >= W + 1; budget > W; odd pool_kernel <= 63.
+ */
+#ifndef MIXKV_H_
+#define MIXKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  MIXKV_OK = 0,
+  MIXKV_ERR_INVALID_ARG = -1,
+  MIXKV_ERR_UNSUPPORTED = -2,
+  MIXKV_ERR_WORKSPACE_TOO_SMALL = -3,
+  MIXKV_ERR_CUDA = -4,
+  MIXKV_ERR_TIMEOUT = -5
+} mixkv_status;
+
+enum { MIXKV_MIX_HEADWISE = 0, MIXKV_MIX_IMPORTANCE_ONLY = 1, MIXKV_MIX_DIVERSITY_ONLY = 2,
+       MIXKV_MIX_PLAIN_SUM = 3 };
+enum { MIXKV_POOL_AVG = 0, MIXKV_POOL_MAX = 1 };
+enum { MIXKV_BUDGET_FIXED = 0, MIXKV_BUDGET_ADAPTIVE = 1 };
+
+typedef struct mixkv_params {
+  int32_t kv_heads;     /* H */
+  int32_t gqa_ratio;    /* G: query heads per KV head */
+  int32_t head_dim;     /* d: must be 128 */
+  int32_t window;       /* W: observation window, paper default 32 (Sec. 3.2) */
+  int32_t pool_kernel;  /* odd k >= 1; 1-D pooling of the attention score, 1 = none */
+  int32_t pool_mode;    /* MIXKV_POOL_AVG (zero padded, divides by k) or MIXKV_POOL_MAX */
+  int32_t use_vnorm;    /* 1: add the value-norm intrinsic importance of Eq. 2 */
+  int32_t mix_mode;     /* MIXKV_MIX_*: Eq. 5, or one of the ablation variants of Table 4 */
+  int32_t budget_mode;  /* MIXKV_BUDGET_FIXED: B per head; _ADAPTIVE: B*H per sequence */
+  int32_t budget;       /* B: rows kept per head INCLUDING the W window rows (Alg. 1) */
+  float ada_floor;      /* adaptive: fraction of B - W guaranteed to every head (0..1) */
+  float eps;            /* epsilon of the two min-max normalisations (Sec. 3.2, 3.3) */
+  float softmax_scale;  /* 0 => 1/sqrt(d) */
+} mixkv_params;
+
+/* Fills *p with the paper's defaults: W 32, average pooling k 7, VNorm on, Eq. 5 mixing,
+ * fixed budget, ada_floor 0.2, eps 1e-6, scale 1/sqrt(d).  Sets H, G and B as given. */
+void mixkv_default_params(mixkv_params* p, int32_t kv_heads, int32_t gqa_ratio, int32_t budget);
+
+/* Bytes of device workspace the three entry points below need for a batch whose sequence
+ * lengths sum to total_tokens (max single length max_seq_len).  Host-only; no CUDA call. */
+int mixkv_workspace_size(const mixkv_params* p, int32_t batch, int64_t total_tokens,
+                         int32_t max_seq_len, size_t* bytes);
+
+/* Scores of every candidate key (Sec. 3.2-3.3; Algorithm 1 step 1 and the mixing of step 2):
+ *   s_ex   = pool_k( sum over the G query heads of the mean over the W window rows of the
+ *            causal softmax attention weight on key i )             (extrinsic importance)
+ *   s_imp  = s_ex + VNorm_i min-max normalised, rescaled to mean(s_ex)            (Eq. 2)
+ *   s_div  = - cos(K_i, mean over all L keys of the unit keys)                  (diversity)
+ *   rbar   = (L^2 |mean unit key|^2 - L) / (L (L-1))                            (Eq. 3-4)
+ *   s_comp = (1 - rbar) s_imp + rbar * (s_div min-max normalised, rescaled to mean(s_imp))
+ *                                                                                 (Eq. 5)
+ * Key geometry (mean unit key, rbar) uses all L keys of the sequence; score vectors and
+ * their min / max / mean use the P candidate positions.
+ *   s_comp        out, required, [H, Ptot]
+ *   s_ex_opt      out, optional (NULL to skip), pooled attention score [H, Ptot]
+ *   s_div_opt     out, optional, raw diversity score [H, Ptot]
+ *   rbar_opt      out, optional, [batch, H]
+ *   rbar_in_opt   in, optional, [batch, H]: redundancy to mix with instead of the computed
+ *                 one (head weights calibrated offline, Sec. 4.3)
+ *   V may be NULL when use_vnorm == 0. */
+int mixkv_scores(const void* K, const void* V, const void* Qwin,
+                 const int32_t* cu_seqlens_host, int32_t batch, int32_t L,
+                 const mixkv_params* p, void* workspace, size_t workspace_bytes,
+                 float* s_comp, float* s_ex_opt, float* s_div_opt, float* rbar_opt,
+                 const float* rbar_in_opt, int32_t* status_dev, void* stream);
+
+/* TopB of Sec. 3.1 / Algorithm 1 on caller-supplied scores [H, Ptot]: per (sequence, head)
+ * the b_h highest scores among the P_b candidates, ties to the lower position, written in
+ * ascending position order.  b_h = min(B - W, P_b) for fixed budgets.  Adaptive budgets
+ * (per sequence): every head is guaranteed f = floor(ada_floor * (B - W)); the remaining
+ * H * (B - W - f) slots go to the highest scores of the H heads taken together (ties to the
+ * lower (head, position)); b_h = min(f + share_h, P_b).
+ *   idx          out, packed in (b, h) order; capacity batch * H * (B - W) int32 is always
+ *                enough
+ *   counts       out, [batch * H], b_h
+ *   idx_offsets  out, [batch * H + 1], exclusive prefix sum of counts */
+int mixkv_select(const float* scores, const int32_t* cu_seqlens_host, int32_t batch, int32_t L,
+                 const mixkv_params* p, void* workspace, size_t workspace_bytes,
+                 int32_t* idx, int32_t* counts, int32_t* idx_offsets,
+                 int32_t* status_dev, void* stream);
+
+/* The whole per-layer step of Algorithm 1: mixkv_scores, mixkv_select, then the gather:
+ * for every (b, h) the selected rows of K and V in ascending position order followed by the
+ * W window rows, packed in (b, h) order.
+ *   K_out, V_out      out, [rows, d] bf16; capacity batch * H * B rows is always enough
+ *   out_row_offsets   out, [batch * H + 1]: first output row of each (b, h); last = rows
+ *   idx_opt / counts_opt / idx_offsets_opt / s_comp_opt   optional outputs as above (NULL:
+ *                     kept in the workspace) */
+int mixkv_compress_layer(const void* K, const void* V, const void* Qwin,
+                         const int32_t* cu_seqlens_host, int32_t batch, int32_t L,
+                         const mixkv_params* p, void* workspace, size_t workspace_bytes,
+                         const float* rbar_in_opt, void* K_out, void* V_out,
+                         int32_t* out_row_offsets, int32_t* idx_opt, int32_t* counts_opt,
+                         int32_t* idx_offsets_opt, float* s_comp_opt,
+                         int32_t* status_dev, void* stream);
+
+/* Number of kernels one mixkv_compress_layer call enqueues for these parameters. */
+int mixkv_launches_per_layer(const mixkv_params* p);
+
+/* Static, human-readable name of a status code. */
+const char* mixkv_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MIXKV_H_ */

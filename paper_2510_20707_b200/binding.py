@@ -1,0 +1,226 @@
+"""ctypes binding of the MixKV C ABI (``include/mixkv.h``).
+
+Argument marshalling only: every function hands device pointers of torch tensors to the
+library entry point of the same name and returns the tensors it filled.  No arithmetic of
+the method happens here, and nothing falls back to PyTorch ops or the CPU: if
+``libmixkv.so`` is missing, :func:`load_library` raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import Dict, Optional, Sequence
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libmixkv.so")
+
+EXPORTS = ("mixkv_default_params", "mixkv_workspace_size", "mixkv_scores", "mixkv_select",
+           "mixkv_compress_layer", "mixkv_launches_per_layer", "mixkv_status_string")
+
+
+class MixKVError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        super().__init__(f"{what}: {status_string(status)} ({status})")
+        self.status = status
+
+
+class _CParams(C.Structure):
+    _fields_ = [("kv_heads", C.c_int32), ("gqa_ratio", C.c_int32), ("head_dim", C.c_int32),
+                ("window", C.c_int32), ("pool_kernel", C.c_int32), ("pool_mode", C.c_int32),
+                ("use_vnorm", C.c_int32), ("mix_mode", C.c_int32), ("budget_mode", C.c_int32),
+                ("budget", C.c_int32), ("ada_floor", C.c_float), ("eps", C.c_float),
+                ("softmax_scale", C.c_float)]
+
+
+@dataclass
+class Params:
+    """Mirror of ``mixkv_params`` (see include/mixkv.h for the meaning of each field)."""
+    kv_heads: int
+    gqa_ratio: int
+    head_dim: int = 128
+    window: int = 32
+    pool_kernel: int = 7
+    pool_mode: int = 0
+    use_vnorm: int = 1
+    mix_mode: int = 0
+    budget_mode: int = 0
+    budget: int = 64
+    ada_floor: float = 0.2
+    eps: float = 1e-6
+    softmax_scale: float = 0.0
+
+    def c(self) -> _CParams:
+        return _CParams(self.kv_heads, self.gqa_ratio, self.head_dim, self.window,
+                        self.pool_kernel, self.pool_mode, self.use_vnorm, self.mix_mode,
+                        self.budget_mode, self.budget, self.ada_floor, self.eps,
+                        self.softmax_scale)
+
+
+_lib: Optional[C.CDLL] = None
+
+
+def load_library() -> C.CDLL:
+    """Loads libmixkv.so from the package directory; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(
+                f"{LIB_PATH} not found: build it with `python -m paper_2510_20707_b200.build` "
+                "(there is no CPU or PyTorch fallback)")
+        lib = C.CDLL(LIB_PATH)
+        vp, i32, sz = C.c_void_p, C.c_int32, C.c_size_t
+        lib.mixkv_status_string.restype = C.c_char_p
+        lib.mixkv_status_string.argtypes = [C.c_int]
+        lib.mixkv_default_params.restype = None
+        lib.mixkv_default_params.argtypes = [C.POINTER(_CParams), i32, i32, i32]
+        lib.mixkv_workspace_size.argtypes = [C.POINTER(_CParams), i32, C.c_int64, i32,
+                                             C.POINTER(sz)]
+        lib.mixkv_launches_per_layer.argtypes = [C.POINTER(_CParams)]
+        lib.mixkv_scores.argtypes = [vp, vp, vp, C.POINTER(i32), i32, i32, C.POINTER(_CParams),
+                                     vp, sz, vp, vp, vp, vp, vp, vp, vp]
+        lib.mixkv_select.argtypes = [vp, C.POINTER(i32), i32, i32, C.POINTER(_CParams), vp, sz,
+                                     vp, vp, vp, vp, vp]
+        lib.mixkv_compress_layer.argtypes = [vp, vp, vp, C.POINTER(i32), i32, i32,
+                                             C.POINTER(_CParams), vp, sz, vp, vp, vp, vp, vp, vp,
+                                             vp, vp, vp, vp]
+        _lib = lib
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return load_library().mixkv_status_string(int(status)).decode()
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    assert t.is_contiguous(), "tensors handed to the library must be contiguous"
+    return t.data_ptr()
+
+
+def _cu_array(cu: Optional[Sequence[int]]):
+    if cu is None:
+        return None, 1
+    arr = (C.c_int32 * len(cu))(*[int(x) for x in cu])
+    return arr, len(cu) - 1
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream
+
+
+def workspace_size(params: Params, batch: int, total_tokens: int, max_seq_len: int) -> int:
+    out = C.c_size_t(0)
+    pc = params.c()
+    rc = load_library().mixkv_workspace_size(C.byref(pc), batch, total_tokens, max_seq_len,
+                                             C.byref(out))
+    if rc != 0:
+        raise MixKVError(rc, "mixkv_workspace_size")
+    return int(out.value)
+
+
+def launches_per_layer(params: Params) -> int:
+    pc = params.c()
+    return int(load_library().mixkv_launches_per_layer(C.byref(pc)))
+
+
+def _workspace(params, cu, Ltot, device, workspace):
+    batch = 1 if cu is None else len(cu) - 1
+    max_len = Ltot if cu is None else max(int(cu[b + 1]) - int(cu[b]) for b in range(batch))
+    need = workspace_size(params, batch, Ltot, max_len)
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=device)
+    return workspace, batch
+
+
+def scores(K: torch.Tensor, V: Optional[torch.Tensor], Q: torch.Tensor, params: Params,
+           cu_seqlens: Optional[Sequence[int]] = None, rbar_in: Optional[torch.Tensor] = None,
+           workspace: Optional[torch.Tensor] = None, stream=None,
+           want_parts: bool = True) -> Dict[str, torch.Tensor]:
+    """mixkv_scores: K, V [H, Ltot, 128] bf16, Q [batch, H*G, W, 128] bf16 (device tensors)."""
+    H, Ltot, d = K.shape
+    workspace, batch = _workspace(params, cu_seqlens, Ltot, K.device, workspace)
+    Ptot = Ltot - batch * params.window
+    f32 = dict(dtype=torch.float32, device=K.device)
+    out = {"s_comp": torch.empty((H, Ptot), **f32)}
+    if want_parts:
+        out["s_ex"] = torch.empty((H, Ptot), **f32)
+        out["s_div"] = torch.empty((H, Ptot), **f32)
+        out["rbar"] = torch.empty((batch, H), **f32)
+    status = torch.zeros(1, dtype=torch.int32, device=K.device)
+    cu, _ = _cu_array(cu_seqlens)
+    pc = params.c()
+    rc = load_library().mixkv_scores(
+        _ptr(K), _ptr(V), _ptr(Q), cu, batch, Ltot, C.byref(pc), _ptr(workspace),
+        workspace.numel(), _ptr(out["s_comp"]), _ptr(out.get("s_ex")), _ptr(out.get("s_div")),
+        _ptr(out.get("rbar")), _ptr(rbar_in), _ptr(status), _stream(stream))
+    if rc != 0:
+        raise MixKVError(rc, "mixkv_scores")
+    out["status"] = status
+    return out
+
+
+def select(s: torch.Tensor, params: Params, cu_seqlens: Optional[Sequence[int]] = None,
+           workspace: Optional[torch.Tensor] = None, stream=None) -> Dict[str, torch.Tensor]:
+    """mixkv_select on scores [H, Ptot] fp32 (device tensor)."""
+    H, Ptot = s.shape
+    batch = 1 if cu_seqlens is None else len(cu_seqlens) - 1
+    Ltot = Ptot + batch * params.window
+    workspace, batch = _workspace(params, cu_seqlens, Ltot, s.device, workspace)
+    i32 = dict(dtype=torch.int32, device=s.device)
+    cap = max(batch * H * (params.budget - params.window), 1)
+    out = {"idx": torch.empty(cap, **i32), "counts": torch.empty(batch * H, **i32),
+           "idx_offsets": torch.empty(batch * H + 1, **i32)}
+    status = torch.zeros(1, **i32)
+    cu, _ = _cu_array(cu_seqlens)
+    pc = params.c()
+    rc = load_library().mixkv_select(_ptr(s), cu, batch, Ltot, C.byref(pc), _ptr(workspace),
+                                     workspace.numel(), _ptr(out["idx"]), _ptr(out["counts"]),
+                                     _ptr(out["idx_offsets"]), _ptr(status), _stream(stream))
+    if rc != 0:
+        raise MixKVError(rc, "mixkv_select")
+    out["status"] = status
+    return out
+
+
+def compress_layer(K: torch.Tensor, V: torch.Tensor, Q: torch.Tensor, params: Params,
+                   cu_seqlens: Optional[Sequence[int]] = None,
+                   rbar_in: Optional[torch.Tensor] = None,
+                   workspace: Optional[torch.Tensor] = None, stream=None,
+                   out: Optional[Dict[str, torch.Tensor]] = None,
+                   want_aux: bool = True) -> Dict[str, torch.Tensor]:
+    """mixkv_compress_layer.  Returns K_out / V_out [batch*H*B, 128] (rows beyond
+    out_row_offsets[-1] are untouched), out_row_offsets and, if want_aux, idx / counts /
+    idx_offsets / s_comp.  `out` lets a caller reuse output tensors across calls."""
+    H, Ltot, d = K.shape
+    workspace, batch = _workspace(params, cu_seqlens, Ltot, K.device, workspace)
+    Ptot = Ltot - batch * params.window
+    if out is None:
+        i32 = dict(dtype=torch.int32, device=K.device)
+        rows = batch * H * params.budget
+        out = {"K_out": torch.empty((rows, d), dtype=torch.bfloat16, device=K.device),
+               "V_out": torch.empty((rows, d), dtype=torch.bfloat16, device=K.device),
+               "out_row_offsets": torch.empty(batch * H + 1, **i32),
+               "status": torch.zeros(1, **i32)}
+        if want_aux:
+            cap = max(batch * H * (params.budget - params.window), 1)
+            out["idx"] = torch.empty(cap, **i32)
+            out["counts"] = torch.empty(batch * H, **i32)
+            out["idx_offsets"] = torch.empty(batch * H + 1, **i32)
+            out["s_comp"] = torch.empty((H, Ptot), dtype=torch.float32, device=K.device)
+    cu, _ = _cu_array(cu_seqlens)
+    pc = params.c()
+    rc = load_library().mixkv_compress_layer(
+        _ptr(K), _ptr(V), _ptr(Q), cu, batch, Ltot, C.byref(pc), _ptr(workspace),
+        workspace.numel(), _ptr(rbar_in), _ptr(out["K_out"]), _ptr(out["V_out"]),
+        _ptr(out["out_row_offsets"]), _ptr(out.get("idx")), _ptr(out.get("counts")),
+        _ptr(out.get("idx_offsets")), _ptr(out.get("s_comp")), _ptr(out["status"]),
+        _stream(stream))
+    if rc != 0:
+        raise MixKVError(rc, "mixkv_compress_layer")
+    return out

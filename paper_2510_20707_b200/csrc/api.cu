@@ -1,0 +1,270 @@
+// C ABI of the MixKV library: argument checks, workspace carve-up, kernel sequencing.
+#include <math.h>
+#include <string.h>
+
+#include "common.cuh"
+
+namespace mixkv {
+
+namespace {
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+int check_params(const mixkv_params* p) {
+  if (!p) return MIXKV_ERR_INVALID_ARG;
+  if (p->kv_heads < 1 || p->gqa_ratio < 1 || p->window < 1) return MIXKV_ERR_INVALID_ARG;
+  if (p->pool_kernel < 1 || (p->pool_kernel & 1) == 0) return MIXKV_ERR_INVALID_ARG;
+  if (p->pool_mode != MIXKV_POOL_AVG && p->pool_mode != MIXKV_POOL_MAX) return MIXKV_ERR_INVALID_ARG;
+  if (p->mix_mode < 0 || p->mix_mode > 3) return MIXKV_ERR_INVALID_ARG;
+  if (p->budget_mode != MIXKV_BUDGET_FIXED && p->budget_mode != MIXKV_BUDGET_ADAPTIVE)
+    return MIXKV_ERR_INVALID_ARG;
+  if (p->budget <= p->window) return MIXKV_ERR_INVALID_ARG;
+  if (!(p->ada_floor >= 0.f && p->ada_floor <= 1.f)) return MIXKV_ERR_INVALID_ARG;
+  if (!(p->eps >= 0.f) || !(p->softmax_scale >= 0.f)) return MIXKV_ERR_INVALID_ARG;
+  if (p->head_dim != kHeadDim) return MIXKV_ERR_UNSUPPORTED;
+  const long long nq = (long long)p->gqa_ratio * p->window;
+  if (nq < 16 || nq > kMaxNQ || (nq % 16) != 0) return MIXKV_ERR_UNSUPPORTED;
+  if (p->pool_kernel > 63) return MIXKV_ERR_UNSUPPORTED;
+  if (p->kv_heads > 64) return MIXKV_ERR_UNSUPPORTED;
+  return MIXKV_OK;
+}
+
+// Builds the sequence table from the host offsets (or a single length).
+int build_table(const mixkv_params* p, const int32_t* cu, int batch, int L, SeqTable* st,
+                int* max_len) {
+  if (batch < 1) return MIXKV_ERR_INVALID_ARG;
+  if (batch > kMaxBatch) return MIXKV_ERR_UNSUPPORTED;
+  if (!cu && batch != 1) return MIXKV_ERR_INVALID_ARG;
+  memset(st, 0, sizeof(*st));
+  st->batch = batch;
+  st->H = p->kv_heads;
+  st->G = p->gqa_ratio;
+  st->W = p->window;
+  st->NQ = p->gqa_ratio * p->window;
+  int mx = 0;
+  for (int b = 0; b <= batch; ++b) st->cu[b] = cu ? cu[b] : (b == 0 ? 0 : L);
+  if (st->cu[0] != 0) return MIXKV_ERR_INVALID_ARG;
+  for (int b = 0; b < batch; ++b) {
+    const long long len = (long long)st->cu[b + 1] - st->cu[b];
+    if (len < p->window + 1 || len < 2) return MIXKV_ERR_INVALID_ARG;
+    if (len > mx) mx = (int)len;
+    st->chunk_start[b + 1] = st->chunk_start[b] + (int)((len + kChunk - 1) / kChunk);
+    st->pchunk_start[b + 1] =
+        st->pchunk_start[b] + (int)((len - p->window + kPChunk - 1) / kPChunk);
+  }
+  st->Ltot = st->cu[batch];
+  st->Ptot = st->Ltot - batch * p->window;
+  st->chunks_total = st->chunk_start[batch];
+  st->pchunks_total = st->pchunk_start[batch];
+  *max_len = mx;
+  return MIXKV_OK;
+}
+
+// Upper bound of selected (non-window) rows over the whole batch.
+long long idx_capacity(const mixkv_params* p, const SeqTable& st) {
+  long long cap = 0;
+  for (int b = 0; b < st.batch; ++b) {
+    const long long P = st.cu[b + 1] - st.cu[b] - st.W;
+    long long per_seq = (long long)st.H * (p->budget - p->window);
+    if (per_seq > st.H * P) per_seq = st.H * P;
+    cap += per_seq;
+  }
+  return cap;
+}
+
+// Lays the workspace out; with base == nullptr only the size is computed.
+void carve(const mixkv_params* p, const SeqTable& st, unsigned char* base, Workspace* ws) {
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    unsigned char* ptr = base ? base + off : nullptr;
+    off = align_up(off + bytes, 256);
+    return ptr;
+  };
+  const size_t H = st.H, BH = (size_t)st.batch * st.H;
+  ws->kinv = (float*)take(H * st.Ltot * 4);
+  ws->vnorm = (float*)take(H * st.Ptot * 4);
+  ws->s_ex_raw = (float*)take(H * st.Ptot * 4);
+  ws->s_ex = (float*)take(H * st.Ptot * 4);
+  ws->s_div = (float*)take(H * st.Ptot * 4);
+  ws->s_comp = (float*)take(H * st.Ptot * 4);
+  ws->rowstat = (float2*)take(H * st.chunks_total * st.NQ * 8);
+  ws->ksum = (float*)take(H * st.chunks_total * kHeadDim * 4);
+  ws->vstat = (float4*)take(H * st.chunks_total * 16);
+  ws->dstat = (float4*)take(H * st.chunks_total * 16);
+  ws->exsum = (float*)take(H * st.pchunks_total * 4);
+  ws->bq = (float*)take(BH * st.NQ * 4);
+  ws->kbar_rows = (__nv_bfloat16*)take(BH * 3 * kHeadDim * 2);
+  ws->rbar = (float*)take(BH * 4);
+  ws->vfinal = (float4*)take(BH * 16);
+  ws->counts = (int*)take(BH * 4);
+  ws->idx_offsets = (int*)take((BH + 1) * 4);
+  ws->idx = (int*)take((size_t)idx_capacity(p, st) * 4);
+  ws->status = (int*)take(4);
+  ws->bytes = off;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int make_ctx(const mixkv_params* p, const int32_t* cu, int batch, int L, void* workspace,
+             size_t workspace_bytes, void* stream, LaunchCtx* c) {
+  int rc = check_params(p);
+  if (rc != MIXKV_OK) return rc;
+  int max_len = 0;
+  rc = build_table(p, cu, batch, L, &c->st, &max_len);
+  if (rc != MIXKV_OK) return rc;
+  if (!workspace || !aligned16(workspace)) return MIXKV_ERR_INVALID_ARG;
+  carve(p, c->st, (unsigned char*)workspace, &c->ws);
+  if (c->ws.bytes > workspace_bytes) return MIXKV_ERR_WORKSPACE_TOO_SMALL;
+  c->p = *p;
+  const float scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)kHeadDim);
+  c->scale_log2e = scale * kLog2e;
+  c->max_seq_len = max_len;
+  c->max_prefix = max_len - p->window;
+  c->stream = (cudaStream_t)stream;
+  return MIXKV_OK;
+}
+
+int enqueue_scores(const LaunchCtx& c, const void* K, const void* V, const void* Q, float* s_comp,
+                   float* s_ex_out, float* s_div_out, float* rbar_out, const float* rbar_in) {
+  float* s_ex = s_ex_out ? s_ex_out : c.ws.s_ex;
+  float* s_div = s_div_out ? s_div_out : c.ws.s_div;
+  if (launch_pass1(c, K, V, Q) != cudaSuccess) return MIXKV_ERR_CUDA;
+  if (launch_finalize(c) != cudaSuccess) return MIXKV_ERR_CUDA;
+  if (launch_pass2(c, K, Q, s_div) != cudaSuccess) return MIXKV_ERR_CUDA;
+  if (launch_pool(c, s_ex) != cudaSuccess) return MIXKV_ERR_CUDA;
+  if (launch_mix(c, s_ex, s_div, rbar_in, s_comp, rbar_out) != cudaSuccess) return MIXKV_ERR_CUDA;
+  return MIXKV_OK;
+}
+
+int enqueue_select(const LaunchCtx& c, const float* scores, int* idx, int* counts,
+                   int* idx_offsets, int* out_row_offsets) {
+  if (launch_budget(c, scores, counts) != cudaSuccess) return MIXKV_ERR_CUDA;
+  if (launch_select(c, scores, counts, idx, idx_offsets, out_row_offsets) != cudaSuccess)
+    return MIXKV_ERR_CUDA;
+  return MIXKV_OK;
+}
+
+}  // namespace
+}  // namespace mixkv
+
+using namespace mixkv;
+
+extern "C" {
+
+void mixkv_default_params(mixkv_params* p, int32_t kv_heads, int32_t gqa_ratio, int32_t budget) {
+  if (!p) return;
+  memset(p, 0, sizeof(*p));
+  p->kv_heads = kv_heads;
+  p->gqa_ratio = gqa_ratio;
+  p->head_dim = kHeadDim;
+  p->window = 32;
+  p->pool_kernel = 7;
+  p->pool_mode = MIXKV_POOL_AVG;
+  p->use_vnorm = 1;
+  p->mix_mode = MIXKV_MIX_HEADWISE;
+  p->budget_mode = MIXKV_BUDGET_FIXED;
+  p->budget = budget;
+  p->ada_floor = 0.2f;
+  p->eps = 1e-6f;
+  p->softmax_scale = 0.f;
+}
+
+int mixkv_workspace_size(const mixkv_params* p, int32_t batch, int64_t total_tokens,
+                         int32_t max_seq_len, size_t* bytes) {
+  int rc = check_params(p);
+  if (rc != MIXKV_OK) return rc;
+  if (!bytes || batch < 1 || total_tokens < batch || max_seq_len < 1) return MIXKV_ERR_INVALID_ARG;
+  if (batch > kMaxBatch) return MIXKV_ERR_UNSUPPORTED;
+  if (total_tokens > 0x7fffffffLL / 2) return MIXKV_ERR_UNSUPPORTED;
+  // a table with the worst-case chunk counts for these totals
+  SeqTable st;
+  memset(&st, 0, sizeof(st));
+  st.batch = batch;
+  st.H = p->kv_heads;
+  st.G = p->gqa_ratio;
+  st.W = p->window;
+  st.NQ = p->gqa_ratio * p->window;
+  st.Ltot = (int)total_tokens;
+  st.Ptot = (int)total_tokens;  // >= the true candidate count
+  st.chunks_total = (int)(total_tokens / kChunk) + batch;
+  st.pchunks_total = (int)(total_tokens / kPChunk) + batch;
+  // capacity of the index list: every sequence at its budget
+  st.cu[0] = 0;
+  for (int b = 1; b <= batch; ++b) st.cu[b] = 0;
+  Workspace ws;
+  carve(p, st, nullptr, &ws);
+  // idx_capacity() saw empty sequences above; add the true bound
+  const size_t idx_bytes = (size_t)batch * p->kv_heads * (size_t)(p->budget - p->window) * 4;
+  *bytes = ws.bytes + align_up(idx_bytes, 256) + 256;
+  return MIXKV_OK;
+}
+
+int mixkv_scores(const void* K, const void* V, const void* Qwin, const int32_t* cu_seqlens_host,
+                 int32_t batch, int32_t L, const mixkv_params* p, void* workspace,
+                 size_t workspace_bytes, float* s_comp, float* s_ex_opt, float* s_div_opt,
+                 float* rbar_opt, const float* rbar_in_opt, int32_t* status_dev, void* stream) {
+  (void)status_dev;
+  LaunchCtx c;
+  int rc = make_ctx(p, cu_seqlens_host, batch, L, workspace, workspace_bytes, stream, &c);
+  if (rc != MIXKV_OK) return rc;
+  if (!K || !Qwin || !s_comp || (p->use_vnorm && !V)) return MIXKV_ERR_INVALID_ARG;
+  if (!aligned16(K) || !aligned16(Qwin) || (V && !aligned16(V))) return MIXKV_ERR_INVALID_ARG;
+  return enqueue_scores(c, K, V, Qwin, s_comp, s_ex_opt, s_div_opt, rbar_opt, rbar_in_opt);
+}
+
+int mixkv_select(const float* scores, const int32_t* cu_seqlens_host, int32_t batch, int32_t L,
+                 const mixkv_params* p, void* workspace, size_t workspace_bytes, int32_t* idx,
+                 int32_t* counts, int32_t* idx_offsets, int32_t* status_dev, void* stream) {
+  (void)status_dev;
+  LaunchCtx c;
+  int rc = make_ctx(p, cu_seqlens_host, batch, L, workspace, workspace_bytes, stream, &c);
+  if (rc != MIXKV_OK) return rc;
+  if (!scores || !idx || !counts || !idx_offsets) return MIXKV_ERR_INVALID_ARG;
+  return enqueue_select(c, scores, idx, counts, idx_offsets, nullptr);
+}
+
+int mixkv_compress_layer(const void* K, const void* V, const void* Qwin,
+                         const int32_t* cu_seqlens_host, int32_t batch, int32_t L,
+                         const mixkv_params* p, void* workspace, size_t workspace_bytes,
+                         const float* rbar_in_opt, void* K_out, void* V_out,
+                         int32_t* out_row_offsets, int32_t* idx_opt, int32_t* counts_opt,
+                         int32_t* idx_offsets_opt, float* s_comp_opt, int32_t* status_dev,
+                         void* stream) {
+  (void)status_dev;
+  LaunchCtx c;
+  int rc = make_ctx(p, cu_seqlens_host, batch, L, workspace, workspace_bytes, stream, &c);
+  if (rc != MIXKV_OK) return rc;
+  if (!K || !V || !Qwin || !K_out || !V_out || !out_row_offsets) return MIXKV_ERR_INVALID_ARG;
+  if (!aligned16(K) || !aligned16(V) || !aligned16(Qwin) || !aligned16(K_out) || !aligned16(V_out))
+    return MIXKV_ERR_INVALID_ARG;
+  float* s_comp = s_comp_opt ? s_comp_opt : c.ws.s_comp;
+  int* idx = idx_opt ? idx_opt : c.ws.idx;
+  int* counts = counts_opt ? counts_opt : c.ws.counts;
+  int* offs = idx_offsets_opt ? idx_offsets_opt : c.ws.idx_offsets;
+  rc = enqueue_scores(c, K, V, Qwin, s_comp, nullptr, nullptr, nullptr, rbar_in_opt);
+  if (rc != MIXKV_OK) return rc;
+  rc = enqueue_select(c, s_comp, idx, counts, offs, out_row_offsets);
+  if (rc != MIXKV_OK) return rc;
+  if (launch_gather(c, K, V, idx, offs, out_row_offsets, K_out, V_out) != cudaSuccess)
+    return MIXKV_ERR_CUDA;
+  return MIXKV_OK;
+}
+
+int mixkv_launches_per_layer(const mixkv_params* p) {
+  (void)p;
+  return 8;  // pass1, finalize, pass2, pool, mix, budget, select, gather
+}
+
+const char* mixkv_status_string(int status) {
+  switch (status) {
+    case MIXKV_OK: return "ok";
+    case MIXKV_ERR_INVALID_ARG: return "invalid argument";
+    case MIXKV_ERR_UNSUPPORTED: return "unsupported configuration";
+    case MIXKV_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case MIXKV_ERR_CUDA: return "CUDA error";
+    case MIXKV_ERR_TIMEOUT: return "device-side bounded wait expired";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"

@@ -1,0 +1,109 @@
+// Shared declarations of the MixKV CUDA library (sm_100a): problem description handed to
+// every kernel, the workspace carve-up, and small device helpers.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "mixkv.h"
+
+namespace mixkv {
+
+constexpr int kHeadDim = 128;        // d, fixed
+constexpr int kMaxBatch = 64;        // sequences per call
+constexpr int kMaxNQ = 240;          // G*W upper bound (16 spare rows carry the mean key)
+constexpr int kChunk = 512;          // keys per CTA in the two K passes
+constexpr int kPChunk = 2048;        // candidate positions per CTA in pool / mix
+constexpr int kExtraRows = 16;       // rows appended to the query tile in pass 2
+constexpr float kLog2e = 1.4426950408889634f;
+
+// Everything a kernel needs to find its slice of the ragged batch.
+struct SeqTable {
+  int batch, H, G, W, NQ;
+  int Ltot, Ptot;
+  int chunks_total;                  // sum over sequences of ceil(L_b / kChunk)
+  int pchunks_total;                 // sum over sequences of ceil(P_b / kPChunk)
+  int cu[kMaxBatch + 1];             // sequence offsets into Ltot
+  int chunk_start[kMaxBatch + 1];    // prefix sum of key chunks
+  int pchunk_start[kMaxBatch + 1];   // prefix sum of candidate chunks
+};
+
+// Device workspace carve-up (all pointers into the caller's workspace).
+struct Workspace {
+  float* kinv;        // [H, Ltot]   1 / |K_i|  (0 for a zero key)
+  float* vnorm;       // [H, Ptot]   |V_i|
+  float* s_ex_raw;    // [H, Ptot]   window attention score before pooling
+  float* s_ex;        // [H, Ptot]   after pooling
+  float* s_div;       // [H, Ptot]
+  float* s_comp;      // [H, Ptot]
+  float2* rowstat;    // [H, chunks_total, NQ]  per-chunk softmax (max, sum) in log2 units
+  float* ksum;        // [H, chunks_total, d]   per-chunk sum of unit keys
+  float4* vstat;      // [H, chunks_total]      (min, max, sum, -) of |V_i| over candidates
+  float4* dstat;      // [H, chunks_total]      (min, max, sum, -) of s_div over candidates
+  float* exsum;       // [H, pchunks_total]     per-chunk sum of pooled s_ex
+  float* bq;          // [batch, H, NQ]  log2 normaliser of each window row (incl. 1/W)
+  __nv_bfloat16* kbar_rows;  // [batch, H, 3, d]  mean unit key split into bf16 hi/lo/lo2
+  float* rbar;        // [batch, H]
+  float4* vfinal;     // [batch, H] (min, max, sum, -) of |V_i|
+  int* counts;        // [batch*H]
+  int* idx_offsets;   // [batch*H + 1]
+  int* idx;           // [batch*H*(B-W)] (or more for adaptive)
+  int* status;        // [1]
+  size_t bytes;
+};
+
+struct LaunchCtx {
+  SeqTable st;
+  Workspace ws;
+  mixkv_params p;
+  float scale_log2e;   // softmax scale * log2(e)
+  int max_seq_len;
+  int max_prefix;
+  cudaStream_t stream;
+};
+
+// ---- kernels (defined in the .cu files) ------------------------------------------
+cudaError_t launch_pass1(const LaunchCtx& c, const void* K, const void* V, const void* Q);
+cudaError_t launch_finalize(const LaunchCtx& c);
+cudaError_t launch_pass2(const LaunchCtx& c, const void* K, const void* Q, float* s_div_out);
+cudaError_t launch_pool(const LaunchCtx& c, float* s_ex_out);
+cudaError_t launch_mix(const LaunchCtx& c, const float* s_ex, const float* s_div,
+                       const float* rbar_in, float* s_comp, float* rbar_out);
+cudaError_t launch_budget(const LaunchCtx& c, const float* scores, int* counts);
+cudaError_t launch_select(const LaunchCtx& c, const float* scores, const int* counts, int* idx,
+                          int* idx_offsets, int* out_row_offsets);
+cudaError_t launch_gather(const LaunchCtx& c, const void* K, const void* V, const int* idx,
+                          const int* idx_offsets, const int* out_row_offsets, void* K_out,
+                          void* V_out);
+
+// ---- device helpers ----------------------------------------------------------------
+__device__ __forceinline__ int find_seq(const int* start, int batch, int x) {
+  int b = 0;
+  while (b + 1 < batch && x >= start[b + 1]) ++b;
+  return b;
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_min(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fminf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+}  // namespace mixkv

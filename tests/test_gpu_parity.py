@@ -1,0 +1,118 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the
+same seeded inputs (tolerances in tests/parity.py)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2510_20707_b200 import binding, synth
+from parity import (check_rbar, check_scores, check_selection, params_pair, run_layer_parity,
+                    to_bits, to_dev)
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("variant", ["literal", "calibrated"])
+def test_c1_full_layer(variant):
+    run_layer_parity(synth.CONFIGS["C1"], 0, variant)
+
+
+@pytest.mark.parametrize("H,G,W,L,B,pool", [
+    (1, 1, 16, 17, 17, 1),        # a single candidate position
+    (2, 2, 8, 33, 12, 3),
+    (2, 1, 16, 257, 40, 7),
+    (3, 3, 16, 1000, 100, 5),     # several chunks with a ragged tail
+    (1, 7, 32, 513, 64, 7),       # one key past a chunk boundary
+    (2, 4, 32, 1537, 96, 7),
+    (1, 15, 16, 700, 80, 9),      # G*W = 240, the largest supported tile
+])
+def test_odd_shapes(H, G, W, L, B, pool):
+    wl = synth.small_workload(H=H, G=G, W=W, seq_lens=(L,), pool_kernel=pool, budget=B, seed=L)
+    run_layer_parity(wl)
+
+
+def test_ragged_batch_fixed_and_adaptive():
+    wl = synth.small_workload(H=4, G=2, W=16, seq_lens=(300, 1025, 47, 640), pool_kernel=7,
+                              budget=48, seed=5)
+    run_layer_parity(wl)
+    run_layer_parity(synth.with_budget(wl, 48, budget_mode=1), variant="calibrated")
+
+
+@pytest.mark.parametrize("kw", [
+    dict(pool_mode=1), dict(use_vnorm=0), dict(mix_mode=1), dict(mix_mode=2), dict(mix_mode=3),
+    dict(use_vnorm=0, mix_mode=1), dict(eps=1e-3), dict(softmax_scale=0.05),
+])
+def test_modes(kw):
+    wl = synth.small_workload(H=2, G=2, W=16, seq_lens=(900,), pool_kernel=7, budget=80, seed=11)
+    run_layer_parity(wl, variant="calibrated", **kw)
+
+
+def test_budget_at_least_L_keeps_everything():
+    wl = synth.small_workload(H=2, G=2, W=16, seq_lens=(200,), budget=200, seed=2)
+    x = synth.make_layer(wl, 0)
+    _, pg = params_pair(wl)
+    out = binding.compress_layer(to_dev(x["K"]), to_dev(x["V"]), to_dev(x["Q"]), pg)
+    torch.cuda.synchronize()
+    assert out["out_row_offsets"].tolist() == [0, 200, 400]
+    assert np.array_equal(to_bits(out["K_out"]).reshape(2, 200, 128), x["K"])
+    assert np.array_equal(to_bits(out["V_out"]).reshape(2, 200, 128), x["V"])
+
+
+def test_offline_head_weights():
+    wl = synth.small_workload(H=2, G=2, W=16, seq_lens=(500,), budget=60, seed=4)
+    x = synth.make_layer(wl, 0, "calibrated")
+    po, pg = params_pair(wl)
+    rin = np.array([[0.15, 0.85]], np.float32)
+    ref = oracle.scores(x["K"], x["V"], x["Q"], po, rbar_in=rin)
+    got = binding.scores(to_dev(x["K"]), to_dev(x["V"]), to_dev(x["Q"]), pg,
+                         rbar_in=torch.from_numpy(rin).cuda())
+    check_scores("s_comp", got["s_comp"].cpu().numpy(), ref["s_comp"], wl.cu_seqlens, 16)
+    check_rbar(got["rbar"].cpu().numpy(), ref["rbar"].astype(np.float64))
+
+
+def test_select_with_ties_is_exact():
+    # on caller-supplied scores the selection is integer work: bit-identical to the oracle
+    rng = np.random.default_rng(0)
+    H, P, W = 3, 5000, 16
+    s = rng.integers(0, 50, size=(H, P)).astype(np.float32)
+    s[1] = 1.0                                                # a head of all-equal scores
+    s[2, ::7] = -0.0
+    for mode in (0, 1):
+        po = oracle.Params(kv_heads=H, gqa_ratio=1, window=W, budget=W + 333, budget_mode=mode)
+        pg = binding.Params(kv_heads=H, gqa_ratio=1, window=W, budget=W + 333, budget_mode=mode)
+        ref = oracle.select(s, po)
+        got = binding.select(torch.from_numpy(s).cuda(), pg)
+        offs = got["idx_offsets"].cpu().numpy()
+        assert np.array_equal(got["counts"].cpu().numpy(), ref["counts"].reshape(-1))
+        assert np.array_equal(offs, ref["idx_offsets"])
+        assert np.array_equal(got["idx"].cpu().numpy()[:offs[-1]], ref["idx"])
+
+
+def test_identical_keys_head():
+    # r = 1: the mix is pure diversity, whose spread is rounding noise; only the things
+    # that stay well defined are checked (rbar, the count, valid ascending indices)
+    H, G, W, L = 1, 1, 16, 300
+    rng = np.random.default_rng(3)
+    K = np.tile(rng.standard_normal(128).astype(np.float32), (H, L, 1))
+    V = rng.standard_normal((H, L, 128)).astype(np.float32)
+    Q = rng.standard_normal((1, G, W, 128)).astype(np.float32)
+    pg = binding.Params(kv_heads=H, gqa_ratio=G, window=W, budget=48)
+    out = binding.compress_layer(to_dev(synth.f32_to_bf16_bits(K)), to_dev(synth.f32_to_bf16_bits(V)),
+                                 to_dev(synth.f32_to_bf16_bits(Q)), pg)
+    torch.cuda.synchronize()
+    idx = out["idx"].cpu().numpy()[:32]
+    assert out["counts"].tolist() == [32] and (np.diff(idx) > 0).all() and idx.max() < L - W
+
+
+@pytest.mark.parametrize("name,layer", [("C2", 0), ("C2", 27), ("C5", 0)])
+def test_full_size_layers(name, layer):
+    run_layer_parity(synth.CONFIGS[name], layer, "calibrated")
+
+
+def test_c4_ragged_adaptive_layer():
+    run_layer_parity(synth.CONFIGS["C4"], 0, "calibrated")
+
+
+@pytest.mark.parametrize("name", ["C3", "C3b"])
+def test_c3_long_video_layer(name):
+    run_layer_parity(synth.CONFIGS[name], 13, "calibrated")
