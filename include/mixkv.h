@@ -134,8 +134,25 @@ int mixkv_compress_layer(const void* K, const void* V, const void* Qwin,
                          int32_t* idx_offsets_opt, float* s_comp_opt,
                          int32_t* status_dev, void* stream);
 
-/* Number of kernels one mixkv_compress_layer call enqueues for these parameters. */
+/* Measurement hook (no counterpart in the paper): mixkv_compress_layer with CUDA events
+ * recorded on `stream` around its kernels.  events_host is a HOST array of n_events
+ * cudaEvent_t handles created by the caller with timing enabled: events_host[i] is recorded
+ * just before the i-th kernel and events_host[k] after the last of the k kernels
+ * (k = mixkv_launches_per_layer); entries beyond n_events are skipped, so n_events = 2
+ * brackets the first kernel only.  Everything else is as mixkv_compress_layer. */
+int mixkv_compress_layer_traced(const void* K, const void* V, const void* Qwin,
+                                const int32_t* cu_seqlens_host, int32_t batch, int32_t L,
+                                const mixkv_params* p, void* workspace, size_t workspace_bytes,
+                                const float* rbar_in_opt, void* K_out, void* V_out,
+                                int32_t* out_row_offsets, int32_t* idx_opt, int32_t* counts_opt,
+                                int32_t* idx_offsets_opt, float* s_comp_opt,
+                                int32_t* status_dev, void* stream,
+                                void* const* events_host, int32_t n_events);
+
+/* Number of kernels one mixkv_compress_layer call enqueues for these parameters, and the
+ * name of the i-th of them (NULL when i is out of range). */
 int mixkv_launches_per_layer(const mixkv_params* p);
+const char* mixkv_stage_name(const mixkv_params* p, int32_t i);
 
 /* Static, human-readable name of a status code. */
 const char* mixkv_status_string(int status);

@@ -18,7 +18,8 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libmixkv.so")
 
 EXPORTS = ("mixkv_default_params", "mixkv_workspace_size", "mixkv_scores", "mixkv_select",
-           "mixkv_compress_layer", "mixkv_launches_per_layer", "mixkv_status_string")
+           "mixkv_compress_layer", "mixkv_compress_layer_traced", "mixkv_launches_per_layer",
+           "mixkv_stage_name", "mixkv_status_string")
 
 
 class MixKVError(RuntimeError):
@@ -86,6 +87,10 @@ def load_library() -> C.CDLL:
         lib.mixkv_compress_layer.argtypes = [vp, vp, vp, C.POINTER(i32), i32, i32,
                                              C.POINTER(_CParams), vp, sz, vp, vp, vp, vp, vp, vp,
                                              vp, vp, vp, vp]
+        lib.mixkv_compress_layer_traced.argtypes = lib.mixkv_compress_layer.argtypes + [
+            C.POINTER(vp), i32]
+        lib.mixkv_stage_name.restype = C.c_char_p
+        lib.mixkv_stage_name.argtypes = [C.POINTER(_CParams), i32]
         _lib = lib
     return _lib
 
@@ -127,6 +132,12 @@ def workspace_size(params: Params, batch: int, total_tokens: int, max_seq_len: i
 def launches_per_layer(params: Params) -> int:
     pc = params.c()
     return int(load_library().mixkv_launches_per_layer(C.byref(pc)))
+
+
+def stage_names(params: Params):
+    pc = params.c()
+    lib = load_library()
+    return [lib.mixkv_stage_name(C.byref(pc), i).decode() for i in range(launches_per_layer(params))]
 
 
 def _workspace(params, cu, Ltot, device, workspace):
@@ -193,7 +204,7 @@ def compress_layer(K: torch.Tensor, V: torch.Tensor, Q: torch.Tensor, params: Pa
                    rbar_in: Optional[torch.Tensor] = None,
                    workspace: Optional[torch.Tensor] = None, stream=None,
                    out: Optional[Dict[str, torch.Tensor]] = None,
-                   want_aux: bool = True) -> Dict[str, torch.Tensor]:
+                   want_aux: bool = True, trace_events=None) -> Dict[str, torch.Tensor]:
     """mixkv_compress_layer.  Returns K_out / V_out [batch*H*B, 128] (rows beyond
     out_row_offsets[-1] are untouched), out_row_offsets and, if want_aux, idx / counts /
     idx_offsets / s_comp.  `out` lets a caller reuse output tensors across calls."""
@@ -215,12 +226,16 @@ def compress_layer(K: torch.Tensor, V: torch.Tensor, Q: torch.Tensor, params: Pa
             out["s_comp"] = torch.empty((H, Ptot), dtype=torch.float32, device=K.device)
     cu, _ = _cu_array(cu_seqlens)
     pc = params.c()
-    rc = load_library().mixkv_compress_layer(
-        _ptr(K), _ptr(V), _ptr(Q), cu, batch, Ltot, C.byref(pc), _ptr(workspace),
-        workspace.numel(), _ptr(rbar_in), _ptr(out["K_out"]), _ptr(out["V_out"]),
-        _ptr(out["out_row_offsets"]), _ptr(out.get("idx")), _ptr(out.get("counts")),
-        _ptr(out.get("idx_offsets")), _ptr(out.get("s_comp")), _ptr(out["status"]),
-        _stream(stream))
+    args = (_ptr(K), _ptr(V), _ptr(Q), cu, batch, Ltot, C.byref(pc), _ptr(workspace),
+            workspace.numel(), _ptr(rbar_in), _ptr(out["K_out"]), _ptr(out["V_out"]),
+            _ptr(out["out_row_offsets"]), _ptr(out.get("idx")), _ptr(out.get("counts")),
+            _ptr(out.get("idx_offsets")), _ptr(out.get("s_comp")), _ptr(out["status"]),
+            _stream(stream))
+    if trace_events is None:
+        rc = load_library().mixkv_compress_layer(*args)
+    else:
+        # trace_events: a ctypes array of cudaEvent_t handles (see mixkv_compress_layer_traced)
+        rc = load_library().mixkv_compress_layer_traced(*args, trace_events, len(trace_events))
     if rc != 0:
         raise MixKVError(rc, "mixkv_compress_layer")
     return out

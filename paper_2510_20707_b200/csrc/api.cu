@@ -48,14 +48,20 @@ int build_table(const mixkv_params* p, const int32_t* cu, int batch, int L, SeqT
     const long long len = (long long)st->cu[b + 1] - st->cu[b];
     if (len < p->window + 1 || len < 2) return MIXKV_ERR_INVALID_ARG;
     if (len > mx) mx = (int)len;
-    st->chunk_start[b + 1] = st->chunk_start[b] + (int)((len + kChunk - 1) / kChunk);
     st->pchunk_start[b + 1] =
         st->pchunk_start[b] + (int)((len - p->window + kPChunk - 1) / kPChunk);
+    st->tile1_start[b + 1] = st->tile1_start[b] + st->H * (int)((len + kTile - 1) / kTile);
+    st->tile2_start[b + 1] =
+        st->tile2_start[b] + st->H * (int)((len - p->window + kTile - 1) / kTile);
   }
   st->Ltot = st->cu[batch];
   st->Ptot = st->Ltot - batch * p->window;
-  st->chunks_total = st->chunk_start[batch];
   st->pchunks_total = st->pchunk_start[batch];
+  st->nt1 = st->tile1_start[batch];
+  st->nt2 = st->tile2_start[batch];
+  const int sms = device_sm_count();
+  st->g1 = st->nt1 < sms ? st->nt1 : sms;
+  st->g2 = st->nt2 < sms ? st->nt2 : sms;
   *max_len = mx;
   return MIXKV_OK;
 }
@@ -87,10 +93,10 @@ void carve(const mixkv_params* p, const SeqTable& st, unsigned char* base, Works
   ws->s_ex = (float*)take(H * st.Ptot * 4);
   ws->s_div = (float*)take(H * st.Ptot * 4);
   ws->s_comp = (float*)take(H * st.Ptot * 4);
-  ws->rowstat = (float2*)take(H * st.chunks_total * st.NQ * 8);
-  ws->ksum = (float*)take(H * st.chunks_total * kHeadDim * 4);
-  ws->vstat = (float4*)take(H * st.chunks_total * 16);
-  ws->dstat = (float4*)take(H * st.chunks_total * 16);
+  ws->rowstat = (float2*)take((size_t)st.nt1 * 2 * st.NQ * 8);
+  ws->ksum = (float*)take((size_t)st.nt1 * kHeadDim * 4);
+  ws->vstat = (float4*)take((size_t)st.nt1 * 16);
+  ws->dstat = (float4*)take((size_t)st.nt2 * 16);
   ws->exsum = (float*)take(H * st.pchunks_total * 4);
   ws->bq = (float*)take(BH * st.NQ * 4);
   ws->kbar_rows = (__nv_bfloat16*)take(BH * 3 * kHeadDim * 2);
@@ -121,24 +127,33 @@ int make_ctx(const mixkv_params* p, const int32_t* cu, int batch, int L, void* w
   c->max_seq_len = max_len;
   c->max_prefix = max_len - p->window;
   c->stream = (cudaStream_t)stream;
+  c->trace_events = nullptr;
+  c->n_trace_events = 0;
+  c->stage = 0;
   return MIXKV_OK;
 }
 
 int enqueue_scores(const LaunchCtx& c, const void* K, const void* V, const void* Q, float* s_comp,
-                   float* s_ex_out, float* s_div_out, float* rbar_out, const float* rbar_in) {
+                   float* s_ex_out, float* s_div_out, float* rbar_out, const float* rbar_in,
+                   int* status) {
   float* s_ex = s_ex_out ? s_ex_out : c.ws.s_ex;
   float* s_div = s_div_out ? s_div_out : c.ws.s_div;
-  if (launch_pass1(c, K, V, Q) != cudaSuccess) return MIXKV_ERR_CUDA;
-  if (launch_finalize(c) != cudaSuccess) return MIXKV_ERR_CUDA;
-  if (launch_pass2(c, K, Q, s_div) != cudaSuccess) return MIXKV_ERR_CUDA;
+  c.mark();
+  if (launch_pass1(c, K, V, Q, status) != cudaSuccess) return MIXKV_ERR_CUDA;
+  c.mark();
+  if (launch_pass2(c, K, Q, s_div, status) != cudaSuccess) return MIXKV_ERR_CUDA;
+  c.mark();
   if (launch_pool(c, s_ex) != cudaSuccess) return MIXKV_ERR_CUDA;
+  c.mark();
   if (launch_mix(c, s_ex, s_div, rbar_in, s_comp, rbar_out) != cudaSuccess) return MIXKV_ERR_CUDA;
   return MIXKV_OK;
 }
 
 int enqueue_select(const LaunchCtx& c, const float* scores, int* idx, int* counts,
                    int* idx_offsets, int* out_row_offsets) {
+  c.mark();
   if (launch_budget(c, scores, counts) != cudaSuccess) return MIXKV_ERR_CUDA;
+  c.mark();
   if (launch_select(c, scores, counts, idx, idx_offsets, out_row_offsets) != cudaSuccess)
     return MIXKV_ERR_CUDA;
   return MIXKV_OK;
@@ -186,8 +201,8 @@ int mixkv_workspace_size(const mixkv_params* p, int32_t batch, int64_t total_tok
   st.NQ = p->gqa_ratio * p->window;
   st.Ltot = (int)total_tokens;
   st.Ptot = (int)total_tokens;  // >= the true candidate count
-  st.chunks_total = (int)(total_tokens / kChunk) + batch;
   st.pchunks_total = (int)(total_tokens / kPChunk) + batch;
+  st.nt1 = st.nt2 = p->kv_heads * ((int)(total_tokens / kTile) + batch);
   // capacity of the index list: every sequence at its budget
   st.cu[0] = 0;
   for (int b = 1; b <= batch; ++b) st.cu[b] = 0;
@@ -203,13 +218,13 @@ int mixkv_scores(const void* K, const void* V, const void* Qwin, const int32_t* 
                  int32_t batch, int32_t L, const mixkv_params* p, void* workspace,
                  size_t workspace_bytes, float* s_comp, float* s_ex_opt, float* s_div_opt,
                  float* rbar_opt, const float* rbar_in_opt, int32_t* status_dev, void* stream) {
-  (void)status_dev;
   LaunchCtx c;
   int rc = make_ctx(p, cu_seqlens_host, batch, L, workspace, workspace_bytes, stream, &c);
   if (rc != MIXKV_OK) return rc;
   if (!K || !Qwin || !s_comp || (p->use_vnorm && !V)) return MIXKV_ERR_INVALID_ARG;
   if (!aligned16(K) || !aligned16(Qwin) || (V && !aligned16(V))) return MIXKV_ERR_INVALID_ARG;
-  return enqueue_scores(c, K, V, Qwin, s_comp, s_ex_opt, s_div_opt, rbar_opt, rbar_in_opt);
+  return enqueue_scores(c, K, V, Qwin, s_comp, s_ex_opt, s_div_opt, rbar_opt, rbar_in_opt,
+                        status_dev);
 }
 
 int mixkv_select(const float* scores, const int32_t* cu_seqlens_host, int32_t batch, int32_t L,
@@ -223,17 +238,20 @@ int mixkv_select(const float* scores, const int32_t* cu_seqlens_host, int32_t ba
   return enqueue_select(c, scores, idx, counts, idx_offsets, nullptr);
 }
 
-int mixkv_compress_layer(const void* K, const void* V, const void* Qwin,
-                         const int32_t* cu_seqlens_host, int32_t batch, int32_t L,
-                         const mixkv_params* p, void* workspace, size_t workspace_bytes,
-                         const float* rbar_in_opt, void* K_out, void* V_out,
-                         int32_t* out_row_offsets, int32_t* idx_opt, int32_t* counts_opt,
-                         int32_t* idx_offsets_opt, float* s_comp_opt, int32_t* status_dev,
-                         void* stream) {
-  (void)status_dev;
+int mixkv_compress_layer_traced(const void* K, const void* V, const void* Qwin,
+                                const int32_t* cu_seqlens_host, int32_t batch, int32_t L,
+                                const mixkv_params* p, void* workspace, size_t workspace_bytes,
+                                const float* rbar_in_opt, void* K_out, void* V_out,
+                                int32_t* out_row_offsets, int32_t* idx_opt, int32_t* counts_opt,
+                                int32_t* idx_offsets_opt, float* s_comp_opt, int32_t* status_dev,
+                                void* stream, void* const* events_host, int32_t n_events) {
   LaunchCtx c;
   int rc = make_ctx(p, cu_seqlens_host, batch, L, workspace, workspace_bytes, stream, &c);
   if (rc != MIXKV_OK) return rc;
+  if (events_host && n_events > 0) {
+    c.trace_events = events_host;
+    c.n_trace_events = n_events;
+  }
   if (!K || !V || !Qwin || !K_out || !V_out || !out_row_offsets) return MIXKV_ERR_INVALID_ARG;
   if (!aligned16(K) || !aligned16(V) || !aligned16(Qwin) || !aligned16(K_out) || !aligned16(V_out))
     return MIXKV_ERR_INVALID_ARG;
@@ -241,18 +259,39 @@ int mixkv_compress_layer(const void* K, const void* V, const void* Qwin,
   int* idx = idx_opt ? idx_opt : c.ws.idx;
   int* counts = counts_opt ? counts_opt : c.ws.counts;
   int* offs = idx_offsets_opt ? idx_offsets_opt : c.ws.idx_offsets;
-  rc = enqueue_scores(c, K, V, Qwin, s_comp, nullptr, nullptr, nullptr, rbar_in_opt);
+  rc = enqueue_scores(c, K, V, Qwin, s_comp, nullptr, nullptr, nullptr, rbar_in_opt, status_dev);
   if (rc != MIXKV_OK) return rc;
   rc = enqueue_select(c, s_comp, idx, counts, offs, out_row_offsets);
   if (rc != MIXKV_OK) return rc;
+  c.mark();
   if (launch_gather(c, K, V, idx, offs, out_row_offsets, K_out, V_out) != cudaSuccess)
     return MIXKV_ERR_CUDA;
+  c.mark();
   return MIXKV_OK;
+}
+
+int mixkv_compress_layer(const void* K, const void* V, const void* Qwin,
+                         const int32_t* cu_seqlens_host, int32_t batch, int32_t L,
+                         const mixkv_params* p, void* workspace, size_t workspace_bytes,
+                         const float* rbar_in_opt, void* K_out, void* V_out,
+                         int32_t* out_row_offsets, int32_t* idx_opt, int32_t* counts_opt,
+                         int32_t* idx_offsets_opt, float* s_comp_opt, int32_t* status_dev,
+                         void* stream) {
+  return mixkv_compress_layer_traced(K, V, Qwin, cu_seqlens_host, batch, L, p, workspace,
+                                     workspace_bytes, rbar_in_opt, K_out, V_out, out_row_offsets,
+                                     idx_opt, counts_opt, idx_offsets_opt, s_comp_opt, status_dev,
+                                     stream, nullptr, 0);
+}
+
+const char* mixkv_stage_name(const mixkv_params* p, int32_t i) {
+  (void)p;
+  static const char* const names[] = {"pass1", "pass2", "pool", "mix", "budget", "select", "gather"};
+  return (i >= 0 && i < 7) ? names[i] : nullptr;
 }
 
 int mixkv_launches_per_layer(const mixkv_params* p) {
   (void)p;
-  return 8;  // pass1, finalize, pass2, pool, mix, budget, select, gather
+  return 7;  // pass1, pass2, pool, mix, budget, select, gather
 }
 
 const char* mixkv_status_string(int status) {

@@ -13,7 +13,7 @@ namespace mixkv {
 constexpr int kHeadDim = 128;        // d, fixed
 constexpr int kMaxBatch = 64;        // sequences per call
 constexpr int kMaxNQ = 240;          // G*W upper bound (16 spare rows carry the mean key)
-constexpr int kChunk = 512;          // keys per CTA in the two K passes
+constexpr int kTile = 128;           // keys per tensor-core tile
 constexpr int kPChunk = 2048;        // candidate positions per CTA in pool / mix
 constexpr int kExtraRows = 16;       // rows appended to the query tile in pass 2
 constexpr float kLog2e = 1.4426950408889634f;
@@ -22,11 +22,14 @@ constexpr float kLog2e = 1.4426950408889634f;
 struct SeqTable {
   int batch, H, G, W, NQ;
   int Ltot, Ptot;
-  int chunks_total;                  // sum over sequences of ceil(L_b / kChunk)
   int pchunks_total;                 // sum over sequences of ceil(P_b / kPChunk)
   int cu[kMaxBatch + 1];             // sequence offsets into Ltot
-  int chunk_start[kMaxBatch + 1];    // prefix sum of key chunks
   int pchunk_start[kMaxBatch + 1];   // prefix sum of candidate chunks
+  // persistent 128-key tile schedules of the two tensor-core passes, (b, h, t) order
+  int nt1, g1;                       // pass 1: tiles over all L keys, CTAs
+  int nt2, g2;                       // pass 2: tiles over the P candidate keys, CTAs
+  int tile1_start[kMaxBatch + 1];    // prefix sum of H * ceil(L_b / 128)
+  int tile2_start[kMaxBatch + 1];    // prefix sum of H * ceil(P_b / 128)
 };
 
 // Device workspace carve-up (all pointers into the caller's workspace).
@@ -37,10 +40,12 @@ struct Workspace {
   float* s_ex;        // [H, Ptot]   after pooling
   float* s_div;       // [H, Ptot]
   float* s_comp;      // [H, Ptot]
-  float2* rowstat;    // [H, chunks_total, NQ]  per-chunk softmax (max, sum) in log2 units
-  float* ksum;        // [H, chunks_total, d]   per-chunk sum of unit keys
-  float4* vstat;      // [H, chunks_total]      (min, max, sum, -) of |V_i| over candidates
-  float4* dstat;      // [H, chunks_total]      (min, max, sum, -) of s_div over candidates
+  // per-segment partial results; a segment is a run of tiles of one (b, h) inside one CTA's
+  // range and its slot is the id of its first tile
+  float2* rowstat;    // [nt1, 2, NQ]  softmax (max, sum) of each window row, log2 units
+  float* ksum;        // [nt1, d]      sum of unit keys
+  float4* vstat;      // [nt1]         (min, max, sum, -) of |V_i| over candidates
+  float4* dstat;      // [nt2]         (min, max, sum, -) of s_div over candidates
   float* exsum;       // [H, pchunks_total]     per-chunk sum of pooled s_ex
   float* bq;          // [batch, H, NQ]  log2 normaliser of each window row (incl. 1/W)
   __nv_bfloat16* kbar_rows;  // [batch, H, 3, d]  mean unit key split into bf16 hi/lo/lo2
@@ -61,12 +66,24 @@ struct LaunchCtx {
   int max_seq_len;
   int max_prefix;
   cudaStream_t stream;
+  void* const* trace_events;  // optional measurement hook: events recorded between kernels
+  int n_trace_events;
+  mutable int stage;
+
+  // Records the event that marks the start of the next kernel (or the end of the last).
+  void mark() const {
+    if (trace_events && stage < n_trace_events && trace_events[stage])
+      cudaEventRecord((cudaEvent_t)trace_events[stage], stream);
+    ++stage;
+  }
 };
 
 // ---- kernels (defined in the .cu files) ------------------------------------------
-cudaError_t launch_pass1(const LaunchCtx& c, const void* K, const void* V, const void* Q);
-cudaError_t launch_finalize(const LaunchCtx& c);
-cudaError_t launch_pass2(const LaunchCtx& c, const void* K, const void* Q, float* s_div_out);
+cudaError_t launch_pass1(const LaunchCtx& c, const void* K, const void* V, const void* Q,
+                         int* status);
+cudaError_t launch_pass2(const LaunchCtx& c, const void* K, const void* Q, float* s_div_out,
+                         int* status);
+int device_sm_count();
 cudaError_t launch_pool(const LaunchCtx& c, float* s_ex_out);
 cudaError_t launch_mix(const LaunchCtx& c, const float* s_ex, const float* s_div,
                        const float* rbar_in, float* s_comp, float* rbar_out);

@@ -1,72 +1,11 @@
 // Everything after the two K passes: finishing the per-head statistics, pooling, the
 // head-wise mix (Eq. 2, Eq. 5), budgets, per-head top-B selection and the gather
 // (Algorithm 1, step 2 and the TopB line).
-#include "common.cuh"
+#include "tc_common.cuh"
 
 namespace mixkv {
 
 namespace {
-
-// ------------------------------------------------------------------------- finalize
-// One CTA per (sequence, head): merge the per-chunk softmax statistics into one log2
-// normaliser per window row, the per-chunk unit-key sums into the mean unit key (stored as
-// a bf16 hi/lo/lo2 split) and the redundancy of Eq. 4, and the value-norm statistics.
-__global__ void __launch_bounds__(256)
-k_finalize(const SeqTable st, const Workspace ws, const int use_vnorm) {
-  __shared__ float sred[8];
-  const int bh = blockIdx.x, b = bh / st.H, h = bh % st.H;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int c0 = st.chunk_start[b], c1 = st.chunk_start[b + 1];
-  const int L = st.cu[b + 1] - st.cu[b];
-  const size_t pc0 = (size_t)h * st.chunks_total;
-  for (int q = tid; q < st.NQ; q += 256) {
-    float M = -1e30f;
-    for (int c = c0; c < c1; ++c) M = fmaxf(M, ws.rowstat[(pc0 + c) * st.NQ + q].x);
-    float Z = 0.f;
-    for (int c = c0; c < c1; ++c) {
-      const float2 mz = ws.rowstat[(pc0 + c) * st.NQ + q];
-      Z += mz.y * exp2f(mz.x - M);
-    }
-    ws.bq[(size_t)bh * st.NQ + q] = M + log2f(Z * (float)st.W);
-  }
-  float part = 0.f;
-  if (tid < kHeadDim) {
-    float s = 0.f;
-    for (int c = c0; c < c1; ++c) s += ws.ksum[(pc0 + c) * kHeadDim + tid];
-    part = s * s;
-    const float kb = s / (float)L;
-    const __nv_bfloat16 hi = __float2bfloat16_rn(kb);
-    const float r1 = kb - __bfloat162float(hi);
-    const __nv_bfloat16 lo = __float2bfloat16_rn(r1);
-    const __nv_bfloat16 lo2 = __float2bfloat16_rn(r1 - __bfloat162float(lo));
-    __nv_bfloat16* rows = ws.kbar_rows + (size_t)bh * 3 * kHeadDim;
-    rows[tid] = hi;
-    rows[kHeadDim + tid] = lo;
-    rows[2 * kHeadDim + tid] = lo2;
-  }
-  part = warp_sum(part);
-  if (lane == 0) sred[warp] = part;
-  __syncthreads();
-  if (tid == 0) {
-    double n2 = 0.0;
-    for (int w = 0; w < 8; ++w) n2 += (double)sred[w];
-    const double T = (double)L;
-    ws.rbar[bh] = (float)((n2 - T) / (T * (T - 1.0)));  // Eq. 4 with |sum|^2 = T^2 |kbar|^2
-  }
-  if (use_vnorm && warp == 1) {
-    float a = INFINITY, bb = -INFINITY, s = 0.f;
-    for (int c = c0 + lane; c < c1; c += 32) {
-      const float4 v = ws.vstat[pc0 + c];
-      a = fminf(a, v.x);
-      bb = fmaxf(bb, v.y);
-      s += v.z;
-    }
-    a = warp_min(a);
-    bb = warp_max(bb);
-    s = warp_sum(s);
-    if (lane == 0) ws.vfinal[bh] = make_float4(a, bb, s, 0.f);
-  }
-}
 
 // ----------------------------------------------------------------------------- pool
 // 1-D pooling of the raw attention score over the candidate positions of one sequence,
@@ -136,11 +75,18 @@ k_mix(const SeqTable st, const Workspace ws, const float* __restrict__ s_ex,
     for (int c = st.pchunk_start[b] + lane; c < st.pchunk_start[b + 1]; c += 32)
       ex += ws.exsum[(size_t)h * st.pchunks_total + c];
     float a = INFINITY, bb = -INFINITY, s = 0.f;
-    for (int c = st.chunk_start[b] + lane; c < st.chunk_start[b + 1]; c += 32) {
-      const float4 v = ws.dstat[(size_t)h * st.chunks_total + c];
-      a = fminf(a, v.x);
-      bb = fmaxf(bb, v.y);
-      s += v.z;
+    {
+      const int per_head = (st.tile2_start[b + 1] - st.tile2_start[b]) / st.H;
+      const int U0 = st.tile2_start[b] + h * per_head;
+      int k = 0;
+      for (SegIter sg(U0, U0 + per_head, st.nt2, st.g2); sg.valid(); sg.next(), ++k) {
+        if ((k & 31) == lane) {
+          const float4 v = ws.dstat[sg.start];
+          a = fminf(a, v.x);
+          bb = fmaxf(bb, v.y);
+          s += v.z;
+        }
+      }
     }
     ex = warp_sum(ex);
     a = warp_min(a);
@@ -401,11 +347,6 @@ k_gather(const SeqTable st, const __nv_bfloat16* __restrict__ K, const __nv_bflo
 }
 
 }  // namespace
-
-cudaError_t launch_finalize(const LaunchCtx& c) {
-  k_finalize<<<c.st.batch * c.st.H, 256, 0, c.stream>>>(c.st, c.ws, c.p.use_vnorm);
-  return cudaGetLastError();
-}
 
 cudaError_t launch_pool(const LaunchCtx& c, float* s_ex_out) {
   k_pool<<<dim3(c.st.pchunks_total, c.st.H), 256, 0, c.stream>>>(c.st, c.ws, s_ex_out,
