@@ -63,7 +63,6 @@ __device__ __forceinline__ void raise(int* status, volatile int* abort) {
 // 2+2 value-norm warps.
 constexpr int kP1Threads = 18 * 32;
 constexpr int kKsWarp0 = 12;   // warps 12..15
-constexpr int kVWarpsN = 4;    // warps 2, 3, 16, 17
 
 template <int MB>
 __global__ void __launch_bounds__(kP1Threads, 1)
@@ -215,20 +214,23 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUte
         const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + ts * (MB * 128) + col0;
 #pragma unroll 1
         for (int c0 = 0; c0 < NC; c0 += 32) {
-          uint32_t r[32];
-          tmem_ld32(taddr + c0, r);
+          uint32_t ra[16], rb[16];
+          tmem_ld16(taddr + c0, ra);
+          tmem_ld16(taddr + c0 + 16, rb);
           tmem_ld_wait();
-          float v[32];
-#pragma unroll
-          for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+          tmem_ld_fence(ra);
+          tmem_ld_fence(rb);
           if (need_mask) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (k0 + c0 + j > lim) v[j] = -INFINITY;
+            for (int j = 0; j < 16; ++j) {
+              if (k0 + c0 + j > lim) ra[j] = 0xff800000u;        // -inf
+              if (k0 + c0 + 16 + j > lim) rb[j] = 0xff800000u;
+            }
           }
-          float mx = v[0];
+          float mx = fmaxf(__uint_as_float(ra[0]), __uint_as_float(rb[0]));
 #pragma unroll
-          for (int j = 1; j < 32; ++j) mx = fmaxf(mx, v[j]);
+          for (int j = 1; j < 16; ++j)
+            mx = fmaxf(mx, fmaxf(__uint_as_float(ra[j]), __uint_as_float(rb[j])));
           const float mn = fmaxf(m_run, mx * scale_log2e);
           if (mn > m_run) {
             z_run *= ex2(m_run - mn);
@@ -236,9 +238,9 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUte
           }
           float z0 = 0.f, z1 = 0.f;
 #pragma unroll
-          for (int j = 0; j < 32; j += 2) {
-            z0 += ex2(fmaf(v[j], scale_log2e, -m_run));
-            z1 += ex2(fmaf(v[j + 1], scale_log2e, -m_run));
+          for (int j = 0; j < 16; ++j) {
+            z0 += ex2(fmaf(__uint_as_float(ra[j]), scale_log2e, -m_run));
+            z1 += ex2(fmaf(__uint_as_float(rb[j]), scale_log2e, -m_run));
           }
           z_run += z0 + z1;
         }
@@ -333,33 +335,36 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUte
       const size_t poff = (size_t)tc.h * st.Ptot + (st.cu[tc.b] - tc.b * W);
       const int ibase = tc.t * kTile + vw * 32 + hw;
       if (tc.t * kTile + vw * 32 < P) {
-        uint4 u[16];
+#pragma unroll 1
+        for (int kb = 0; kb < 16; kb += 8) {
+          uint4 u[8];
 #pragma unroll
-        for (int k = 0; k < 16; ++k) {
-          const int i = ibase + 2 * k;
-          u[k] = make_uint4(0, 0, 0, 0);
-          if (i < P)
-            u[k] = __ldg(reinterpret_cast<const uint4*>(V + (row0 + i) * kHeadDim) + hl);
-        }
-#pragma unroll
-        for (int k = 0; k < 16; ++k) {
-          const int i = ibase + 2 * k;
-          const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&u[k]);
-          float ss = 0.f;
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const float2 f = __bfloat1622float2(p2[e]);
-            ss = fmaf(f.x, f.x, ss);
-            ss = fmaf(f.y, f.y, ss);
+          for (int k = 0; k < 8; ++k) {
+            const int i = ibase + 2 * (kb + k);
+            u[k] = make_uint4(0, 0, 0, 0);
+            if (i < P)
+              u[k] = __ldg(reinterpret_cast<const uint4*>(V + (row0 + i) * kHeadDim) + hl);
           }
 #pragma unroll
-          for (int o = 8; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-          if (i < P && hl == 0) {
-            const float n = sqrtf(ss);
-            ws.vnorm[poff + i] = n;
-            vmin = fminf(vmin, n);
-            vmax = fmaxf(vmax, n);
-            vsum += n;
+          for (int k = 0; k < 8; ++k) {
+            const int i = ibase + 2 * (kb + k);
+            const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&u[k]);
+            float ss = 0.f;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const float2 f = __bfloat1622float2(p2[e]);
+              ss = fmaf(f.x, f.x, ss);
+              ss = fmaf(f.y, f.y, ss);
+            }
+#pragma unroll
+            for (int o = 8; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+            if (i < P && hl == 0) {
+              const float n = sqrtf(ss);
+              ws.vnorm[poff + i] = n;
+              vmin = fminf(vmin, n);
+              vmax = fmaxf(vmax, n);
+              vsum += n;
+            }
           }
         }
       }
@@ -407,7 +412,9 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUte
   float* sbq = reinterpret_cast<float*>(sK + kStages * kTileBytes);  // [256]
   float* sx = sbq + 256;                      // [2][128] partial sums WG0 -> WG1
   float* sred = sx + 256;                     // [32]
-  PipeBars* bars = reinterpret_cast<PipeBars*>(sred + 32);
+  float* sksp = sred + 32;                    // [2][128] unit-key sums of the two prep warps
+  float2* spart = reinterpret_cast<float2*>(sksp + 256);   // [8][256] per-warp row statistics
+  PipeBars* bars = reinterpret_cast<PipeBars*>(spart + 8 * 256);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int lo = cta_first_tile(blockIdx.x, st.nt2, st.g2);
@@ -516,12 +523,24 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUte
       const int L = st.cu[tc.b + 1] - st.cu[tc.b];
       const int per_head = (st.tile1_start[tc.b + 1] - st.tile1_start[tc.b]) / H;
       const int T0 = st.tile1_start[tc.b] + tc.h * per_head;
-      float s0 = 0.f, s1 = 0.f;
-      for (SegIter sg(T0, T0 + per_head, st.nt1, st.g1); sg.valid(); sg.next()) {
-        const float2 f = *reinterpret_cast<const float2*>(ws.ksum + (size_t)sg.start * kHeadDim + 2 * pt);
-        s0 += f.x;
-        s1 += f.y;
+      // pass 1 left one partial sum per segment of this (b, h): segment e starts at T0 for
+      // e = 0 and at the first tile of CTA c0 + e otherwise
+      const int c0 = tile_owner(T0, st.nt1, st.g1);
+      const int nseg = tile_owner(T0 + per_head - 1, st.nt1, st.g1) - c0 + 1;
+      {
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
+        for (int e = warp - 2; e < nseg; e += 2) {
+          const int start = e == 0 ? T0 : cta_first_tile(c0 + e, st.nt1, st.g1);
+          const float4 f = *reinterpret_cast<const float4*>(ws.ksum + (size_t)start * kHeadDim + 4 * lane);
+          acc.x += f.x, acc.y += f.y, acc.z += f.z, acc.w += f.w;
+        }
+        named_bar_sync(4, 64);   // the previous segment's readers of sksp are done
+        *reinterpret_cast<float4*>(sksp + (warp - 2) * 128 + 4 * lane) = acc;
+        named_bar_sync(4, 64);
       }
+      const float s0 = sksp[2 * pt] + sksp[128 + 2 * pt];
+      const float s1 = sksp[2 * pt + 1] + sksp[128 + 2 * pt + 1];
       const bool owner = tc.t == 0;
       if (owner) {
         float n2 = warp_sum(s0 * s0 + s1 * s1);
@@ -565,14 +584,12 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUte
         }
         if (use_vnorm && warp == 3) {
           float a = INFINITY, b2 = -INFINITY, c2 = 0.f;
-          int k = 0;
-          for (SegIter sg(T0, T0 + per_head, st.nt1, st.g1); sg.valid(); sg.next(), ++k) {
-            if ((k & 31) == lane) {
-              const float4 v = ws.vstat[sg.start];
-              a = fminf(a, v.x);
-              b2 = fmaxf(b2, v.y);
-              c2 += v.z;
-            }
+          for (int e = lane; e < nseg; e += 32) {
+            const int start = e == 0 ? T0 : cta_first_tile(c0 + e, st.nt1, st.g1);
+            const float4 v = ws.vstat[start];
+            a = fminf(a, v.x);
+            b2 = fmaxf(b2, v.y);
+            c2 += v.z;
           }
           a = warp_min(a);
           b2 = warp_max(b2);
@@ -599,21 +616,46 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUte
         // merge pass 1's per-segment softmax statistics of this (b, h) into one log2
         // normaliser per window row (the 1/W of the window mean folded in)
         named_bar_sync(1, kEpiThreads);
-        if (et < NQ) {
+        {
           const int per_head = (st.tile1_start[tc.b + 1] - st.tile1_start[tc.b]) / H;
           const int T0 = st.tile1_start[tc.b] + tc.h * per_head;
+          const int c0 = tile_owner(T0, st.nt1, st.g1);
+          const int nseg = tile_owner(T0 + per_head - 1, st.nt1, st.g1) - c0 + 1;
           const int nunits = NQ <= 128 ? 2 : 1;
-          float M = -1e30f;
-          for (SegIter sg(T0, T0 + per_head, st.nt1, st.g1); sg.valid(); sg.next())
-            for (int u = 0; u < nunits; ++u)
-              M = fmaxf(M, ws.rowstat[((size_t)sg.start * 2 + u) * NQ + et].x);
-          float Z = 0.f;
-          for (SegIter sg(T0, T0 + per_head, st.nt1, st.g1); sg.valid(); sg.next())
-            for (int u = 0; u < nunits; ++u) {
-              const float2 mz = ws.rowstat[((size_t)sg.start * 2 + u) * NQ + et];
-              Z += mz.y * exp2f(mz.x - M);
+          const int ew = warp - kEpiWarp0;
+          float M[8], Z[8];
+#pragma unroll
+          for (int r = 0; r < 8; ++r) M[r] = -1e30f, Z[r] = 0.f;
+          for (int k = ew; k < nseg * nunits; k += kEpiWarps) {
+            const int e = k / nunits, u = k - e * nunits;
+            const int start = e == 0 ? T0 : cta_first_tile(c0 + e, st.nt1, st.g1);
+            const float2* src = ws.rowstat + ((size_t)start * 2 + u) * NQ;
+#pragma unroll
+            for (int r = 0; r < 8; ++r) {
+              const int q = lane + 32 * r;
+              if (q < NQ) {
+                const float2 mz = src[q];
+                const float mn = fmaxf(M[r], mz.x);
+                Z[r] = Z[r] * ex2(M[r] - mn) + mz.y * ex2(mz.x - mn);
+                M[r] = mn;
+              }
             }
-          sbq[et] = M + log2f(Z * (float)W);
+          }
+#pragma unroll
+          for (int r = 0; r < 8; ++r) spart[ew * 256 + lane + 32 * r] = make_float2(M[r], Z[r]);
+          named_bar_sync(1, kEpiThreads);
+          if (et < NQ) {
+            float Mx = -1e30f;
+#pragma unroll
+            for (int w = 0; w < kEpiWarps; ++w) Mx = fmaxf(Mx, spart[w * 256 + et].x);
+            float Zs = 0.f;
+#pragma unroll
+            for (int w = 0; w < kEpiWarps; ++w) {
+              const float2 mz = spart[w * 256 + et];
+              Zs += mz.y * exp2f(mz.x - Mx);
+            }
+            sbq[et] = Mx + log2f(Zs * (float)W);
+          }
         }
         dmin = INFINITY, dmax = -INFINITY, dsum = 0.f;
         seg_first = id;
@@ -621,28 +663,50 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUte
         named_bar_sync(1, kEpiThreads);
       }
       const int ts = it & 1, tph = (it >> 1) & 1;
+      const int ikey = tc.t * kTile + key;
+      float kinv_i = 0.f;
+      if (wg == 1 && ikey < P) kinv_i = ws.kinv[(size_t)tc.h * st.Ltot + st.cu[tc.b] + ikey];
       const bool ok = mbar_wait(&bars->tfull[ts], tph, abort);
       tc_fence_after();
       const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + ts * 256;
       float acc0 = 0.f, acc1 = 0.f, dot = 0.f;
+      if (ok && cbeg < cend) {
+        // 16-column chunks, the next one in flight while this one is reduced
+        uint32_t ra[16], rb[16];
+        tmem_ld16(taddr + cbeg, ra);
 #pragma unroll 1
-      for (int c0 = cbeg; c0 < (ok ? cend : cbeg); c0 += 16) {
-        uint32_t r[16];
-        tmem_ld16(taddr + c0, r);
-        tmem_ld_wait();
+        for (int c0 = cbeg; c0 < cend; c0 += 32) {
+          tmem_ld_wait();
+          tmem_ld_fence(ra);
+          if (c0 + 16 < cend) tmem_ld16(taddr + c0 + 16, rb);
 #pragma unroll
-        for (int j = 0; j < 16; j += 4) {
-          const float4 nb = *reinterpret_cast<const float4*>(sbq + c0 + j);
-          acc0 += ex2(fmaf(__uint_as_float(r[j]), scale_log2e, -nb.x));
-          acc1 += ex2(fmaf(__uint_as_float(r[j + 1]), scale_log2e, -nb.y));
-          acc0 += ex2(fmaf(__uint_as_float(r[j + 2]), scale_log2e, -nb.z));
-          acc1 += ex2(fmaf(__uint_as_float(r[j + 3]), scale_log2e, -nb.w));
+          for (int j = 0; j < 16; j += 4) {
+            const float4 nb = *reinterpret_cast<const float4*>(sbq + c0 + j);
+            acc0 += ex2(fmaf(__uint_as_float(ra[j]), scale_log2e, -nb.x));
+            acc1 += ex2(fmaf(__uint_as_float(ra[j + 1]), scale_log2e, -nb.y));
+            acc0 += ex2(fmaf(__uint_as_float(ra[j + 2]), scale_log2e, -nb.z));
+            acc1 += ex2(fmaf(__uint_as_float(ra[j + 3]), scale_log2e, -nb.w));
+          }
+          if (c0 + 16 < cend) {
+            tmem_ld_wait();
+            tmem_ld_fence(rb);
+            if (c0 + 32 < cend) tmem_ld16(taddr + c0 + 32, ra);
+#pragma unroll
+            for (int j = 0; j < 16; j += 4) {
+              const float4 nb = *reinterpret_cast<const float4*>(sbq + c0 + 16 + j);
+              acc0 += ex2(fmaf(__uint_as_float(rb[j]), scale_log2e, -nb.x));
+              acc1 += ex2(fmaf(__uint_as_float(rb[j + 1]), scale_log2e, -nb.y));
+              acc0 += ex2(fmaf(__uint_as_float(rb[j + 2]), scale_log2e, -nb.z));
+              acc1 += ex2(fmaf(__uint_as_float(rb[j + 3]), scale_log2e, -nb.w));
+            }
+          }
         }
       }
       if (wg == 1 && ok) {
         uint32_t r[16];
         tmem_ld16(taddr + NQ, r);
         tmem_ld_wait();
+        tmem_ld_fence(r);
         dot = (__uint_as_float(r[0]) + __uint_as_float(r[1])) + __uint_as_float(r[2]);
       }
       tc_fence_before();
@@ -654,7 +718,7 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUte
         if (i < P) {
           const size_t poff = (size_t)tc.h * st.Ptot + (st.cu[tc.b] - tc.b * W);
           ws.s_ex_raw[poff + i] = (acc0 + acc1) + sx[ts * 128 + key];
-          const float sd = -dot * ws.kinv[(size_t)tc.h * st.Ltot + st.cu[tc.b] + i];
+          const float sd = -dot * kinv_i;
           s_div_out[poff + i] = sd;
           dmin = fminf(dmin, sd);
           dmax = fmaxf(dmax, sd);
@@ -740,7 +804,7 @@ size_t pass1_smem(int MB) {
 }
 size_t pass2_smem() {
   return 1024 + (size_t)2 * (kMaxNQ + kExtraRows) * 128 + kStages * kTileBytes + 256 * 4 +
-         256 * 4 + 32 * 4 + sizeof(PipeBars) + 64;
+         256 * 4 + 32 * 4 + 256 * 4 + 8 * 256 * 8 + sizeof(PipeBars) + 64;
 }
 
 }  // namespace

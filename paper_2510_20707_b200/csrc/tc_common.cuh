@@ -163,6 +163,17 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 __device__ __forceinline__ void tmem_ld_wait() {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
+// The registers written by tcgen05.ld are only valid after tcgen05.wait::ld.  This empty
+// statement makes every later use of r depend on a point after the wait (volatile asm
+// statements keep their order), so the compiler cannot hoist arithmetic above it.
+__device__ __forceinline__ void tmem_ld_fence(uint32_t (&r)[16]) {
+  asm volatile(""
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]),
+                 "+r"(r[7]), "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]),
+                 "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
+               :
+               : "memory");
+}
 __device__ __forceinline__ void fence_proxy_async_smem() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
@@ -197,6 +208,11 @@ __device__ __forceinline__ TileCoord tile_coord(const int* tile_start, int batch
 // First tile of CTA c when nt tiles are split over g CTAs (contiguous ranges).
 __host__ __device__ __forceinline__ int cta_first_tile(int c, int nt, int g) {
   return (int)(((long long)c * nt) / g);
+}
+
+// CTA whose contiguous range contains tile t.
+__host__ __device__ __forceinline__ int tile_owner(int t, int nt, int g) {
+  return (int)((((long long)t + 1) * g - 1) / nt);
 }
 
 // Enumerates
