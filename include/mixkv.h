@@ -48,7 +48,8 @@ typedef enum {
   MIXKV_ERR_UNSUPPORTED = -2,
   MIXKV_ERR_WORKSPACE_TOO_SMALL = -3,
   MIXKV_ERR_CUDA = -4,
-  MIXKV_ERR_TIMEOUT = -5
+  MIXKV_ERR_TIMEOUT = -5,
+  MIXKV_ERR_STATIC_SCRATCH_EXCEEDED = -6
 } mixkv_status;
 
 enum { MIXKV_MIX_HEADWISE = 0, MIXKV_MIX_IMPORTANCE_ONLY = 1, MIXKV_MIX_DIVERSITY_ONLY = 2,
@@ -103,6 +104,35 @@ int mixkv_scores(const void* K, const void* V, const void* Qwin,
                  const mixkv_params* p, void* workspace, size_t workspace_bytes,
                  float* s_comp, float* s_ex_opt, float* s_div_opt, float* rbar_opt,
                  const float* rbar_in_opt, int32_t* status_dev, void* stream);
+
+/* mixkv_scores for callers that cannot obtain device memory for a workspace (the paper has
+ * no counterpart; this is a packaging variant of mixkv_scores, same kernels, same results).
+ * Typical users: a serving engine that hands every free byte of HBM to its own paged KV pool
+ * at start-up, so that a later cudaMalloc fails or fragments the pool; a plug-in running
+ * inside somebody else's step loop, where cudaMalloc / cudaFree would stall the whole device
+ * with their implicit synchronisation; a host language binding that can pass pointers it
+ * was given but owns no allocator.  Such callers still pass their inputs and outputs; only
+ * the scratch the kernels need between them comes from the library: a fixed array of
+ * MIXKV_STATIC_SCRATCH_BYTES that lives in the library's device image, so every GPU that
+ * loads the library sets that much memory aside until the process exits.
+ *  - Problems whose workspace (mixkv_workspace_size) would exceed the array are refused with
+ *    MIXKV_ERR_STATIC_SCRATCH_EXCEEDED and nothing is enqueued.  As a guide the array covers
+ *    about 128k (head, token) pairs, e.g. H = 4 at L = 32768 or H = 8 at L = 16384.
+ *  - The call performs no cudaMalloc / cudaFree and calls no allocating library routine.
+ *  - The first call on each device looks up the array's device address (once per device, with
+ *    that device current) and keeps it for later calls; make that first call outside any
+ *    stream capture.
+ *  - All calls on one device share the one array, and it keeps whatever the previous call
+ *    left in it.  Nothing in it needs to start from zero (every cell is written before it is
+ *    read inside a call), but two calls whose kernels overlap on the GPU (different streams
+ *    without an ordering between them) race on it: order such calls yourself.
+ * Arguments are those of mixkv_scores without workspace / workspace_bytes. */
+#define MIXKV_STATIC_SCRATCH_BYTES (12u << 20)
+int mixkv_scores_static(const void* K, const void* V, const void* Qwin,
+                        const int32_t* cu_seqlens_host, int32_t batch, int32_t L,
+                        const mixkv_params* p, float* s_comp, float* s_ex_opt, float* s_div_opt,
+                        float* rbar_opt, const float* rbar_in_opt, int32_t* status_dev,
+                        void* stream);
 
 /* TopB of Sec. 3.1 / Algorithm 1 on caller-supplied scores [H, Ptot]: per (sequence, head)
  * the b_h highest scores among the P_b candidates, ties to the lower position, written in

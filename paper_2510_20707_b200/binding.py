@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_PKG, "libmixkv.so")
 
 EXPORTS = ("mixkv_default_params", "mixkv_workspace_size", "mixkv_scores", "mixkv_select",
            "mixkv_compress_layer", "mixkv_compress_layer_traced", "mixkv_launches_per_layer",
-           "mixkv_stage_name", "mixkv_status_string")
+           "mixkv_stage_name", "mixkv_status_string", "mixkv_scores_static")
 
 
 class MixKVError(RuntimeError):
@@ -82,6 +82,8 @@ def load_library() -> C.CDLL:
         lib.mixkv_launches_per_layer.argtypes = [C.POINTER(_CParams)]
         lib.mixkv_scores.argtypes = [vp, vp, vp, C.POINTER(i32), i32, i32, C.POINTER(_CParams),
                                      vp, sz, vp, vp, vp, vp, vp, vp, vp]
+        lib.mixkv_scores_static.argtypes = [vp, vp, vp, C.POINTER(i32), i32, i32,
+                                            C.POINTER(_CParams), vp, vp, vp, vp, vp, vp, vp]
         lib.mixkv_select.argtypes = [vp, C.POINTER(i32), i32, i32, C.POINTER(_CParams), vp, sz,
                                      vp, vp, vp, vp, vp]
         lib.mixkv_compress_layer.argtypes = [vp, vp, vp, C.POINTER(i32), i32, i32,
@@ -172,6 +174,34 @@ def scores(K: torch.Tensor, V: Optional[torch.Tensor], Q: torch.Tensor, params: 
         _ptr(out.get("rbar")), _ptr(rbar_in), _ptr(status), _stream(stream))
     if rc != 0:
         raise MixKVError(rc, "mixkv_scores")
+    out["status"] = status
+    return out
+
+
+def scores_static(K: torch.Tensor, V: Optional[torch.Tensor], Q: torch.Tensor, params: Params,
+                  cu_seqlens: Optional[Sequence[int]] = None,
+                  rbar_in: Optional[torch.Tensor] = None, stream=None) -> Dict[str, torch.Tensor]:
+    """mixkv_scores_static: the same scores as :func:`scores`, for callers that cannot give
+    the library a workspace.  The scratch the kernels need lives inside the library (a fixed
+    array, see MIXKV_STATIC_SCRATCH_BYTES in the header), so this function hands over inputs
+    and outputs only; the output tensors below are the caller's, as in :func:`scores`.
+    Raises MixKVError (status -6) when the problem is too large for the built-in array.
+    Calls on one device share that array: do not let two of them overlap on the GPU."""
+    H, Ltot, d = K.shape
+    batch = 1 if cu_seqlens is None else len(cu_seqlens) - 1
+    Ptot = Ltot - batch * params.window
+    f32 = dict(dtype=torch.float32, device=K.device)
+    out = {"s_comp": torch.empty((H, Ptot), **f32), "s_ex": torch.empty((H, Ptot), **f32),
+           "s_div": torch.empty((H, Ptot), **f32), "rbar": torch.empty((batch, H), **f32)}
+    status = torch.zeros(1, dtype=torch.int32, device=K.device)
+    cu, _ = _cu_array(cu_seqlens)
+    pc = params.c()
+    rc = load_library().mixkv_scores_static(
+        _ptr(K), _ptr(V), _ptr(Q), cu, batch, Ltot, C.byref(pc), _ptr(out["s_comp"]),
+        _ptr(out["s_ex"]), _ptr(out["s_div"]), _ptr(out["rbar"]), _ptr(rbar_in), _ptr(status),
+        _stream(stream))
+    if rc != 0:
+        raise MixKVError(rc, "mixkv_scores_static")
     out["status"] = status
     return out
 

@@ -2,6 +2,8 @@
 #include <math.h>
 #include <string.h>
 
+#include <mutex>
+
 #include "common.cuh"
 
 namespace mixkv {
@@ -283,6 +285,57 @@ int mixkv_compress_layer(const void* K, const void* V, const void* Qwin,
                                      stream, nullptr, 0);
 }
 
+// ---- the no-allocation variant of mixkv_scores -------------------------------------------
+// Scratch for callers that cannot allocate: part of the library's device image, one copy per
+// GPU that loads the library.  In host code the name g_static_scratch is only a handle for
+// cudaGetSymbolAddress, never a device address.
+static __device__ __align__(256) unsigned char g_static_scratch[MIXKV_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mutex;
+void* g_scratch_addr[kMaxDevices] = {nullptr};
+
+// Device address of the scratch array on the current device; looked up once per device.
+int static_scratch(void** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return MIXKV_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_scratch_mutex);
+  if (!g_scratch_addr[dev]) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return MIXKV_ERR_CUDA;
+    g_scratch_addr[dev] = ptr;
+  }
+  *out = g_scratch_addr[dev];
+  return MIXKV_OK;
+}
+}  // namespace
+
+int mixkv_scores_static(const void* K, const void* V, const void* Qwin,
+                        const int32_t* cu_seqlens_host, int32_t batch, int32_t L,
+                        const mixkv_params* p, float* s_comp, float* s_ex_opt, float* s_div_opt,
+                        float* rbar_opt, const float* rbar_in_opt, int32_t* status_dev,
+                        void* stream) {
+  // size the problem on the host first: too large a problem is refused before any CUDA call
+  {
+    int rc = check_params(p);
+    if (rc != MIXKV_OK) return rc;
+    SeqTable st;
+    int max_len = 0;
+    rc = build_table(p, cu_seqlens_host, batch, L, &st, &max_len);
+    if (rc != MIXKV_OK) return rc;
+    Workspace ws;
+    carve(p, st, nullptr, &ws);
+    if (ws.bytes > (size_t)MIXKV_STATIC_SCRATCH_BYTES) return MIXKV_ERR_STATIC_SCRATCH_EXCEEDED;
+  }
+  void* scratch = nullptr;
+  int rc = static_scratch(&scratch);
+  if (rc != MIXKV_OK) return rc;
+  return mixkv_scores(K, V, Qwin, cu_seqlens_host, batch, L, p, scratch,
+                      (size_t)MIXKV_STATIC_SCRATCH_BYTES, s_comp, s_ex_opt, s_div_opt, rbar_opt,
+                      rbar_in_opt, status_dev, stream);
+}
+
 const char* mixkv_stage_name(const mixkv_params* p, int32_t i) {
   (void)p;
   static const char* const names[] = {"pass1", "pass2", "pool", "mix", "budget", "select", "gather"};
@@ -302,6 +355,8 @@ const char* mixkv_status_string(int status) {
     case MIXKV_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
     case MIXKV_ERR_CUDA: return "CUDA error";
     case MIXKV_ERR_TIMEOUT: return "device-side bounded wait expired";
+    case MIXKV_ERR_STATIC_SCRATCH_EXCEEDED:
+      return "problem needs more scratch than the built-in array of the no-allocation entry point";
     default: return "unknown status";
   }
 }
