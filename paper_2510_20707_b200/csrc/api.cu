@@ -92,22 +92,19 @@ void carve(const mixkv_params* p, const SeqTable& st, unsigned char* base, Works
   ws->kinv = (float*)take(H * st.Ltot * 4);
   ws->vnorm = (float*)take(H * st.Ptot * 4);
   ws->s_ex_raw = (float*)take(H * st.Ptot * 4);
-  ws->s_ex = (float*)take(H * st.Ptot * 4);
   ws->s_div = (float*)take(H * st.Ptot * 4);
   ws->s_comp = (float*)take(H * st.Ptot * 4);
   ws->rowstat = (float2*)take((size_t)st.nt1 * 2 * st.NQ * 8);
   ws->ksum = (float*)take((size_t)st.nt1 * kHeadDim * 4);
-  ws->vstat = (float4*)take((size_t)st.nt1 * 16);
+  ws->vstat = (float4*)take((size_t)st.nt2 * 16);
   ws->dstat = (float4*)take((size_t)st.nt2 * 16);
   ws->exsum = (float*)take(H * st.pchunks_total * 4);
   ws->bq = (float*)take(BH * st.NQ * 4);
-  ws->kbar_rows = (__nv_bfloat16*)take(BH * 3 * kHeadDim * 2);
+  ws->kbar_rows = (__nv_bfloat16*)take(BH * kExtraRows * kHeadDim * 2);
   ws->rbar = (float*)take(BH * 4);
-  ws->vfinal = (float4*)take(BH * 16);
   ws->counts = (int*)take(BH * 4);
   ws->idx_offsets = (int*)take((BH + 1) * 4);
   ws->idx = (int*)take((size_t)idx_capacity(p, st) * 4);
-  ws->status = (int*)take(4);
   ws->bytes = off;
 }
 
@@ -135,30 +132,60 @@ int make_ctx(const mixkv_params* p, const int32_t* cu, int batch, int L, void* w
   return MIXKV_OK;
 }
 
-int enqueue_scores(const LaunchCtx& c, const void* K, const void* V, const void* Q, float* s_comp,
-                   float* s_ex_out, float* s_div_out, float* rbar_out, const float* rbar_in,
-                   int* status) {
-  float* s_ex = s_ex_out ? s_ex_out : c.ws.s_ex;
-  float* s_div = s_div_out ? s_div_out : c.ws.s_div;
+// pass 1, merge, pass 2 (and the pooled-score sums max pooling needs): everything the mix reads.
+int enqueue_passes(const LaunchCtx& c, const void* K, const void* V, const void* Q, float* s_div,
+                   float* rbar_out, int* status) {
   c.mark();
-  if (launch_pass1(c, K, V, Q, status) != cudaSuccess) return MIXKV_ERR_CUDA;
+  if (launch_pass1(c, K, Q, status) != cudaSuccess) return MIXKV_ERR_CUDA;
   c.mark();
-  if (launch_pass2(c, K, Q, s_div, status) != cudaSuccess) return MIXKV_ERR_CUDA;
+  if (launch_merge(c, rbar_out) != cudaSuccess) return MIXKV_ERR_CUDA;
   c.mark();
-  if (launch_pool(c, s_ex) != cudaSuccess) return MIXKV_ERR_CUDA;
-  c.mark();
-  if (launch_mix(c, s_ex, s_div, rbar_in, s_comp, rbar_out) != cudaSuccess) return MIXKV_ERR_CUDA;
+  if (launch_pass2(c, K, V, Q, s_div, status) != cudaSuccess) return MIXKV_ERR_CUDA;
+  if (c.p.pool_mode == MIXKV_POOL_MAX) {
+    c.mark();
+    if (launch_poolsum(c) != cudaSuccess) return MIXKV_ERR_CUDA;
+  }
   return MIXKV_OK;
 }
 
-int enqueue_select(const LaunchCtx& c, const float* scores, int* idx, int* counts,
-                   int* idx_offsets, int* out_row_offsets) {
+int enqueue_scores(const LaunchCtx& c, const void* K, const void* V, const void* Q, float* s_comp,
+                   float* s_ex_out, float* s_div_out, float* rbar_out, const float* rbar_in,
+                   int* status) {
+  float* s_div = s_div_out ? s_div_out : c.ws.s_div;
+  int rc = enqueue_passes(c, K, V, Q, s_div, rbar_out, status);
+  if (rc != MIXKV_OK) return rc;
   c.mark();
-  if (launch_budget(c, scores, counts) != cudaSuccess) return MIXKV_ERR_CUDA;
-  c.mark();
-  if (launch_select(c, scores, counts, idx, idx_offsets, out_row_offsets) != cudaSuccess)
-    return MIXKV_ERR_CUDA;
+  if (launch_mixpool(c, s_div, rbar_in, s_ex_out, s_comp) != cudaSuccess) return MIXKV_ERR_CUDA;
   return MIXKV_OK;
+}
+
+// Budgets (adaptive only) and the selection on given scores; gathers when t.K_out is set.
+int enqueue_select(const LaunchCtx& c, const float* scores, int* counts, TailArgs t) {
+  t.scores = scores;
+  t.counts_dev = nullptr;
+  t.counts_out = counts;
+  if (c.p.budget_mode == MIXKV_BUDGET_ADAPTIVE) {
+    c.mark();
+    if (launch_budget(c, scores, counts) != cudaSuccess) return MIXKV_ERR_CUDA;
+    t.counts_dev = counts;
+    t.counts_out = nullptr;
+  }
+  c.mark();
+  if (launch_tail(c, t) != cudaSuccess) return MIXKV_ERR_CUDA;
+  return MIXKV_OK;
+}
+
+// Names of the kernels a layer call enqueues, in order.
+int layer_stages(const mixkv_params* p, bool fused_ok, const char** names) {
+  int n = 0;
+  names[n++] = "pass1";
+  names[n++] = "merge";
+  names[n++] = "pass2";
+  if (p->pool_mode == MIXKV_POOL_MAX) names[n++] = "poolsum";
+  if (p->budget_mode == MIXKV_BUDGET_ADAPTIVE || !fused_ok) names[n++] = "mixpool";
+  if (p->budget_mode == MIXKV_BUDGET_ADAPTIVE) names[n++] = "budget";
+  names[n++] = "tail";
+  return n;
 }
 
 }  // namespace
@@ -237,7 +264,11 @@ int mixkv_select(const float* scores, const int32_t* cu_seqlens_host, int32_t ba
   int rc = make_ctx(p, cu_seqlens_host, batch, L, workspace, workspace_bytes, stream, &c);
   if (rc != MIXKV_OK) return rc;
   if (!scores || !idx || !counts || !idx_offsets) return MIXKV_ERR_INVALID_ARG;
-  return enqueue_select(c, scores, idx, counts, idx_offsets, nullptr);
+  TailArgs t;
+  memset(&t, 0, sizeof(t));
+  t.idx = idx;
+  t.idx_offsets = idx_offsets;
+  return enqueue_select(c, scores, counts, t);
 }
 
 int mixkv_compress_layer_traced(const void* K, const void* V, const void* Qwin,
@@ -258,16 +289,33 @@ int mixkv_compress_layer_traced(const void* K, const void* V, const void* Qwin,
   if (!aligned16(K) || !aligned16(V) || !aligned16(Qwin) || !aligned16(K_out) || !aligned16(V_out))
     return MIXKV_ERR_INVALID_ARG;
   float* s_comp = s_comp_opt ? s_comp_opt : c.ws.s_comp;
-  int* idx = idx_opt ? idx_opt : c.ws.idx;
   int* counts = counts_opt ? counts_opt : c.ws.counts;
-  int* offs = idx_offsets_opt ? idx_offsets_opt : c.ws.idx_offsets;
-  rc = enqueue_scores(c, K, V, Qwin, s_comp, nullptr, nullptr, nullptr, rbar_in_opt, status_dev);
+  TailArgs t;
+  memset(&t, 0, sizeof(t));
+  t.idx = idx_opt ? idx_opt : c.ws.idx;
+  t.idx_offsets = idx_offsets_opt ? idx_offsets_opt : c.ws.idx_offsets;
+  t.out_row_offsets = out_row_offsets;
+  t.K = K;
+  t.V = V;
+  t.K_out = K_out;
+  t.V_out = V_out;
+  rc = enqueue_passes(c, K, V, Qwin, c.ws.s_div, nullptr, status_dev);
   if (rc != MIXKV_OK) return rc;
-  rc = enqueue_select(c, s_comp, idx, counts, offs, out_row_offsets);
-  if (rc != MIXKV_OK) return rc;
-  c.mark();
-  if (launch_gather(c, K, V, idx, offs, out_row_offsets, K_out, V_out) != cudaSuccess)
-    return MIXKV_ERR_CUDA;
+  if (p->budget_mode == MIXKV_BUDGET_FIXED && tail_can_fuse(c)) {
+    // one kernel: mix, select, gather
+    t.s_div = c.ws.s_div;
+    t.rbar_in = rbar_in_opt;
+    t.s_comp_out = s_comp;
+    t.counts_out = counts;
+    c.mark();
+    if (launch_tail(c, t) != cudaSuccess) return MIXKV_ERR_CUDA;
+  } else {
+    c.mark();
+    if (launch_mixpool(c, c.ws.s_div, rbar_in_opt, nullptr, s_comp) != cudaSuccess)
+      return MIXKV_ERR_CUDA;
+    rc = enqueue_select(c, s_comp, counts, t);
+    if (rc != MIXKV_OK) return rc;
+  }
   c.mark();
   return MIXKV_OK;
 }
@@ -337,14 +385,16 @@ int mixkv_scores_static(const void* K, const void* V, const void* Qwin,
 }
 
 const char* mixkv_stage_name(const mixkv_params* p, int32_t i) {
-  (void)p;
-  static const char* const names[] = {"pass1", "pass2", "pool", "mix", "budget", "select", "gather"};
-  return (i >= 0 && i < 7) ? names[i] : nullptr;
+  if (!p) return nullptr;
+  const char* names[8];
+  const int n = layer_stages(p, true, names);
+  return (i >= 0 && i < n) ? names[i] : nullptr;
 }
 
 int mixkv_launches_per_layer(const mixkv_params* p) {
-  (void)p;
-  return 7;  // pass1, pass2, pool, mix, budget, select, gather
+  if (!p) return 0;
+  const char* names[8];
+  return layer_stages(p, true, names);
 }
 
 const char* mixkv_status_string(int status) {

@@ -37,24 +37,21 @@ struct Workspace {
   float* kinv;        // [H, Ltot]   1 / |K_i|  (0 for a zero key)
   float* vnorm;       // [H, Ptot]   |V_i|
   float* s_ex_raw;    // [H, Ptot]   window attention score before pooling
-  float* s_ex;        // [H, Ptot]   after pooling
   float* s_div;       // [H, Ptot]
   float* s_comp;      // [H, Ptot]
   // per-segment partial results; a segment is a run of tiles of one (b, h) inside one CTA's
   // range and its slot is the id of its first tile
   float2* rowstat;    // [nt1, 2, NQ]  softmax (max, sum) of each window row, log2 units
   float* ksum;        // [nt1, d]      sum of unit keys
-  float4* vstat;      // [nt1]         (min, max, sum, -) of |V_i| over candidates
-  float4* dstat;      // [nt2]         (min, max, sum, -) of s_div over candidates
-  float* exsum;       // [H, pchunks_total]     per-chunk sum of pooled s_ex
-  float* bq;          // [batch, H, NQ]  log2 normaliser of each window row (incl. 1/W)
-  __nv_bfloat16* kbar_rows;  // [batch, H, 3, d]  mean unit key split into bf16 hi/lo/lo2
-  float* rbar;        // [batch, H]
-  float4* vfinal;     // [batch, H] (min, max, sum, -) of |V_i|
+  float4* vstat;      // [nt2]         (min, max, sum, -) of |V_i| over candidates
+  float4* dstat;      // [nt2]         (min, max, sum) of s_div, window-count-weighted sum of s_ex_raw
+  float* exsum;       // [H, pchunks_total]   per-chunk sum of pooled s_ex (max pooling only)
+  float* bq;          // [batch*H, NQ]  log2 normaliser of each window row (incl. 1/W)
+  __nv_bfloat16* kbar_rows;  // [batch*H, 16, d]  mean unit key as bf16 hi/lo/lo2 rows, 13 zero rows
+  float* rbar;        // [batch*H]
   int* counts;        // [batch*H]
   int* idx_offsets;   // [batch*H + 1]
-  int* idx;           // [batch*H*(B-W)] (or more for adaptive)
-  int* status;        // [1]
+  int* idx;           // [batch*H*(B-W)]
   size_t bytes;
 };
 
@@ -79,20 +76,64 @@ struct LaunchCtx {
 };
 
 // ---- kernels (defined in the .cu files) ------------------------------------------
-cudaError_t launch_pass1(const LaunchCtx& c, const void* K, const void* V, const void* Q,
-                         int* status);
-cudaError_t launch_pass2(const LaunchCtx& c, const void* K, const void* Q, float* s_div_out,
-                         int* status);
+cudaError_t launch_pass1(const LaunchCtx& c, const void* K, const void* Q, int* status);
+cudaError_t launch_merge(const LaunchCtx& c, float* rbar_out);
+cudaError_t launch_pass2(const LaunchCtx& c, const void* K, const void* V, const void* Q,
+                         float* s_div_out, int* status);
 int device_sm_count();
-cudaError_t launch_pool(const LaunchCtx& c, float* s_ex_out);
-cudaError_t launch_mix(const LaunchCtx& c, const float* s_ex, const float* s_div,
-                       const float* rbar_in, float* s_comp, float* rbar_out);
+cudaError_t launch_poolsum(const LaunchCtx& c);
+cudaError_t launch_mixpool(const LaunchCtx& c, const float* s_div, const float* rbar_in,
+                           float* s_ex_out, float* s_comp);
 cudaError_t launch_budget(const LaunchCtx& c, const float* scores, int* counts);
-cudaError_t launch_select(const LaunchCtx& c, const float* scores, const int* counts, int* idx,
-                          int* idx_offsets, int* out_row_offsets);
-cudaError_t launch_gather(const LaunchCtx& c, const void* K, const void* V, const int* idx,
-                          const int* idx_offsets, const int* out_row_offsets, void* K_out,
-                          void* V_out);
+// Selection (and optionally the mix before it and the gather after it) by one CTA cluster per
+// (sequence, head).  scores != nullptr: select on them; else mix first (s_div, rbar_in) and
+// write the mixed scores to s_comp_out.  counts_dev == nullptr: fixed budgets.
+struct TailArgs {
+  const float* scores;
+  const float* s_div;
+  const float* rbar_in;
+  float* s_comp_out;
+  const int* counts_dev;
+  int* counts_out;
+  int* idx;
+  int* idx_offsets;
+  int* out_row_offsets;
+  const void* K;
+  const void* V;
+  void* K_out;
+  void* V_out;
+};
+cudaError_t launch_tail(const LaunchCtx& c, const TailArgs& a);
+// Whether the longest sequence is short enough for the fused mix + select + gather kernel.
+bool tail_can_fuse(const LaunchCtx& c);
+
+// Launch with programmatic dependent launch (and an optional cluster size): the kernel may
+// start while its predecessor in the stream drains; every kernel calls pdl_wait() before it
+// touches global memory.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                       cudaStream_t stream, int cluster, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[2];
+  int n = 0;
+  attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[n].val.programmaticStreamSerializationAllowed = 1;
+  ++n;
+  if (cluster > 1) {
+    attr[n].id = cudaLaunchAttributeClusterDimension;
+    attr[n].val.clusterDim.x = (unsigned)cluster;
+    attr[n].val.clusterDim.y = 1;
+    attr[n].val.clusterDim.z = 1;
+    ++n;
+  }
+  cfg.attrs = attr;
+  cfg.numAttrs = (unsigned)n;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
 
 // ---- device helpers ----------------------------------------------------------------
 __device__ __forceinline__ int find_seq(const int* start, int batch, int x) {
@@ -115,6 +156,19 @@ __device__ __forceinline__ float warp_max(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
   return v;
+}
+
+// Programmatic dependent launch: let the next kernel of the stream be scheduled, and wait
+// until everything before this kernel in the stream has completed and is visible.
+__device__ __forceinline__ void pdl_launch_dependents() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
 }
 
 __device__ __forceinline__ float ex2(float x) {

@@ -1,20 +1,134 @@
-// Everything after the two K passes: finishing the per-head statistics, pooling, the
-// head-wise mix (Eq. 2, Eq. 5), budgets, per-head top-B selection and the gather
-// (Algorithm 1, step 2 and the TopB line).
+// Everything after the two K passes: the per-head scalars, pooling, the head-wise mix (Eq. 2,
+// Eq. 5), budgets, per-head top-B selection and the gather (Algorithm 1, step 2 and the TopB
+// line).  The fixed-budget layer call runs all of it in ONE kernel, k_tail: a cluster of eight
+// CTAs per (sequence, head) mixes the scores of its slice, finds the selection threshold by
+// radix passes whose histograms are combined through distributed shared memory, compacts the
+// kept positions in ascending order and copies the kept K / V rows.
+#include <cooperative_groups.h>
+
 #include "tc_common.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace mixkv {
 
 namespace {
 
-// ----------------------------------------------------------------------------- pool
-// 1-D pooling of the raw attention score over the candidate positions of one sequence,
-// stride 1, half-width k/2; average pooling pads with zeros and divides by k.
+// ------------------------------------------------------------------- per-head scalars
+// Everything Eq. 2 / Eq. 5 need besides the per-position values, folded from the per-segment
+// partials pass 2 left behind.  Computed by one warp; the five results go to sc[0..4]:
+//   s_in_scaled  = (|V_i| - sc[0]) * sc[1]
+//   s_div_scaled = (s_div_i - sc[2]) * sc[3]
+//   sc[4]        = redundancy used by the mix
+__device__ void head_scalars(const SeqTable& st, const Workspace& ws, const int b, const int h,
+                             const int pool_k, const int pool_mode, const int use_vnorm,
+                             const float eps, const float* __restrict__ rbar_in, const int lane,
+                             float* sc) {
+  const int bh = b * st.H + h;
+  const int P = st.cu[b + 1] - st.cu[b] - st.W;
+  float dmin = INFINITY, dmax = -INFINITY, dsum = 0.f, exw = 0.f;
+  float vmin = INFINITY, vmax = -INFINITY, vsum = 0.f;
+  {
+    const int per_head = (st.tile2_start[b + 1] - st.tile2_start[b]) / st.H;
+    const int U0 = st.tile2_start[b] + h * per_head;
+    int k = 0;
+    for (SegIter sg(U0, U0 + per_head, st.nt2, st.g2); sg.valid(); sg.next(), ++k) {
+      if ((k & 31) == lane) {
+        const float4 d4 = ws.dstat[sg.start];
+        dmin = fminf(dmin, d4.x);
+        dmax = fmaxf(dmax, d4.y);
+        dsum += d4.z;
+        exw += d4.w;
+        if (use_vnorm) {
+          const float4 v4 = ws.vstat[sg.start];
+          vmin = fminf(vmin, v4.x);
+          vmax = fmaxf(vmax, v4.y);
+          vsum += v4.z;
+        }
+      }
+    }
+  }
+  float ex;
+  if (pool_mode == MIXKV_POOL_AVG) {
+    // sum of the zero-padded average-pooled score = sum of raw[m] * (windows covering m) / k
+    ex = warp_sum(exw) / (float)pool_k;
+  } else {
+    float e = 0.f;
+    for (int c = st.pchunk_start[b] + lane; c < st.pchunk_start[b + 1]; c += 32)
+      e += ws.exsum[(size_t)h * st.pchunks_total + c];
+    ex = warp_sum(e);
+  }
+  dmin = warp_min(dmin);
+  dmax = warp_max(dmax);
+  dsum = warp_sum(dsum);
+  vmin = warp_min(vmin);
+  vmax = warp_max(vmax);
+  vsum = warp_sum(vsum);
+  if (lane == 0) {
+    const float invP = 1.0f / (float)P;
+    const float mean_ex = ex * invP;
+    float v0 = 0.f, cin = 0.f, mean_imp = mean_ex;
+    if (use_vnorm) {
+      const float vinv = 1.0f / (vmax - vmin + eps);
+      const float mean_in = (vsum * invP - vmin) * vinv;
+      const float a_in = mean_ex / (mean_in + eps);
+      v0 = vmin;
+      cin = vinv * a_in;
+      mean_imp = mean_ex + mean_in * a_in;
+    }
+    const float dinv = 1.0f / (dmax - dmin + eps);
+    const float mean_dn = (dsum * invP - dmin) * dinv;
+    const float a_div = mean_imp / (mean_dn + eps);
+    sc[0] = v0;
+    sc[1] = cin;
+    sc[2] = dmin;
+    sc[3] = dinv * a_div;
+    sc[4] = rbar_in ? rbar_in[bh] : ws.rbar[bh];
+  }
+}
+
+// Pooled attention score at one position from a staged window w[0..k) (centre at w[k/2]);
+// positions outside the candidates were staged as 0 (average) or -inf (max).
+__device__ __forceinline__ float pool_window(const float* w, const int k, const int mode,
+                                             const float invk) {
+  if (mode == MIXKV_POOL_AVG) {
+    float v = 0.f;
+    for (int u = 0; u < k; ++u) v += w[u];
+    return v * invk;
+  }
+  float v = -INFINITY;
+  for (int u = 0; u < k; ++u) v = fmaxf(v, w[u]);
+  return v;
+}
+
+__device__ __forceinline__ float mix_one(const float ex, const float vn, const float dv,
+                                         const float* sc, const int use_vnorm,
+                                         const int mix_mode) {
+  float imp = ex;
+  if (use_vnorm) imp += (vn - sc[0]) * sc[1];
+  const float dsc = (dv - sc[2]) * sc[3];
+  const float r = sc[4];
+  switch (mix_mode) {
+    case MIXKV_MIX_HEADWISE: return (1.0f - r) * imp + r * dsc;   // Eq. 5
+    case MIXKV_MIX_IMPORTANCE_ONLY: return imp;
+    case MIXKV_MIX_DIVERSITY_ONLY: return dv;
+    default: return imp + dsc;
+  }
+}
+
+struct MixParams {
+  int pool_k, pool_mode, use_vnorm, mix_mode;
+  float eps;
+};
+
+// --------------------------------------------------------------------------- poolsum
+// Max pooling only: per-chunk sums of the pooled score (its mean enters Eq. 2).
 __global__ void __launch_bounds__(256)
-k_pool(const SeqTable st, const Workspace ws, float* __restrict__ s_ex_out, const int k,
-       const int mode) {
+k_poolsum(const SeqTable st, const Workspace ws, const int k) {
   __shared__ float tile[kPChunk + 64];
   __shared__ float sred[8];
+  pdl_launch_dependents();
+  pdl_wait();
   const int pcx = blockIdx.x, h = blockIdx.y;
   const int b = find_seq(st.pchunk_start, st.batch, pcx);
   const int P = st.cu[b + 1] - st.cu[b] - st.W;
@@ -22,27 +136,13 @@ k_pool(const SeqTable st, const Workspace ws, float* __restrict__ s_ex_out, cons
   const int p1 = min(p0 + kPChunk, P);
   const size_t poff = (size_t)h * st.Ptot + (st.cu[b] - b * st.W);
   const int half = k >> 1;
-  const float pad = mode == 0 ? 0.f : -INFINITY;
   for (int t = threadIdx.x; t < (p1 - p0) + 2 * half; t += 256) {
     const int i = p0 - half + t;
-    tile[t] = (i >= 0 && i < P) ? ws.s_ex_raw[poff + i] : pad;
+    tile[t] = (i >= 0 && i < P) ? ws.s_ex_raw[poff + i] : -INFINITY;
   }
   __syncthreads();
   float sum = 0.f;
-  const float invk = 1.0f / (float)k;
-  for (int t = threadIdx.x; t < p1 - p0; t += 256) {
-    float v;
-    if (mode == 0) {
-      v = 0.f;
-      for (int u = 0; u < k; ++u) v += tile[t + u];
-      v *= invk;
-    } else {
-      v = -INFINITY;
-      for (int u = 0; u < k; ++u) v = fmaxf(v, tile[t + u]);
-    }
-    s_ex_out[poff + p0 + t] = v;
-    sum += v;
-  }
+  for (int t = threadIdx.x; t < p1 - p0; t += 256) sum += pool_window(tile + t, k, MIXKV_POOL_MAX, 0.f);
   sum = warp_sum(sum);
   if ((threadIdx.x & 31) == 0) sred[threadIdx.x >> 5] = sum;
   __syncthreads();
@@ -53,85 +153,39 @@ k_pool(const SeqTable st, const Workspace ws, float* __restrict__ s_ex_out, cons
   }
 }
 
-// ------------------------------------------------------------------------------ mix
-// Eq. 2 and Eq. 5.  Every CTA first rebuilds the scalars of its (sequence, head) from the
-// per-chunk partials (a few dozen values), then mixes its slice.
+// --------------------------------------------------------------------------- mixpool
+// Pooling and the mix over a grid of position chunks (the scores entry point, adaptive budgets).
 __global__ void __launch_bounds__(256)
-k_mix(const SeqTable st, const Workspace ws, const float* __restrict__ s_ex,
-      const float* __restrict__ s_div, const float* __restrict__ rbar_in,
-      float* __restrict__ s_comp, float* __restrict__ rbar_out, const int use_vnorm,
-      const int mix_mode, const float eps) {
+k_mixpool(const SeqTable st, const Workspace ws, const float* __restrict__ s_div,
+          const float* __restrict__ rbar_in, float* __restrict__ s_ex_out,
+          float* __restrict__ s_comp, const MixParams mp) {
+  __shared__ float tile[kPChunk + 64];
   __shared__ float sc[8];
+  pdl_launch_dependents();
+  pdl_wait();
   const int pcx = blockIdx.x, h = blockIdx.y;
   const int b = find_seq(st.pchunk_start, st.batch, pcx);
-  const int bh = b * st.H + h;
   const int P = st.cu[b + 1] - st.cu[b] - st.W;
   const int p0 = (pcx - st.pchunk_start[b]) * kPChunk;
   const int p1 = min(p0 + kPChunk, P);
   const size_t poff = (size_t)h * st.Ptot + (st.cu[b] - b * st.W);
-  if (threadIdx.x < 32) {
-    const int lane = threadIdx.x;
-    float ex = 0.f;
-    for (int c = st.pchunk_start[b] + lane; c < st.pchunk_start[b + 1]; c += 32)
-      ex += ws.exsum[(size_t)h * st.pchunks_total + c];
-    float a = INFINITY, bb = -INFINITY, s = 0.f;
-    {
-      const int per_head = (st.tile2_start[b + 1] - st.tile2_start[b]) / st.H;
-      const int U0 = st.tile2_start[b] + h * per_head;
-      int k = 0;
-      for (SegIter sg(U0, U0 + per_head, st.nt2, st.g2); sg.valid(); sg.next(), ++k) {
-        if ((k & 31) == lane) {
-          const float4 v = ws.dstat[sg.start];
-          a = fminf(a, v.x);
-          bb = fmaxf(bb, v.y);
-          s += v.z;
-        }
-      }
-    }
-    ex = warp_sum(ex);
-    a = warp_min(a);
-    bb = warp_max(bb);
-    s = warp_sum(s);
-    if (lane == 0) {
-      const float invP = 1.0f / (float)P;
-      const float mean_ex = ex * invP;
-      float vmin = 0.f, vinv = 0.f, a_in = 0.f, mean_imp = mean_ex;
-      if (use_vnorm) {
-        const float4 v = ws.vfinal[bh];
-        vmin = v.x;
-        vinv = 1.0f / (v.y - v.x + eps);
-        const float mean_in = (v.z * invP - v.x) * vinv;
-        a_in = mean_ex / (mean_in + eps);
-        mean_imp = mean_ex + mean_in * a_in;
-      }
-      const float dinv = 1.0f / (bb - a + eps);
-      const float mean_dn = (s * invP - a) * dinv;
-      const float a_div = mean_imp / (mean_dn + eps);
-      const float r = rbar_in ? rbar_in[bh] : ws.rbar[bh];
-      sc[0] = vmin;
-      sc[1] = vinv * a_in;     // s_in_scaled = (n - vmin) * sc[1]
-      sc[2] = a;
-      sc[3] = dinv * a_div;    // s_div_scaled = (s_div - dmin) * sc[3]
-      sc[4] = r;
-      if (rbar_out && pcx == st.pchunk_start[b]) rbar_out[bh] = ws.rbar[bh];
-    }
+  const int half = mp.pool_k >> 1;
+  const float pad = mp.pool_mode == MIXKV_POOL_AVG ? 0.f : -INFINITY;
+  if (threadIdx.x < 32)
+    head_scalars(st, ws, b, h, mp.pool_k, mp.pool_mode, mp.use_vnorm, mp.eps, rbar_in,
+                 threadIdx.x, sc);
+  for (int t = threadIdx.x; t < (p1 - p0) + 2 * half; t += 256) {
+    const int i = p0 - half + t;
+    tile[t] = (i >= 0 && i < P) ? ws.s_ex_raw[poff + i] : pad;
   }
   __syncthreads();
-  const float vmin = sc[0], cin = sc[1], dmin = sc[2], cdiv = sc[3], r = sc[4];
-  for (int i = p0 + threadIdx.x; i < p1; i += 256) {
-    const float ex = s_ex[poff + i];
-    const float dv = s_div[poff + i];
-    float imp = ex;
-    if (use_vnorm) imp += (ws.vnorm[poff + i] - vmin) * cin;
-    const float dsc = (dv - dmin) * cdiv;
-    float c;
-    switch (mix_mode) {
-      case MIXKV_MIX_HEADWISE: c = (1.0f - r) * imp + r * dsc; break;
-      case MIXKV_MIX_IMPORTANCE_ONLY: c = imp; break;
-      case MIXKV_MIX_DIVERSITY_ONLY: c = dv; break;
-      default: c = imp + dsc; break;
-    }
-    s_comp[poff + i] = c;
+  const float invk = 1.0f / (float)mp.pool_k;
+  for (int t = threadIdx.x; t < p1 - p0; t += 256) {
+    const int i = p0 + t;
+    const float ex = pool_window(tile + t, mp.pool_k, mp.pool_mode, invk);
+    if (s_ex_out) s_ex_out[poff + i] = ex;
+    const float vn = mp.use_vnorm ? ws.vnorm[poff + i] : 0.f;
+    s_comp[poff + i] = mix_one(ex, vn, s_div[poff + i], sc, mp.use_vnorm, mp.mix_mode);
   }
 }
 
@@ -159,9 +213,16 @@ __device__ void radix_threshold(const float* base, size_t stride, int n_rows, in
     __syncthreads();
     for (int r = 0; r < n_rows; ++r) {
       const float* row = base + (size_t)r * stride;
-      for (int i = threadIdx.x; i < len; i += blockDim.x) {
-        const unsigned key = order_key(row[i]);
-        if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
+      for (int i0 = 0; i0 < len; i0 += blockDim.x) {   // uniform trip count: full-warp votes
+        const int i = i0 + threadIdx.x;
+        unsigned digit = 0xffffffffu;
+        if (i < len) {
+          const unsigned key = order_key(row[i]);
+          if ((key & mask) == prefix) digit = (key >> shift) & 255u;
+        }
+        const unsigned peers = __match_any_sync(0xffffffffu, digit);
+        if (digit != 0xffffffffu && (int)(__ffs(peers) - 1) == (int)(threadIdx.x & 31))
+          atomicAdd(&hist[digit], __popc(peers));
       }
     }
     __syncthreads();
@@ -184,18 +245,16 @@ __device__ void radix_threshold(const float* base, size_t stride, int n_rows, in
   *need_eq = remaining;
 }
 
-// Head budgets of one sequence.  Fixed: min(B - W, P).  Adaptive: see mixkv.h.
+// Head budgets of one sequence under the adaptive rule (see mixkv.h).
 __global__ void __launch_bounds__(1024)
 k_budget(const SeqTable st, const float* __restrict__ scores, int* __restrict__ counts,
-         const int budget_mode, const int Bp, const int floor_slots) {
+         const int Bp, const int floor_slots) {
   __shared__ int hist[256];
   __shared__ int s_gt[64], s_eq[64];
+  pdl_launch_dependents();
+  pdl_wait();
   const int b = blockIdx.x, H = st.H;
   const int P = st.cu[b + 1] - st.cu[b] - st.W;
-  if (budget_mode == MIXKV_BUDGET_FIXED) {
-    for (int h = threadIdx.x; h < H; h += blockDim.x) counts[b * H + h] = min(Bp, P);
-    return;
-  }
   const long long total = (long long)H * P;
   long long N = (long long)H * (Bp - floor_slots);
   if (N > total) N = total;
@@ -237,131 +296,274 @@ k_budget(const SeqTable st, const float* __restrict__ scores, int* __restrict__ 
   }
 }
 
-// Per (sequence, head) top-b selection, ascending position order.
-__global__ void __launch_bounds__(1024)
-k_select(const SeqTable st, const float* __restrict__ scores, const int* __restrict__ counts,
-         int* __restrict__ idx, int* __restrict__ idx_offsets, int* __restrict__ out_row_offsets) {
-  __shared__ int hist[256];
-  __shared__ int s_gt[32], s_eq[32];
+// ------------------------------------------------------------------------------ tail
+constexpr int kTailCluster = 8;
+constexpr int kTailThreads = 512;
+constexpr int kTailCacheCap = 16384;   // positions one CTA keeps in shared memory
+
+struct TailKernelArgs {
+  const float* scores;        // select on these (FUSED == false)
+  const float* s_div;         // FUSED: parts of the mix
+  const float* rbar_in;
+  float* s_comp_out;          // FUSED: mixed scores are written here
+  const int* counts_dev;      // adaptive budgets; nullptr = fixed
+  int* counts_out;
+  int* idx;
+  int* idx_offsets;
+  int* out_row_offsets;       // may be nullptr
+  const __nv_bfloat16* K;     // gather when K_out != nullptr
+  const __nv_bfloat16* V;
+  __nv_bfloat16* K_out;
+  __nv_bfloat16* V_out;
+  int Bp;                     // B - W
+  int cached;                 // keys of the slice fit the shared-memory cache
+  MixParams mp;
+};
+
+// Selected rows of (b', h') pairs before bh, fixed budgets.
+__device__ __forceinline__ int fixed_offset(const SeqTable& st, int bh, int Bp) {
+  const int b = bh / st.H, h = bh % st.H;
+  int off = 0;
+  for (int x = 0; x < b; ++x) off += st.H * min(Bp, st.cu[x + 1] - st.cu[x] - st.W);
+  if (b < st.batch) off += h * min(Bp, st.cu[b + 1] - st.cu[b] - st.W);
+  return off;
+}
+
+template <bool FUSED>
+__global__ void __launch_bounds__(kTailThreads, 1)
+k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
+  extern __shared__ __align__(16) unsigned char tail_smem[];
+  __shared__ int hist[2][256];
+  __shared__ int s_scan[16][2];
+  __shared__ int s_tot[2];
+  __shared__ int s_sel[2];      // digit, remaining
   __shared__ int s_off;
-  const int bh = blockIdx.x, b = bh / st.H, h = bh % st.H;
+  __shared__ float sc[8];
+  cg::cluster_group cluster = cg::this_cluster();
+  const int crank = (int)cluster.block_rank();
+  const int bh = blockIdx.x / kTailCluster, b = bh / st.H, h = bh % st.H;
   const int BH = st.batch * st.H;
-  const int P = st.cu[b + 1] - st.cu[b] - st.W;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  // where this (b, h) starts in the packed outputs
-  {
-    int part = 0;
-    for (int t = tid; t < bh; t += blockDim.x) part += counts[t];
-    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
-    if (lane == 0) s_gt[warp] = part;
-    __syncthreads();
-    if (tid == 0) {
-      int off = 0;
-      for (int w = 0; w < 32; ++w) off += s_gt[w];
+  const int W = st.W;
+  const int P = st.cu[b + 1] - st.cu[b] - W;
+  const size_t poff = (size_t)h * st.Ptot + (st.cu[b] - b * W);
+  // slice of this CTA: positions [c0, c0 + n); thread t owns the run [c0 + t*R, c0 + (t+1)*R)
+  const int chunk = (P + kTailCluster - 1) / kTailCluster;
+  const int R = (chunk + kTailThreads - 1) / kTailThreads;
+  const int c0 = min(crank * chunk, P);
+  const int n = min(chunk, P - c0);
+  const int r0 = tid * R, r1 = min(r0 + R, n);   // local run of this thread (may be empty)
+  unsigned* skeys = reinterpret_cast<unsigned*>(tail_smem);            // [R * kTailThreads]
+  float* sraw = reinterpret_cast<float*>(tail_smem) + (size_t)R * kTailThreads;  // FUSED stage
+
+  pdl_launch_dependents();
+  pdl_wait();
+
+  // ---- budget and output offsets of this (b, h)
+  int want;
+  if (tid < 32) {
+    int off = 0, cnt;
+    if (a.counts_dev) {
+      for (int t = lane; t < bh; t += 32) off += a.counts_dev[t];
+      for (int o = 16; o > 0; o >>= 1) off += __shfl_xor_sync(0xffffffffu, off, o);
+      cnt = a.counts_dev[bh];
+    } else {
+      off = fixed_offset(st, bh, a.Bp);
+      cnt = min(a.Bp, P);
+    }
+    if (lane == 0) {
       s_off = off;
-      idx_offsets[bh] = off;
-      if (out_row_offsets) out_row_offsets[bh] = off + bh * st.W;
-      if (bh == BH - 1) {
-        idx_offsets[BH] = off + counts[bh];
-        if (out_row_offsets) out_row_offsets[BH] = off + counts[bh] + BH * st.W;
+      s_sel[1] = cnt;
+      if (crank == 0) {
+        a.idx_offsets[bh] = off;
+        if (a.counts_out) a.counts_out[bh] = cnt;
+        if (a.out_row_offsets) a.out_row_offsets[bh] = off + bh * W;
+        if (bh == BH - 1) {
+          a.idx_offsets[BH] = off + cnt;
+          if (a.out_row_offsets) a.out_row_offsets[BH] = off + cnt + BH * W;
+        }
       }
     }
+  }
+  const float* src = a.scores;
+  if (FUSED) {
+    // ---- pooling and mix of this slice (Eq. 2, Eq. 5); the mixed scores go to s_comp_out
+    const int half = a.mp.pool_k >> 1;
+    const float pad = a.mp.pool_mode == MIXKV_POOL_AVG ? 0.f : -INFINITY;
+    if (warp == 1)
+      head_scalars(st, ws, b, h, a.mp.pool_k, a.mp.pool_mode, a.mp.use_vnorm, a.mp.eps, a.rbar_in,
+                   lane, sc);
+    for (int t = tid; t < n + 2 * half; t += kTailThreads) {
+      const int i = c0 - half + t;
+      sraw[t] = (i >= 0 && i < P) ? ws.s_ex_raw[poff + i] : pad;
+    }
     __syncthreads();
+    const float invk = 1.0f / (float)a.mp.pool_k;
+    for (int j = r0; j < r1; ++j) {
+      const int i = c0 + j;
+      const float ex = pool_window(sraw + j, a.mp.pool_k, a.mp.pool_mode, invk);
+      const float vn = a.mp.use_vnorm ? ws.vnorm[poff + i] : 0.f;
+      const float c = mix_one(ex, vn, a.s_div[poff + i], sc, a.mp.use_vnorm, a.mp.mix_mode);
+      a.s_comp_out[poff + i] = c;
+      skeys[(j - r0) * kTailThreads + tid] = order_key(c);
+    }
+    src = a.s_comp_out;
+  } else if (a.cached) {
+    for (int j = r0; j < r1; ++j) skeys[(j - r0) * kTailThreads + tid] = order_key(src[poff + c0 + j]);
   }
-  const int want = counts[bh];
-  int* out = idx + s_off;
-  if (want <= 0) return;
+  __syncthreads();
+  want = s_sel[1];
+  int* out = a.idx + s_off;
+  const bool cached = FUSED || a.cached;
+  auto key_at = [&](int j) -> unsigned {
+    return cached ? skeys[(j - r0) * kTailThreads + tid] : order_key(src[poff + c0 + j]);
+  };
+
+  bool all = false;
+  unsigned tau = 0;
+  int need_eq = 0;
   if (want >= P) {
-    for (int i = tid; i < P; i += blockDim.x) out[i] = i;
-    return;
+    all = true;     // keep every candidate
+  } else if (want > 0) {
+    // ---- threshold: the want-th largest key of the head, four 8-bit digit passes
+    unsigned prefix = 0, mask = 0;
+    int remaining = want;
+    for (int t = tid; t < 256; t += kTailThreads) hist[0][t] = 0;
+    __syncthreads();
+    for (int pass = 0; pass < 4; ++pass) {
+      const int shift = 24 - 8 * pass, buf = pass & 1;
+      for (int e = 0; e < R; ++e) {   // same trip count in every lane: full-warp votes
+        const int j = r0 + e;
+        unsigned digit = 0xffffffffu;
+        if (j < r1) {
+          const unsigned key = key_at(j);
+          if ((key & mask) == prefix) digit = (key >> shift) & 255u;
+        }
+        const unsigned peers = __match_any_sync(0xffffffffu, digit);
+        if (digit != 0xffffffffu && (int)(__ffs(peers) - 1) == lane)
+          atomicAdd(&hist[buf][digit], __popc(peers));
+      }
+      cluster.sync();
+      // every CTA adds up the cluster's histograms and finds the digit itself
+      int tot = 0;
+      if (tid < 256) {
+#pragma unroll
+        for (int r = 0; r < kTailCluster; ++r)
+          tot += *cluster.map_shared_rank(&hist[buf][tid], r);
+        hist[buf ^ 1][tid] = 0;   // every CTA is past its reads of the other buffer
+      }
+      // suffix sums over the 256 bins: bins above this one
+      int incl = tot;
+      if (tid < 256) {
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int v = __shfl_down_sync(0xffffffffu, incl, o);
+          if (lane + o < 32) incl += v;
+        }
+        if (lane == 0) s_scan[warp][0] = incl;
+      }
+      __syncthreads();
+      if (tid < 256) {
+        int above = incl - tot;
+        for (int w = warp + 1; w < 8; ++w) above += s_scan[w][0];
+        if (above < remaining && remaining <= above + tot) {
+          s_sel[0] = tid;
+          s_sel[1] = remaining - above;
+        }
+      }
+      __syncthreads();
+      prefix |= (unsigned)s_sel[0] << shift;
+      remaining = s_sel[1];
+      mask |= 255u << shift;
+      __syncthreads();
+    }
+    tau = prefix;
+    need_eq = remaining;
   }
-  const float* row = scores + (size_t)h * st.Ptot + (st.cu[b] - b * st.W);
-  unsigned tau;
-  int need_eq;
-  radix_threshold(row, 0, 1, P, want, hist, &tau, &need_eq);
-  // ordered compaction: thread t owns the contiguous positions [t*per, (t+1)*per)
-  const int per = (P + blockDim.x - 1) / blockDim.x;
-  const int lo = min(tid * per, P), hi = min(lo + per, P);
-  int gt = 0, eq = 0;
-  for (int i = lo; i < hi; ++i) {
-    const unsigned key = order_key(row[i]);
-    gt += key > tau;
-    eq += key == tau;
-  }
-  // exclusive scan of (gt, eq) over the CTA
-  int gt_inc = gt, eq_inc = eq;
-  for (int o = 1; o < 32; o <<= 1) {
-    const int a = __shfl_up_sync(0xffffffffu, gt_inc, o);
-    const int c = __shfl_up_sync(0xffffffffu, eq_inc, o);
-    if (lane >= o) gt_inc += a, eq_inc += c;
-  }
-  if (lane == 31) s_gt[warp] = gt_inc, s_eq[warp] = eq_inc;
-  __syncthreads();
-  if (warp == 0) {
-    int a = s_gt[lane], c = s_eq[lane];
-    int ai = a, ci = c;
+
+  // ---- ordered compaction: positions with key > tau, plus the first need_eq with key == tau
+  if (want > 0) {
+    int gt = 0, eq = 0;
+    if (all) {
+      gt = max(r1 - r0, 0);
+    } else {
+      for (int j = r0; j < r1; ++j) {
+        const unsigned key = key_at(j);
+        gt += key > tau;
+        eq += key == tau;
+      }
+    }
+    int gt_inc = gt, eq_inc = eq;
+#pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-      const int x = __shfl_up_sync(0xffffffffu, ai, o);
-      const int y = __shfl_up_sync(0xffffffffu, ci, o);
-      if (lane >= o) ai += x, ci += y;
+      const int x = __shfl_up_sync(0xffffffffu, gt_inc, o);
+      const int y = __shfl_up_sync(0xffffffffu, eq_inc, o);
+      if (lane >= o) gt_inc += x, eq_inc += y;
     }
-    s_gt[lane] = ai - a;
-    s_eq[lane] = ci - c;
+    if (lane == 31) s_scan[warp][0] = gt_inc, s_scan[warp][1] = eq_inc;
+    __syncthreads();
+    int gt_before = gt_inc - gt, eq_before = eq_inc - eq;
+    for (int w = 0; w < warp; ++w) gt_before += s_scan[w][0], eq_before += s_scan[w][1];
+    if (tid == kTailThreads - 1) {
+      s_tot[0] = gt_before + gt;
+      s_tot[1] = eq_before + eq;
+    }
+    cluster.sync();
+    for (int r = 0; r < crank; ++r) {
+      const int* t = cluster.map_shared_rank(&s_tot[0], r);
+      gt_before += t[0];
+      eq_before += t[1];
+    }
+    for (int j = r0; j < r1; ++j) {
+      const int i = c0 + j;
+      if (all) {
+        out[gt_before++] = i;
+        continue;
+      }
+      const unsigned key = key_at(j);
+      if (key > tau) {
+        out[gt_before + min(eq_before, need_eq)] = i;
+        ++gt_before;
+      } else if (key == tau) {
+        if (eq_before < need_eq) out[gt_before + eq_before] = i;
+        ++eq_before;
+      }
+    }
   }
-  __syncthreads();
-  int gt_before = s_gt[warp] + gt_inc - gt;
-  int eq_before = s_eq[warp] + eq_inc - eq;
-  for (int i = lo; i < hi; ++i) {
-    const unsigned key = order_key(row[i]);
-    if (key > tau) {
-      out[gt_before + min(eq_before, need_eq)] = i;
-      ++gt_before;
-    } else if (key == tau) {
-      if (eq_before < need_eq) out[gt_before + eq_before] = i;
-      ++eq_before;
+  // the index list is complete (and visible to the cluster) after this barrier; it also keeps
+  // every CTA's shared memory alive until its peers have read it
+  cluster.sync();
+
+  // ---- gather: selected rows in ascending position order, then the W window rows
+  if (a.K_out) {
+    const int n_sel = max(want, 0) < P ? max(want, 0) : P;
+    const int rows = n_sel + W;
+    const size_t srow0 = (size_t)h * st.Ltot + st.cu[b];
+    const size_t drow0 = (size_t)(s_off + bh * W);
+    const int hw = tid >> 4, l = tid & 15;                       // 32 half-warps, 16 B per lane
+    constexpr int kRowsPerSweep = kTailCluster * (kTailThreads / 16);
+    for (int rb = crank * (kTailThreads / 16) + hw; rb < rows; rb += 2 * kRowsPerSweep) {
+      const int ra = rb + kRowsPerSweep;
+      const int sa = rb < n_sel ? __ldcg(out + rb) : P + (rb - n_sel);
+      const int sb = ra < rows ? (ra < n_sel ? __ldcg(out + ra) : P + (ra - n_sel)) : -1;
+      const uint4 k0 = __ldg(reinterpret_cast<const uint4*>(a.K + (srow0 + sa) * kHeadDim) + l);
+      const uint4 v0 = __ldg(reinterpret_cast<const uint4*>(a.V + (srow0 + sa) * kHeadDim) + l);
+      uint4 k1 = make_uint4(0, 0, 0, 0), v1 = k1;
+      if (sb >= 0) {
+        k1 = __ldg(reinterpret_cast<const uint4*>(a.K + (srow0 + sb) * kHeadDim) + l);
+        v1 = __ldg(reinterpret_cast<const uint4*>(a.V + (srow0 + sb) * kHeadDim) + l);
+      }
+      reinterpret_cast<uint4*>(a.K_out + (drow0 + rb) * kHeadDim)[l] = k0;
+      reinterpret_cast<uint4*>(a.V_out + (drow0 + rb) * kHeadDim)[l] = v0;
+      if (sb >= 0) {
+        reinterpret_cast<uint4*>(a.K_out + (drow0 + ra) * kHeadDim)[l] = k1;
+        reinterpret_cast<uint4*>(a.V_out + (drow0 + ra) * kHeadDim)[l] = v1;
+      }
     }
   }
 }
 
-// --------------------------------------------------------------------------- gather
-// One half-warp per output row (16 lanes x 16 bytes = one 256-byte bf16 row).
-__global__ void __launch_bounds__(256)
-k_gather(const SeqTable st, const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* __restrict__ V,
-         const int* __restrict__ idx, const int* __restrict__ idx_offsets,
-         const int* __restrict__ out_row_offsets, __nv_bfloat16* __restrict__ K_out,
-         __nv_bfloat16* __restrict__ V_out) {
-  const int bh = blockIdx.y, b = bh / st.H, h = bh % st.H;
-  const int n_sel = idx_offsets[bh + 1] - idx_offsets[bh];
-  const int rows = n_sel + st.W;
-  const int r = blockIdx.x * 16 + (threadIdx.x >> 4);
-  if (r >= rows) return;
-  const int P = st.cu[b + 1] - st.cu[b] - st.W;
-  const int src = r < n_sel ? idx[idx_offsets[bh] + r] : P + (r - n_sel);
-  const size_t srow = (size_t)h * st.Ltot + st.cu[b] + src;
-  const size_t drow = (size_t)out_row_offsets[bh] + r;
-  const int l = threadIdx.x & 15;
-  const __nv_bfloat16* X = blockIdx.z == 0 ? K : V;
-  __nv_bfloat16* Y = blockIdx.z == 0 ? K_out : V_out;
-  reinterpret_cast<uint4*>(Y + drow * kHeadDim)[l] =
-      __ldg(reinterpret_cast<const uint4*>(X + srow * kHeadDim) + l);
-}
-
-}  // namespace
-
-cudaError_t launch_pool(const LaunchCtx& c, float* s_ex_out) {
-  k_pool<<<dim3(c.st.pchunks_total, c.st.H), 256, 0, c.stream>>>(c.st, c.ws, s_ex_out,
-                                                                 c.p.pool_kernel, c.p.pool_mode);
-  return cudaGetLastError();
-}
-
-cudaError_t launch_mix(const LaunchCtx& c, const float* s_ex, const float* s_div,
-                       const float* rbar_in, float* s_comp, float* rbar_out) {
-  k_mix<<<dim3(c.st.pchunks_total, c.st.H), 256, 0, c.stream>>>(
-      c.st, c.ws, s_ex, s_div, rbar_in, s_comp, rbar_out, c.p.use_vnorm, c.p.mix_mode, c.p.eps);
-  return cudaGetLastError();
-}
-
-static int floor_slots(const mixkv_params& p) {
+int floor_slots(const mixkv_params& p) {
   const int Bp = p.budget - p.window;
   int f = (int)floor((double)p.ada_floor * (double)Bp);
   if (f > Bp) f = Bp;
@@ -369,37 +571,82 @@ static int floor_slots(const mixkv_params& p) {
   return f;
 }
 
+MixParams mix_params(const mixkv_params& p) {
+  MixParams mp;
+  mp.pool_k = p.pool_kernel;
+  mp.pool_mode = p.pool_mode;
+  mp.use_vnorm = p.use_vnorm;
+  mp.mix_mode = p.mix_mode;
+  mp.eps = p.eps;
+  return mp;
+}
+
+}  // namespace
+
+cudaError_t launch_poolsum(const LaunchCtx& c) {
+  return launch_pdl(k_poolsum, dim3(c.st.pchunks_total, c.st.H), dim3(256), 0, c.stream, 1, c.st,
+                    c.ws, c.p.pool_kernel);
+}
+
+cudaError_t launch_mixpool(const LaunchCtx& c, const float* s_div, const float* rbar_in,
+                           float* s_ex_out, float* s_comp) {
+  return launch_pdl(k_mixpool, dim3(c.st.pchunks_total, c.st.H), dim3(256), 0, c.stream, 1, c.st,
+                    c.ws, s_div, rbar_in, s_ex_out, s_comp, mix_params(c.p));
+}
+
 cudaError_t launch_budget(const LaunchCtx& c, const float* scores, int* counts) {
-  const int threads = c.p.budget_mode == MIXKV_BUDGET_FIXED ? 64 : 1024;
-  k_budget<<<c.st.batch, threads, 0, c.stream>>>(c.st, scores, counts, c.p.budget_mode,
-                                                 c.p.budget - c.p.window, floor_slots(c.p));
-  return cudaGetLastError();
+  return launch_pdl(k_budget, dim3(c.st.batch), dim3(1024), 0, c.stream, 1, c.st, scores, counts,
+                    c.p.budget - c.p.window, floor_slots(c.p));
 }
 
-cudaError_t launch_select(const LaunchCtx& c, const float* scores, const int* counts, int* idx,
-                          int* idx_offsets, int* out_row_offsets) {
-  k_select<<<c.st.batch * c.st.H, 1024, 0, c.stream>>>(c.st, scores, counts, idx, idx_offsets,
-                                                       out_row_offsets);
-  return cudaGetLastError();
+bool tail_can_fuse(const LaunchCtx& c) {
+  const int chunk = (c.max_prefix + kTailCluster - 1) / kTailCluster;
+  return chunk <= kTailCacheCap;
 }
 
-cudaError_t launch_gather(const LaunchCtx& c, const void* K, const void* V, const int* idx,
-                          const int* idx_offsets, const int* out_row_offsets, void* K_out,
-                          void* V_out) {
-  // upper bound of rows any (b, h) can own
-  const int Bp = c.p.budget - c.p.window;
-  long long max_sel = Bp;
-  if (c.p.budget_mode == MIXKV_BUDGET_ADAPTIVE) {
-    const int f = floor_slots(c.p);
-    max_sel = (long long)f + (long long)c.st.H * (Bp - f);
+cudaError_t launch_tail(const LaunchCtx& c, const TailArgs& t) {
+  TailKernelArgs a;
+  a.scores = t.scores;
+  a.s_div = t.s_div;
+  a.rbar_in = t.rbar_in;
+  a.s_comp_out = t.s_comp_out;
+  a.counts_dev = t.counts_dev;
+  a.counts_out = t.counts_out;
+  a.idx = t.idx;
+  a.idx_offsets = t.idx_offsets;
+  a.out_row_offsets = t.out_row_offsets;
+  a.K = (const __nv_bfloat16*)t.K;
+  a.V = (const __nv_bfloat16*)t.V;
+  a.K_out = (__nv_bfloat16*)t.K_out;
+  a.V_out = (__nv_bfloat16*)t.V_out;
+  a.Bp = c.p.budget - c.p.window;
+  a.mp = mix_params(c.p);
+  const int chunk = (c.max_prefix + kTailCluster - 1) / kTailCluster;
+  const int R = (chunk + kTailThreads - 1) / kTailThreads;
+  const bool fused = t.scores == nullptr;
+  a.cached = chunk <= kTailCacheCap ? 1 : 0;
+  if (fused && !a.cached) return cudaErrorInvalidValue;   // callers check tail_can_fuse() first
+  size_t smem = 0;
+  if (a.cached) smem += (size_t)R * kTailThreads * 4;
+  if (fused) smem += ((size_t)chunk + 64) * 4;
+  static size_t set_fused[64] = {0}, set_plain[64] = {0};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  size_t* have = fused ? set_fused : set_plain;
+  if (smem > 48 * 1024 && (dev < 0 || dev >= 64 || have[dev] < smem)) {
+    const size_t ask = 2 * ((size_t)kTailCacheCap + 512) * 4 + 256;
+    e = fused ? cudaFuncSetAttribute(k_tail<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ask)
+              : cudaFuncSetAttribute(k_tail<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ask);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64) have[dev] = ask;
   }
-  if (max_sel > c.max_prefix) max_sel = c.max_prefix;
-  const int max_rows = (int)max_sel + c.st.W;
-  const dim3 grid((max_rows + 15) / 16, c.st.batch * c.st.H, 2);
-  k_gather<<<grid, 256, 0, c.stream>>>(c.st, (const __nv_bfloat16*)K, (const __nv_bfloat16*)V, idx,
-                                       idx_offsets, out_row_offsets, (__nv_bfloat16*)K_out,
-                                       (__nv_bfloat16*)V_out);
-  return cudaGetLastError();
+  const dim3 grid(c.st.batch * c.st.H * kTailCluster);
+  if (fused)
+    return launch_pdl(k_tail<true>, grid, dim3(kTailThreads), smem, c.stream, kTailCluster, c.st,
+                      c.ws, a);
+  return launch_pdl(k_tail<false>, grid, dim3(kTailThreads), smem, c.stream, kTailCluster, c.st,
+                    c.ws, a);
 }
 
 }  // namespace mixkv
