@@ -59,6 +59,27 @@ __device__ __forceinline__ void drain_ring(uint64_t* full, int stages, int it) {
   }
 }
 
+// Packed fp32 pairs (one instruction for two lanes of arithmetic).
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float a, float b) {
+  f32x2 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float& a, float& b) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+  f32x2 d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
+  f32x2 d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+
 // ======================================================================== pass 1
 constexpr int kP1Stages = 4;   // K tile ring
 
@@ -94,15 +115,19 @@ __device__ __forceinline__ void softmax_chunk(uint32_t (&r)[32], const bool need
     z_run *= ex2(m_run - mn);
     m_run = mn;
   }
-  float z0 = 0.f, z1 = 0.f, z2 = 0.f, z3 = 0.f;
+  const f32x2 sc2 = pack2(scale_log2e, scale_log2e), nm2 = pack2(-m_run, -m_run);
+  f32x2 za = pack2(0.f, 0.f), zb = za;
 #pragma unroll
   for (int j = 0; j < 32; j += 4) {
-    z0 += ex2(fmaf(__uint_as_float(r[j]), scale_log2e, -m_run));
-    z1 += ex2(fmaf(__uint_as_float(r[j + 1]), scale_log2e, -m_run));
-    z2 += ex2(fmaf(__uint_as_float(r[j + 2]), scale_log2e, -m_run));
-    z3 += ex2(fmaf(__uint_as_float(r[j + 3]), scale_log2e, -m_run));
+    float a0, a1, b0, b1;
+    unpack2(fma2(pack2(__uint_as_float(r[j]), __uint_as_float(r[j + 1])), sc2, nm2), a0, a1);
+    unpack2(fma2(pack2(__uint_as_float(r[j + 2]), __uint_as_float(r[j + 3])), sc2, nm2), b0, b1);
+    za = add2(za, pack2(ex2(a0), ex2(a1)));
+    zb = add2(zb, pack2(ex2(b0), ex2(b1)));
   }
-  z_run += (z0 + z1) + (z2 + z3);
+  float z0, z1;
+  unpack2(add2(za, zb), z0, z1);
+  z_run += z0 + z1;
 }
 
 // grid = g1 persistent CTAs: TMA, MMA, 2 idle, 8 epilogue, 4 key-statistics warps.
@@ -116,9 +141,8 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
   constexpr int QR = MB * 128;                 // query rows the MMA reads
   unsigned char* sQ = base;                    // 2 halves x [QR x 128 B]
   unsigned char* sK = sQ + 2 * QR * 128;       // kP1Stages x 32 KB
-  float* skinv = reinterpret_cast<float*>(sK + kP1Stages * kTileBytes);  // [kP1Stages][128]
-  float* sks = skinv + kP1Stages * 128;        // [2][128] key-sum exchange
-  P1Bars* bars = reinterpret_cast<P1Bars*>(sks + 256);
+  float* sks = reinterpret_cast<float*>(sK + kP1Stages * kTileBytes);  // [8][128] key-sum exchange
+  P1Bars* bars = reinterpret_cast<P1Bars*>(sks + 1024);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int NQ = st.NQ, W = st.W, H = st.H;
@@ -162,23 +186,23 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
   if (warp == kWarpTma) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      int it = 0, segn = 0, prev_bh = -1;
-      for (int id = lo; id < hi; ++id) {
-        const TileCoord tc = tile_coord(st.tile1_start, st.batch, H, id);
-        if (tc.bh != prev_bh) {
+      int it = 0, segn = 0;
+      bool seg_start = true;
+      for (TileIter ti(st.tile1_start, st.batch, H, lo, hi); ti.valid(); ti.next()) {
+        if (seg_start) {
           if (segn > 0 && !mbar_wait(&bars->qfree, (segn - 1) & 1, abort)) break;
           mbar_expect_tx(&bars->qfull, NQ * 256);
-          tma_load_2d(sQ, &tmQ, 0, tc.bh * NQ, &bars->qfull);
-          tma_load_2d(sQ + QR * 128, &tmQ, 64, tc.bh * NQ, &bars->qfull);
+          tma_load_2d(sQ, &tmQ, 0, ti.bh() * NQ, &bars->qfull);
+          tma_load_2d(sQ + QR * 128, &tmQ, 64, ti.bh() * NQ, &bars->qfull);
           ++segn;
-          prev_bh = tc.bh;
         }
+        seg_start = ti.seg_last();
         const int s = it % kP1Stages, ph = (it / kP1Stages) & 1;
         if (!mbar_wait(&bars->empty[s], ph ^ 1, abort)) break;
         mbar_expect_tx(&bars->full[s], kTileBytes);
-        const int y = st.cu[tc.b] + tc.t * kTile;
-        tma_load_3d(sK + s * kTileBytes, &tmK, 0, y, tc.h, &bars->full[s]);
-        tma_load_3d(sK + s * kTileBytes + kHalfBytes, &tmK, 64, y, tc.h, &bars->full[s]);
+        const int y = st.cu[ti.b] + ti.t * kTile;
+        tma_load_3d(sK + s * kTileBytes, &tmK, 0, y, ti.h, &bars->full[s]);
+        tma_load_3d(sK + s * kTileBytes + kHalfBytes, &tmK, 64, y, ti.h, &bars->full[s]);
         ++it;
       }
       if (*abort) {
@@ -190,14 +214,14 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       constexpr uint32_t idesc = umma_idesc_bf16(128, kTile);
-      int it = 0, segn = 0, prev_bh = -1;
-      for (int id = lo; id < hi; ++id) {
-        const TileCoord tc = tile_coord(st.tile1_start, st.batch, H, id);
-        if (tc.bh != prev_bh) {
+      int it = 0, segn = 0;
+      bool seg_start = true;
+      for (TileIter ti(st.tile1_start, st.batch, H, lo, hi); ti.valid(); ti.next()) {
+        if (seg_start) {
           if (!mbar_wait(&bars->qfull, segn & 1, abort)) break;
           ++segn;
-          prev_bh = tc.bh;
         }
+        seg_start = ti.seg_last();
         const int s = it % kP1Stages, ph = (it / kP1Stages) & 1, ts = it & 1, tph = (it >> 1) & 1;
         if (!mbar_wait(&bars->full[s], ph, abort)) break;
         if (!mbar_wait(&bars->tempty[ts], tph ^ 1, abort)) break;
@@ -215,9 +239,7 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
         }
         umma_commit(&bars->empty[s]);
         umma_commit(&bars->tfull[ts]);
-        bool last = id + 1 == hi;
-        if (!last) last = tile_coord(st.tile1_start, st.batch, H, id + 1).bh != tc.bh;
-        if (last) umma_commit(&bars->qfree);
+        if (seg_start) umma_commit(&bars->qfree);
         ++it;
       }
       if (*abort) raise(status, abort);
@@ -234,22 +256,22 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
     const bool warp_on = (MB == 2 ? wg * 128 : 0) + quarter * 32 < NQ;
     const int jrow = row % W;
     float m_run = -1e30f, z_run = 0.f;
-    int it = 0, prev_bh = -1, seg_first = lo;
-    for (int id = lo; id < hi; ++id) {
-      const TileCoord tc = tile_coord(st.tile1_start, st.batch, H, id);
-      if (tc.bh != prev_bh) {
+    int it = 0, seg_first = lo;
+    bool seg_start = true;
+    for (TileIter ti(st.tile1_start, st.batch, H, lo, hi); ti.valid(); ti.next()) {
+      if (seg_start) {
         m_run = -1e30f;
         z_run = 0.f;
-        seg_first = id;
-        prev_bh = tc.bh;
+        seg_first = ti.id;
       }
-      const int L = st.cu[tc.b + 1] - st.cu[tc.b], P = L - W;
+      seg_start = ti.seg_last();
+      const int L = st.cu[ti.b + 1] - st.cu[ti.b], P = L - W;
       const int ts = it & 1, tph = (it >> 1) & 1;
       if (!mbar_wait(&bars->tfull[ts], tph, abort)) break;
       tc_fence_after();
       if (warp_on) {
-        const int k0 = tc.t * kTile + (MB == 2 ? 0 : wg * 64);
-        const bool need_mask = tc.t * kTile + kTile > P;
+        const int k0 = ti.t * kTile + (MB == 2 ? 0 : wg * 64);
+        const bool need_mask = ti.t * kTile + kTile > P;
         const int lim = P + jrow;   // last key this row may see
         const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + ts * (MB * 128) + col0;
         uint32_t ra[32], rb[32];
@@ -268,72 +290,93 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
       }
       tc_fence_before();
       mbar_arrive(&bars->tempty[ts]);
-      bool last = id + 1 == hi;
-      if (!last) last = tile_coord(st.tile1_start, st.batch, H, id + 1).bh != tc.bh;
-      if (last && row < NQ)
+      if (seg_start && row < NQ)
         ws.rowstat[((size_t)seg_first * 2 + unit) * NQ + row] = make_float2(m_run, z_run);
       ++it;
     }
   } else if (warp >= kAuxWarp0) {
     // ------------------------------------------------------------------ key statistics
-    const int kt = tid - kAuxWarp0 * 32;         // 0..127: key row of the tile (norm phase)
-    const int wd = kt & 63, hk = kt >> 6;        // word (dims 2wd, 2wd+1) and key half (sum phase)
-    float a0 = 0.f, a1 = 0.f;
-    int it = 0, prev_bh = -1, seg_first = lo;
-    for (int id = lo; id < hi; ++id) {
-      const TileCoord tc = tile_coord(st.tile1_start, st.batch, H, id);
-      if (tc.bh != prev_bh) {
-        a0 = a1 = 0.f;
-        seg_first = id;
-        prev_bh = tc.bh;
+    // Sixteen lanes share a key row (one 16-byte chunk each); a 16-lane group owns 16 rows of
+    // the tile.  Sweep 1 squares, a butterfly leaves the squared norm of row c with lane c,
+    // sweep 2 adds the rows scaled by 1/|k| into eight per-thread sums (dims 8c .. 8c+7).
+    const int kt = tid - kAuxWarp0 * 32;         // 0..127
+    const int grp = kt >> 4, c = kt & 15;
+    const int chalf = c >> 3, cc = c & 7;
+    float acc[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+    int it = 0, seg_first = lo;
+    bool seg_start = true;
+    for (TileIter ti(st.tile1_start, st.batch, H, lo, hi); ti.valid(); ti.next()) {
+      if (seg_start) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+        seg_first = ti.id;
       }
-      const int L = st.cu[tc.b + 1] - st.cu[tc.b];
+      seg_start = ti.seg_last();
+      const int L = st.cu[ti.b + 1] - st.cu[ti.b];
       const int s = it % kP1Stages, ph = (it / kP1Stages) & 1;
-      mbar_wait(&bars->full[s], ph, abort);
-      const unsigned char* tile = sK + s * kTileBytes;
-      float ss0 = 0.f, ss1 = 0.f;
+      const bool ok = mbar_wait(&bars->full[s], ph, abort);
+      const unsigned char* tile = sK + s * kTileBytes + chalf * kHalfBytes;
+      // two batches of eight rows keep the register footprint small
 #pragma unroll
-      for (int half = 0; half < 2; ++half) {
+      for (int bt = 0; bt < 2; ++bt) {
+        uint4 u[8];
+        float p[8];
 #pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          const uint4 u = *reinterpret_cast<const uint4*>(tile + half * kHalfBytes + sw128_offset(kt, c));
-          const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&u);
+        for (int rr = 0; rr < 8; ++rr) {
+          u[rr] = *reinterpret_cast<const uint4*>(tile + sw128_offset(grp * 16 + bt * 8 + rr, cc));
+          const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&u[rr]);
+          float s0 = 0.f, s1 = 0.f;
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             const float2 f = __bfloat1622float2(p2[e]);
-            ss0 = fmaf(f.x, f.x, ss0);
-            ss1 = fmaf(f.y, f.y, ss1);
+            s0 = fmaf(f.x, f.x, s0);
+            s1 = fmaf(f.y, f.y, s1);
+          }
+          p[rr] = s0 + s1;
+        }
+        // butterfly over the 16 lanes of the group: lanes 2r and 2r+1 end with the total of row r
+#pragma unroll
+        for (int o = 8; o >= 2; o >>= 1) {
+          const bool up = (c & o) != 0;
+#pragma unroll
+          for (int k = 0; k < o / 2; ++k) {
+            const float send = up ? p[k] : p[k + o / 2];
+            const float keep = up ? p[k + o / 2] : p[k];
+            p[k] = keep + __shfl_xor_sync(0xffffffffu, send, o);
+          }
+        }
+        p[0] += __shfl_xor_sync(0xffffffffu, p[0], 1);
+        if (bt == 1) {   // the tile now lives in registers: hand the stage back to the producer
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&bars->empty[s]);
+        }
+        const int i = ti.t * kTile + grp * 16 + bt * 8 + (c >> 1);   // the row this lane holds
+        const float inv = (ok && i < L && p[0] > 0.f) ? rsqrtf(p[0]) : 0.f;
+        if (i < L && (c & 1) == 0) ws.kinv[(size_t)ti.h * st.Ltot + st.cu[ti.b] + i] = inv;
+#pragma unroll
+        for (int rr = 0; rr < 8; ++rr) {
+          const float w = __shfl_sync(0xffffffffu, inv, (lane & 16) | (rr << 1));
+          const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&u[rr]);
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float2 f = __bfloat1622float2(p2[e]);
+            acc[2 * e] = fmaf(f.x, w, acc[2 * e]);
+            acc[2 * e + 1] = fmaf(f.y, w, acc[2 * e + 1]);
           }
         }
       }
-      const float ss = ss0 + ss1;
-      const int i = tc.t * kTile + kt;
-      const float inv = (i < L && ss > 0.f) ? 1.0f / sqrtf(ss) : 0.f;
-      skinv[s * 128 + kt] = inv;
-      if (i < L) ws.kinv[(size_t)tc.h * st.Ltot + st.cu[tc.b] + i] = inv;
       if (group_sync_stop(2, 128, kt == 0, abort, bars->vote, it)) break;
-      {
-        const unsigned char* colbase = tile + (wd >> 5) * kHalfBytes + (wd & 3) * 4;
-        const int chunk = (wd & 31) >> 2;
-#pragma unroll 8
-        for (int rr = 0; rr < 64; ++rr) {
-          const int r = hk * 64 + rr;
-          const float2 f = __bfloat1622float2(
-              *reinterpret_cast<const __nv_bfloat162*>(colbase + sw128_offset(r, chunk)));
-          const float w = skinv[s * 128 + r];
-          a0 = fmaf(f.x, w, a0);
-          a1 = fmaf(f.y, w, a1);
-        }
-      }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&bars->empty[s]);
-      bool last = id + 1 == hi;
-      if (!last) last = tile_coord(st.tile1_start, st.batch, H, id + 1).bh != tc.bh;
-      if (last) {
-        sks[hk * 128 + 2 * wd] = a0;
-        sks[hk * 128 + 2 * wd + 1] = a1;
+      if (seg_start) {
+        // fold the eight row groups: sks[grp][dim]
+#pragma unroll
+        for (int e = 0; e < 8; ++e) sks[grp * 128 + c * 8 + e] = acc[e];
         named_bar_sync(2, 128);
-        ws.ksum[(size_t)seg_first * kHeadDim + kt] = sks[kt] + sks[128 + kt];
+        float t = 0.f;
+#pragma unroll
+        for (int g2 = 0; g2 < 8; ++g2) t += sks[g2 * 128 + kt];
+        ws.ksum[(size_t)seg_first * kHeadDim + kt] = t;
         named_bar_sync(2, 128);
       }
       ++it;
@@ -346,10 +389,14 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
 }
 
 // ========================================================================= merge
-// One CTA per (sequence, head): folds the per-segment partials of pass 1.
+// One CTA per (sequence, head): folds the per-segment partials of pass 1.  Warps take segments
+// side by side so that the loads of different segments are in flight together.
 __global__ void __launch_bounds__(256)
 k_merge(const SeqTable st, const Workspace ws, float* __restrict__ rbar_out) {
-  __shared__ float sred[8];
+  __shared__ float2 part[8][256];
+  __shared__ float kpart[2][kHeadDim];
+  __shared__ int sstart[256];
+  __shared__ float sred[4];
   pdl_launch_dependents();
   pdl_wait();
   const int bh = blockIdx.x, b = bh / st.H, h = bh % st.H;
@@ -357,39 +404,56 @@ k_merge(const SeqTable st, const Workspace ws, float* __restrict__ rbar_out) {
   const int NQ = st.NQ;
   const int L = st.cu[b + 1] - st.cu[b];
   const int per_head = (st.tile1_start[b + 1] - st.tile1_start[b]) / st.H;
-  const int T0 = st.tile1_start[b] + h * per_head;
-  // pass 1 left one partial per segment of this (b, h): segment e starts at T0 for e = 0 and at
-  // the first tile of CTA c0 + e otherwise
-  const int c0 = tile_owner(T0, st.nt1, st.g1);
-  const int nseg = tile_owner(T0 + per_head - 1, st.nt1, st.g1) - c0 + 1;
-  if (tid < NQ) {
-    const int nunits = NQ <= 128 ? 2 : 1;
-    float M = -1e30f, Z = 0.f;
-#pragma unroll 4
-    for (int e = 0; e < nseg; ++e) {
-      const int start = e == 0 ? T0 : cta_first_tile(c0 + e, st.nt1, st.g1);
+  const SegList sl(st.tile1_start[b] + h * per_head, per_head, st.nt1, st.g1);
+  const int nunits = NQ <= 128 ? 2 : 1;
+  float M[8], Z[8];
+#pragma unroll
+  for (int r = 0; r < 8; ++r) M[r] = -1e30f, Z[r] = 0.f;
+  float ks = 0.f;
+  const int kd = tid & (kHeadDim - 1), kpar = tid >> 7;
+  for (int e0 = 0; e0 < sl.nseg; e0 += 256) {
+    const int ne = min(256, sl.nseg - e0);
+    __syncthreads();
+    if (tid < ne) sstart[tid] = sl.start(e0 + tid);
+    __syncthreads();
+#pragma unroll 2
+    for (int e = warp; e < ne; e += 8) {
       for (int u = 0; u < nunits; ++u) {
-        const float2 mz = ws.rowstat[((size_t)start * 2 + u) * NQ + tid];
-        const float mn = fmaxf(M, mz.x);
-        Z = Z * exp2f(M - mn) + mz.y * exp2f(mz.x - mn);
-        M = mn;
+        const float2* src = ws.rowstat + ((size_t)sstart[e] * 2 + u) * NQ;
+#pragma unroll
+        for (int r = 0; r < 8; ++r) {
+          const int q = lane + 32 * r;
+          if (q < NQ) {
+            const float2 mz = src[q];
+            const float mn = fmaxf(M[r], mz.x);
+            Z[r] = Z[r] * ex2(M[r] - mn) + mz.y * ex2(mz.x - mn);
+            M[r] = mn;
+          }
+        }
       }
     }
-    // log2 of (Z * W): the 1/W of the window mean is folded into the normaliser
-    ws.bq[(size_t)bh * NQ + tid] = M + log2f(Z * (float)st.W);
-  }
-  float s = 0.f;
-  if (tid < kHeadDim) {
 #pragma unroll 4
-    for (int e = 0; e < nseg; ++e) {
-      const int start = e == 0 ? T0 : cta_first_tile(c0 + e, st.nt1, st.g1);
-      s += ws.ksum[(size_t)start * kHeadDim + tid];
-    }
+    for (int e = kpar; e < ne; e += 2) ks += ws.ksum[(size_t)sstart[e] * kHeadDim + kd];
   }
-  const float n2 = warp_sum(s * s);
-  if (lane == 0) sred[warp] = n2;
+#pragma unroll
+  for (int r = 0; r < 8; ++r) part[warp][lane + 32 * r] = make_float2(M[r], Z[r]);
+  kpart[kpar][kd] = ks;
+  __syncthreads();
+  if (tid < NQ) {
+    float Mx = -1e30f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) Mx = fmaxf(Mx, part[w][tid].x);
+    float Zs = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) Zs += part[w][tid].y * exp2f(part[w][tid].x - Mx);
+    // log2 of (Z * W): the 1/W of the window mean is folded into the normaliser
+    ws.bq[(size_t)bh * NQ + tid] = Mx + (log2f(Zs) + log2f((float)st.W));
+  }
   __nv_bfloat16* rows = ws.kbar_rows + (size_t)bh * kExtraRows * kHeadDim;
   if (tid < kHeadDim) {
+    const float s = kpart[0][tid] + kpart[1][tid];
+    const float n2 = warp_sum(s * s);
+    if (lane == 0) sred[warp] = n2;
     const float kb = s / (float)L;
     const __nv_bfloat16 p0 = __float2bfloat16_rn(kb);
     const float r1 = kb - __bfloat162float(p0);
@@ -413,15 +477,15 @@ k_merge(const SeqTable st, const Workspace ws, float* __restrict__ rbar_out) {
 
 // ======================================================================== pass 2
 constexpr int kP2KStages = 3;              // K tiles (32 KB each)
-constexpr int kP2VStages = 3;              // V half tiles: 64 rows, 16 KB each
+constexpr int kP2VStagesMax = 4;           // V half tiles: 64 rows, 16 KB each
 constexpr int kVSubBytes = 64 * 256;
-constexpr int kNBMax = kMaxNQ + kExtraRows;
+constexpr size_t kSmemLimit = 227 * 1024;
 
 struct P2Bars {
   uint64_t kfull[kP2KStages];
   uint64_t kempty[kP2KStages];
-  uint64_t vfull[kP2VStages];
-  uint64_t vempty[kP2VStages];
+  uint64_t vfull[kP2VStagesMax];
+  uint64_t vempty[kP2VStagesMax];
   uint64_t tfull[2];
   uint64_t tempty[2];
   uint64_t qfull;
@@ -433,32 +497,37 @@ struct P2Bars {
 
 // Sixteen logit columns of one key: adds exp2(logit * scale - normaliser of the column).
 __device__ __forceinline__ void colsum_chunk(const uint32_t (&r)[16], const float* nb_smem,
-                                             const float scale_log2e, float& acc0, float& acc1) {
+                                             const f32x2 sc2, f32x2& acc) {
 #pragma unroll
   for (int j = 0; j < 16; j += 4) {
-    const float4 nb = *reinterpret_cast<const float4*>(nb_smem + j);
-    acc0 += ex2(fmaf(__uint_as_float(r[j]), scale_log2e, -nb.x));
-    acc1 += ex2(fmaf(__uint_as_float(r[j + 1]), scale_log2e, -nb.y));
-    acc0 += ex2(fmaf(__uint_as_float(r[j + 2]), scale_log2e, -nb.z));
-    acc1 += ex2(fmaf(__uint_as_float(r[j + 3]), scale_log2e, -nb.w));
+    const float4 nb = *reinterpret_cast<const float4*>(nb_smem + j);   // negated normalisers
+    float a0, a1, b0, b1;
+    unpack2(fma2(pack2(__uint_as_float(r[j]), __uint_as_float(r[j + 1])), sc2, pack2(nb.x, nb.y)),
+            a0, a1);
+    unpack2(fma2(pack2(__uint_as_float(r[j + 2]), __uint_as_float(r[j + 3])), sc2,
+                 pack2(nb.z, nb.w)),
+            b0, b1);
+    acc = add2(acc, pack2(ex2(a0), ex2(a1)));
+    acc = add2(acc, pack2(ex2(b0), ex2(b1)));
   }
 }
 
-// grid = g2 persistent CTAs: TMA, MMA, 2 idle, 8 epilogue, 4 value-norm warps.
+// grid = g2 persistent CTAs: K producer, MMA, V producer, 1 idle, 8 epilogue, 4 value-norm warps.
 __global__ void __launch_bounds__(kThreads, 1)
 k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
         const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKB,
         const SeqTable st, const Workspace ws, float* __restrict__ s_div_out,
-        const float scale_log2e, const int use_vnorm, const int pool_half, int* status) {
+        const float scale_log2e, const int use_vnorm, const int pool_half, const int vstages,
+        int* status) {
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* base =
       reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
   const int NQ = st.NQ, W = st.W, H = st.H;
   const int NB = NQ + kExtraRows;             // rows of the B operand
   unsigned char* sQ = base;                   // 2 halves x [NB x 128 B]
-  unsigned char* sK = sQ + 2 * kNBMax * 128;  // kP2KStages x 32 KB
-  unsigned char* sV = sK + kP2KStages * kTileBytes;   // kP2VStages x 16 KB
-  float* sbq = reinterpret_cast<float*>(sV + kP2VStages * kVSubBytes);  // [256]
+  unsigned char* sK = sQ + 2 * NB * 128;      // kP2KStages x 32 KB
+  unsigned char* sV = sK + kP2KStages * kTileBytes;   // vstages x 16 KB
+  float* sbq = reinterpret_cast<float*>(sV + vstages * kVSubBytes);  // [256] negated normalisers
   float* sx = sbq + 256;                      // [2][128] partial sums WG0 -> WG1
   float* sred = sx + 256;                     // [32]
   P2Bars* bars = reinterpret_cast<P2Bars*>(sred + 32);
@@ -467,6 +536,7 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
   const int lo = cta_first_tile(blockIdx.x, st.nt2, st.g2);
   const int hi = cta_first_tile(blockIdx.x + 1, st.nt2, st.g2);
   volatile int* abort = &bars->abort;
+  constexpr int kWarpTmaV = 2;
 
   pdl_launch_dependents();
   if (tid == 0) {
@@ -474,7 +544,7 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
       mbar_init(&bars->kfull[s], 1);
       mbar_init(&bars->kempty[s], 1);
     }
-    for (int s = 0; s < kP2VStages; ++s) {
+    for (int s = 0; s < kP2VStagesMax; ++s) {
       mbar_init(&bars->vfull[s], 1);
       mbar_init(&bars->vempty[s], 2);      // the two warps that read a half tile
     }
@@ -490,10 +560,10 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
   if (warp == kWarpMma) tmem_alloc(&bars->tmem_base, 512);
   if (warp == kWarpTma && lane == 0) {
     tma_prefetch_desc(&tmK);
-    tma_prefetch_desc(&tmV);
     tma_prefetch_desc(&tmQ);
     tma_prefetch_desc(&tmKB);
   }
+  if (warp == kWarpTmaV && lane == 0) tma_prefetch_desc(&tmV);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -501,62 +571,71 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
   pdl_wait();
 
   if (warp == kWarpTma) {
-    // ------------------------------------------------------------------ TMA producer
+    // ------------------------------------------------------------------ K / Q producer
     if (lane == 0) {
-      int it = 0, vit = 0, segn = 0, prev_bh = -1;
-      bool ok = true;
-      for (int id = lo; id < hi && ok; ++id) {
-        const TileCoord tc = tile_coord(st.tile2_start, st.batch, H, id);
-        if (tc.bh != prev_bh) {
+      int it = 0, segn = 0;
+      bool seg_start = true;
+      for (TileIter ti(st.tile2_start, st.batch, H, lo, hi); ti.valid(); ti.next()) {
+        if (seg_start) {
           if (segn > 0 && !mbar_wait(&bars->qfree, (segn - 1) & 1, abort)) break;
           mbar_expect_tx(&bars->qfull, NB * 256);
-          tma_load_2d(sQ, &tmQ, 0, tc.bh * NQ, &bars->qfull);
-          tma_load_2d(sQ + NB * 128, &tmQ, 64, tc.bh * NQ, &bars->qfull);
-          tma_load_2d(sQ + NQ * 128, &tmKB, 0, tc.bh * kExtraRows, &bars->qfull);
-          tma_load_2d(sQ + NB * 128 + NQ * 128, &tmKB, 64, tc.bh * kExtraRows, &bars->qfull);
+          tma_load_2d(sQ, &tmQ, 0, ti.bh() * NQ, &bars->qfull);
+          tma_load_2d(sQ + NB * 128, &tmQ, 64, ti.bh() * NQ, &bars->qfull);
+          tma_load_2d(sQ + NQ * 128, &tmKB, 0, ti.bh() * kExtraRows, &bars->qfull);
+          tma_load_2d(sQ + NB * 128 + NQ * 128, &tmKB, 64, ti.bh() * kExtraRows, &bars->qfull);
           ++segn;
-          prev_bh = tc.bh;
         }
+        seg_start = ti.seg_last();
         const int s = it % kP2KStages, ph = (it / kP2KStages) & 1;
         if (!mbar_wait(&bars->kempty[s], ph ^ 1, abort)) break;
         mbar_expect_tx(&bars->kfull[s], kTileBytes);
-        const int y = st.cu[tc.b] + tc.t * kTile;
-        tma_load_3d(sK + s * kTileBytes, &tmK, 0, y, tc.h, &bars->kfull[s]);
-        tma_load_3d(sK + s * kTileBytes + kHalfBytes, &tmK, 64, y, tc.h, &bars->kfull[s]);
+        const int y = st.cu[ti.b] + ti.t * kTile;
+        tma_load_3d(sK + s * kTileBytes, &tmK, 0, y, ti.h, &bars->kfull[s]);
+        tma_load_3d(sK + s * kTileBytes + kHalfBytes, &tmK, 64, y, ti.h, &bars->kfull[s]);
         ++it;
-        if (use_vnorm) {
-          for (int sub = 0; sub < 2; ++sub) {
-            const int vs = vit % kP2VStages, vph = (vit / kP2VStages) & 1;
-            if (!mbar_wait(&bars->vempty[vs], vph ^ 1, abort)) {
-              ok = false;
-              break;
-            }
-            mbar_expect_tx(&bars->vfull[vs], kVSubBytes);
-            unsigned char* dst = sV + vs * kVSubBytes;
-            tma_load_3d(dst, &tmV, 0, y + sub * 64, tc.h, &bars->vfull[vs]);
-            tma_load_3d(dst + kVSubBytes / 2, &tmV, 64, y + sub * 64, tc.h, &bars->vfull[vs]);
-            ++vit;
-          }
-        }
       }
       if (*abort) {
         raise(status, abort);
         drain_ring(bars->kfull, kP2KStages, it);
-        drain_ring(bars->vfull, kP2VStages, vit);
+      }
+    }
+  } else if (warp == kWarpTmaV) {
+    // ------------------------------------------------------------------ V producer
+    if (lane == 0 && use_vnorm) {
+      int vit = 0;
+      bool ok = true;
+      for (TileIter ti(st.tile2_start, st.batch, H, lo, hi); ti.valid() && ok; ti.next()) {
+        const int y = st.cu[ti.b] + ti.t * kTile;
+        for (int sub = 0; sub < 2; ++sub) {
+          const int vs = vit % vstages, vph = (vit / vstages) & 1;
+          if (!mbar_wait(&bars->vempty[vs], vph ^ 1, abort)) {
+            ok = false;
+            break;
+          }
+          mbar_expect_tx(&bars->vfull[vs], kVSubBytes);
+          unsigned char* dst = sV + vs * kVSubBytes;
+          tma_load_3d(dst, &tmV, 0, y + sub * 64, ti.h, &bars->vfull[vs]);
+          tma_load_3d(dst + kVSubBytes / 2, &tmV, 64, y + sub * 64, ti.h, &bars->vfull[vs]);
+          ++vit;
+        }
+      }
+      if (*abort) {
+        raise(status, abort);
+        drain_ring(bars->vfull, vstages, vit);
       }
     }
   } else if (warp == kWarpMma) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       const uint32_t idesc = umma_idesc_bf16(128, NB);
-      int it = 0, segn = 0, prev_bh = -1;
-      for (int id = lo; id < hi; ++id) {
-        const TileCoord tc = tile_coord(st.tile2_start, st.batch, H, id);
-        if (tc.bh != prev_bh) {
+      int it = 0, segn = 0;
+      bool seg_start = true;
+      for (TileIter ti(st.tile2_start, st.batch, H, lo, hi); ti.valid(); ti.next()) {
+        if (seg_start) {
           if (!mbar_wait(&bars->qfull, segn & 1, abort)) break;
           ++segn;
-          prev_bh = tc.bh;
         }
+        seg_start = ti.seg_last();
         const int s = it % kP2KStages, ph = (it / kP2KStages) & 1, ts = it & 1, tph = (it >> 1) & 1;
         if (!mbar_wait(&bars->kfull[s], ph, abort)) break;
         if (!mbar_wait(&bars->tempty[ts], tph ^ 1, abort)) break;
@@ -570,9 +649,7 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
         }
         umma_commit(&bars->kempty[s]);
         umma_commit(&bars->tfull[ts]);
-        bool last = id + 1 == hi;
-        if (!last) last = tile_coord(st.tile2_start, st.batch, H, id + 1).bh != tc.bh;
-        if (last) umma_commit(&bars->qfree);
+        if (seg_start) umma_commit(&bars->qfree);
         ++it;
       }
       if (*abort) raise(status, abort);
@@ -586,27 +663,29 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
     const int CA = ((NQ / 16 + 1) >> 1) * 16;
     const int cbeg = wg == 0 ? 0 : CA;
     const int nch = (wg == 0 ? CA : NQ - CA) / 16;
+    const f32x2 sc2 = pack2(scale_log2e, scale_log2e);
     float dmin = INFINITY, dmax = -INFINITY, dsum = 0.f, exw = 0.f;
-    int it = 0, prev_bh = -1, seg_first = lo;
-    for (int id = lo; id < hi; ++id) {
-      const TileCoord tc = tile_coord(st.tile2_start, st.batch, H, id);
-      const int L = st.cu[tc.b + 1] - st.cu[tc.b], P = L - W;
-      if (tc.bh != prev_bh) {
+    int it = 0, seg_first = lo;
+    bool seg_start = true;
+    for (TileIter ti(st.tile2_start, st.batch, H, lo, hi); ti.valid(); ti.next()) {
+      const int L = st.cu[ti.b + 1] - st.cu[ti.b], P = L - W;
+      if (seg_start) {
         named_bar_sync(1, kEpiThreads);   // the previous segment's readers of sbq are done
-        if (et < NQ) sbq[et] = ws.bq[(size_t)tc.bh * NQ + et];
+        if (et < NQ) sbq[et] = -ws.bq[(size_t)ti.bh() * NQ + et];
         dmin = INFINITY, dmax = -INFINITY, dsum = 0.f, exw = 0.f;
-        seg_first = id;
-        prev_bh = tc.bh;
+        seg_first = ti.id;
         named_bar_sync(1, kEpiThreads);
       }
+      seg_start = ti.seg_last();
       const int ts = it & 1, tph = (it >> 1) & 1;
-      const int ikey = tc.t * kTile + key;
+      const int ikey = ti.t * kTile + key;
       float kinv_i = 0.f;
-      if (wg == 1 && ikey < P) kinv_i = ws.kinv[(size_t)tc.h * st.Ltot + st.cu[tc.b] + ikey];
+      if (wg == 1 && ikey < P) kinv_i = ws.kinv[(size_t)ti.h * st.Ltot + st.cu[ti.b] + ikey];
       const bool ok = mbar_wait(&bars->tfull[ts], tph, abort);
       tc_fence_after();
       const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + ts * 256;
-      float acc0 = 0.f, acc1 = 0.f, dot = 0.f;
+      f32x2 acc = pack2(0.f, 0.f);
+      float dot = 0.f;
       if (ok) {
         uint32_t rd[4];
         if (wg == 1) tmem_ld4(taddr + NQ, rd);
@@ -619,13 +698,13 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
             tmem_ld_wait();
             tmem_ld_fence(ra);
             if (ci + 1 < nch) tmem_ld16(taddr + cbeg + (ci + 1) * 16, rb);
-            colsum_chunk(ra, sbq + cbeg + ci * 16, scale_log2e, acc0, acc1);
+            colsum_chunk(ra, sbq + cbeg + ci * 16, sc2, acc);
           }
           if (ci + 1 < nch) {
             tmem_ld_wait();
             tmem_ld_fence(rb);
             if (ci + 2 < nch) tmem_ld16(taddr + cbeg + (ci + 2) * 16, ra);
-            colsum_chunk(rb, sbq + cbeg + (ci + 1) * 16, scale_log2e, acc0, acc1);
+            colsum_chunk(rb, sbq + cbeg + (ci + 1) * 16, sc2, acc);
           }
         }
         if (wg == 1) {
@@ -636,11 +715,13 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
       }
       tc_fence_before();
       mbar_arrive(&bars->tempty[ts]);
+      float acc0, acc1;
+      unpack2(acc, acc0, acc1);
       if (wg == 0) sx[ts * 128 + key] = acc0 + acc1;
       if (group_sync_stop(1, kEpiThreads, et == 0, abort, bars->vote[0], it)) break;
       if (wg == 1) {
         if (ikey < P) {
-          const size_t poff = (size_t)tc.h * st.Ptot + (st.cu[tc.b] - tc.b * W);
+          const size_t poff = (size_t)ti.h * st.Ptot + (st.cu[ti.b] - ti.b * W);
           const float ex = (acc0 + acc1) + sx[ts * 128 + key];
           ws.s_ex_raw[poff + ikey] = ex;
           const float sd = -dot * kinv_i;
@@ -652,9 +733,7 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
           const int cover = min(ikey, pool_half) + min(P - 1 - ikey, pool_half) + 1;
           exw = fmaf(ex, (float)cover, exw);
         }
-        bool last = id + 1 == hi;
-        if (!last) last = tile_coord(st.tile2_start, st.batch, H, id + 1).bh != tc.bh;
-        if (last) {
+        if (seg_start) {
           const float a = warp_min(dmin), b2 = warp_max(dmax), c2 = warp_sum(dsum),
                       d2 = warp_sum(exw);
           if (lane == 0) {
@@ -683,20 +762,20 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
     const int vt = tid - kAuxWarp0 * 32;         // 0..127
     const int sub = vt >> 6, vr = vt & 63;
     float vmin = INFINITY, vmax = -INFINITY, vsum = 0.f;
-    int it = 0, prev_bh = -1, seg_first = lo;
-    for (int id = lo; id < hi; ++id) {
-      const TileCoord tc = tile_coord(st.tile2_start, st.batch, H, id);
-      if (tc.bh != prev_bh) {
+    int it = 0, seg_first = lo;
+    bool seg_start = true;
+    for (TileIter ti(st.tile2_start, st.batch, H, lo, hi); ti.valid(); ti.next()) {
+      if (seg_start) {
         vmin = INFINITY, vmax = -INFINITY, vsum = 0.f;
-        seg_first = id;
-        prev_bh = tc.bh;
+        seg_first = ti.id;
       }
-      const int P = st.cu[tc.b + 1] - st.cu[tc.b] - W;
+      seg_start = ti.seg_last();
+      const int P = st.cu[ti.b + 1] - st.cu[ti.b] - W;
       const int vit = 2 * it + sub;
-      const int vs = vit % kP2VStages, vph = (vit / kP2VStages) & 1;
+      const int vs = vit % vstages, vph = (vit / vstages) & 1;
       const bool ok = mbar_wait(&bars->vfull[vs], vph, abort);
       const unsigned char* tile = sV + vs * kVSubBytes;
-      float ss0 = 0.f, ss1 = 0.f;
+      float ss[4] = {0.f, 0.f, 0.f, 0.f};
       if (ok) {
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
@@ -708,26 +787,24 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
               const float2 f = __bfloat1622float2(p2[e]);
-              ss0 = fmaf(f.x, f.x, ss0);
-              ss1 = fmaf(f.y, f.y, ss1);
+              ss[e & 1] = fmaf(f.x, f.x, ss[e & 1]);
+              ss[2 + (e & 1)] = fmaf(f.y, f.y, ss[2 + (e & 1)]);
             }
           }
         }
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(&bars->vempty[vs]);
-      const int i = tc.t * kTile + sub * 64 + vr;
+      const int i = ti.t * kTile + sub * 64 + vr;
       if (ok && i < P) {
-        const float n = sqrtf(ss0 + ss1);
-        ws.vnorm[(size_t)tc.h * st.Ptot + (st.cu[tc.b] - tc.b * W) + i] = n;
+        const float n = sqrtf((ss[0] + ss[1]) + (ss[2] + ss[3]));
+        ws.vnorm[(size_t)ti.h * st.Ptot + (st.cu[ti.b] - ti.b * W) + i] = n;
         vmin = fminf(vmin, n);
         vmax = fmaxf(vmax, n);
         vsum += n;
       }
       if (group_sync_stop(3, 128, vt == 0, abort, bars->vote[1], it)) break;
-      bool last = id + 1 == hi;
-      if (!last) last = tile_coord(st.tile2_start, st.batch, H, id + 1).bh != tc.bh;
-      if (last) {
+      if (seg_start) {
         const float a = warp_min(vmin), b2 = warp_max(vmax), c2 = warp_sum(vsum);
         const int vw = warp - kAuxWarp0;
         if (lane == 0) {
@@ -798,12 +875,12 @@ bool map_rows2d(const void* X, long long rows, int box_rows, CUtensorMap* tm) {
 }
 
 size_t pass1_smem(int MB) {
-  return 1024 + (size_t)2 * MB * 128 * 128 + kP1Stages * kTileBytes + kP1Stages * 128 * 4 +
-         256 * 4 + sizeof(P1Bars) + 64;
+  return 1024 + (size_t)2 * MB * 128 * 128 + kP1Stages * kTileBytes + 1024 * 4 + sizeof(P1Bars) +
+         64;
 }
-size_t pass2_smem() {
-  return 1024 + (size_t)2 * kNBMax * 128 + kP2KStages * kTileBytes + kP2VStages * kVSubBytes +
-         256 * 4 + 256 * 4 + 32 * 4 + sizeof(P2Bars) + 64;
+size_t pass2_smem(int NQ, int vstages) {
+  return 1024 + (size_t)2 * (NQ + kExtraRows) * 128 + kP2KStages * kTileBytes +
+         (size_t)vstages * kVSubBytes + 256 * 4 + 256 * 4 + 32 * 4 + sizeof(P2Bars) + 64;
 }
 
 // cudaFuncSetAttribute once per (kernel, device).
@@ -869,12 +946,14 @@ cudaError_t launch_pass2(const LaunchCtx& c, const void* K, const void* V, const
       !map_rows2d(c.ws.kbar_rows, (long long)c.st.batch * c.st.H * kExtraRows, kExtraRows, &tmKB))
     return cudaErrorInvalidValue;
   static bool done[64] = {false};
-  const size_t smem = pass2_smem();
-  cudaError_t e = ensure_smem(k_pass2, smem, done);
+  cudaError_t e = ensure_smem(k_pass2, kSmemLimit, done);
   if (e != cudaSuccess) return e;
+  int vstages = kP2VStagesMax;
+  while (vstages > 2 && pass2_smem(c.st.NQ, vstages) > kSmemLimit) --vstages;
+  const size_t smem = pass2_smem(c.st.NQ, vstages);
   return launch_pdl(k_pass2, dim3(c.st.g2), dim3(kThreads), smem, c.stream, 1, tmK, tmV, tmQ, tmKB,
                     c.st, c.ws, s_div_out, c.scale_log2e, c.p.use_vnorm, c.p.pool_kernel >> 1,
-                    status);
+                    vstages, status);
 }
 
 }  // namespace mixkv

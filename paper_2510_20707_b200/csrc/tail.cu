@@ -30,21 +30,19 @@ __device__ void head_scalars(const SeqTable& st, const Workspace& ws, const int 
   float vmin = INFINITY, vmax = -INFINITY, vsum = 0.f;
   {
     const int per_head = (st.tile2_start[b + 1] - st.tile2_start[b]) / st.H;
-    const int U0 = st.tile2_start[b] + h * per_head;
-    int k = 0;
-    for (SegIter sg(U0, U0 + per_head, st.nt2, st.g2); sg.valid(); sg.next(), ++k) {
-      if ((k & 31) == lane) {
-        const float4 d4 = ws.dstat[sg.start];
-        dmin = fminf(dmin, d4.x);
-        dmax = fmaxf(dmax, d4.y);
-        dsum += d4.z;
-        exw += d4.w;
-        if (use_vnorm) {
-          const float4 v4 = ws.vstat[sg.start];
-          vmin = fminf(vmin, v4.x);
-          vmax = fmaxf(vmax, v4.y);
-          vsum += v4.z;
-        }
+    const SegList sl(st.tile2_start[b] + h * per_head, per_head, st.nt2, st.g2);
+    for (int e = lane; e < sl.nseg; e += 32) {   // lanes take segments side by side
+      const int start = sl.start(e);
+      const float4 d4 = ws.dstat[start];
+      dmin = fminf(dmin, d4.x);
+      dmax = fmaxf(dmax, d4.y);
+      dsum += d4.z;
+      exw += d4.w;
+      if (use_vnorm) {
+        const float4 v4 = ws.vstat[start];
+        vmin = fminf(vmin, v4.x);
+        vmax = fmaxf(vmax, v4.y);
+        vsum += v4.z;
       }
     }
   }
@@ -329,6 +327,10 @@ __device__ __forceinline__ int fixed_offset(const SeqTable& st, int bh, int Bp) 
   return off;
 }
 
+// Shared-memory slot of local position j: one pad word per 32 keeps both the strided walk
+// (thread t, t + 512, ...) and the contiguous runs of the compaction free of bank conflicts.
+__device__ __forceinline__ int kslot(int j) { return j + (j >> 5); }
+
 template <bool FUSED>
 __global__ void __launch_bounds__(kTailThreads, 1)
 k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
@@ -347,20 +349,18 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
   const int W = st.W;
   const int P = st.cu[b + 1] - st.cu[b] - W;
   const size_t poff = (size_t)h * st.Ptot + (st.cu[b] - b * W);
-  // slice of this CTA: positions [c0, c0 + n); thread t owns the run [c0 + t*R, c0 + (t+1)*R)
+  // slice of this CTA: positions [c0, c0 + n)
   const int chunk = (P + kTailCluster - 1) / kTailCluster;
-  const int R = (chunk + kTailThreads - 1) / kTailThreads;
+  const int R = (chunk + kTailThreads - 1) / kTailThreads;   // positions per thread
   const int c0 = min(crank * chunk, P);
   const int n = min(chunk, P - c0);
-  const int r0 = tid * R, r1 = min(r0 + R, n);   // local run of this thread (may be empty)
-  unsigned* skeys = reinterpret_cast<unsigned*>(tail_smem);            // [R * kTailThreads]
-  float* sraw = reinterpret_cast<float*>(tail_smem) + (size_t)R * kTailThreads;  // FUSED stage
+  unsigned* skeys = reinterpret_cast<unsigned*>(tail_smem);            // [kslot(chunk) + 1]
+  float* sraw = reinterpret_cast<float*>(skeys + kslot(chunk) + 1);    // FUSED: staged raw scores
 
   pdl_launch_dependents();
   pdl_wait();
 
   // ---- budget and output offsets of this (b, h)
-  int want;
   if (tid < 32) {
     int off = 0, cnt;
     if (a.counts_dev) {
@@ -386,8 +386,10 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
     }
   }
   const float* src = a.scores;
+  const bool cached = FUSED || a.cached;
+  float held[8];   // FUSED, R <= 8: mixed scores kept until the selection is done
   if (FUSED) {
-    // ---- pooling and mix of this slice (Eq. 2, Eq. 5); the mixed scores go to s_comp_out
+    // ---- pooling and mix of this slice (Eq. 2, Eq. 5), thread t takes positions t, t + 512, ...
     const int half = a.mp.pool_k >> 1;
     const float pad = a.mp.pool_mode == MIXKV_POOL_AVG ? 0.f : -INFINITY;
     if (warp == 1)
@@ -397,26 +399,47 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
       const int i = c0 - half + t;
       sraw[t] = (i >= 0 && i < P) ? ws.s_ex_raw[poff + i] : pad;
     }
+    float vn[8], dv[8];
+    if (R <= 8) {   // issue every load of the slice before the first use
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const int j = e * kTailThreads + tid;
+        vn[e] = (a.mp.use_vnorm && j < n) ? ws.vnorm[poff + c0 + j] : 0.f;
+        dv[e] = j < n ? a.s_div[poff + c0 + j] : 0.f;
+      }
+    }
     __syncthreads();
     const float invk = 1.0f / (float)a.mp.pool_k;
-    for (int j = r0; j < r1; ++j) {
-      const int i = c0 + j;
-      const float ex = pool_window(sraw + j, a.mp.pool_k, a.mp.pool_mode, invk);
-      const float vn = a.mp.use_vnorm ? ws.vnorm[poff + i] : 0.f;
-      const float c = mix_one(ex, vn, a.s_div[poff + i], sc, a.mp.use_vnorm, a.mp.mix_mode);
-      a.s_comp_out[poff + i] = c;
-      skeys[(j - r0) * kTailThreads + tid] = order_key(c);
+    if (R <= 8) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const int j = e * kTailThreads + tid;
+        held[e] = 0.f;
+        if (j < n) {
+          const float ex = pool_window(sraw + j, a.mp.pool_k, a.mp.pool_mode, invk);
+          held[e] = mix_one(ex, vn[e], dv[e], sc, a.mp.use_vnorm, a.mp.mix_mode);
+          skeys[kslot(j)] = order_key(held[e]);
+        }
+      }
+    } else {
+      for (int j = tid; j < n; j += kTailThreads) {
+        const float ex = pool_window(sraw + j, a.mp.pool_k, a.mp.pool_mode, invk);
+        const float v = a.mp.use_vnorm ? ws.vnorm[poff + c0 + j] : 0.f;
+        const float c = mix_one(ex, v, a.s_div[poff + c0 + j], sc, a.mp.use_vnorm, a.mp.mix_mode);
+        a.s_comp_out[poff + c0 + j] = c;
+        skeys[kslot(j)] = order_key(c);
+      }
     }
     src = a.s_comp_out;
   } else if (a.cached) {
-    for (int j = r0; j < r1; ++j) skeys[(j - r0) * kTailThreads + tid] = order_key(src[poff + c0 + j]);
+    for (int j = tid; j < n; j += kTailThreads) skeys[kslot(j)] = order_key(src[poff + c0 + j]);
   }
+  for (int t = tid; t < 256; t += kTailThreads) hist[0][t] = 0;
   __syncthreads();
-  want = s_sel[1];
+  const int want = s_sel[1];
   int* out = a.idx + s_off;
-  const bool cached = FUSED || a.cached;
   auto key_at = [&](int j) -> unsigned {
-    return cached ? skeys[(j - r0) * kTailThreads + tid] : order_key(src[poff + c0 + j]);
+    return cached ? skeys[kslot(j)] : order_key(src[poff + c0 + j]);
   };
 
   bool all = false;
@@ -428,14 +451,12 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
     // ---- threshold: the want-th largest key of the head, four 8-bit digit passes
     unsigned prefix = 0, mask = 0;
     int remaining = want;
-    for (int t = tid; t < 256; t += kTailThreads) hist[0][t] = 0;
-    __syncthreads();
     for (int pass = 0; pass < 4; ++pass) {
       const int shift = 24 - 8 * pass, buf = pass & 1;
       for (int e = 0; e < R; ++e) {   // same trip count in every lane: full-warp votes
-        const int j = r0 + e;
+        const int j = e * kTailThreads + tid;
         unsigned digit = 0xffffffffu;
-        if (j < r1) {
+        if (j < n) {
           const unsigned key = key_at(j);
           if ((key & mask) == prefix) digit = (key >> shift) & 255u;
         }
@@ -445,16 +466,14 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
       }
       cluster.sync();
       // every CTA adds up the cluster's histograms and finds the digit itself
-      int tot = 0;
+      int tot = 0, incl = 0;
       if (tid < 256) {
 #pragma unroll
         for (int r = 0; r < kTailCluster; ++r)
           tot += *cluster.map_shared_rank(&hist[buf][tid], r);
         hist[buf ^ 1][tid] = 0;   // every CTA is past its reads of the other buffer
-      }
-      // suffix sums over the 256 bins: bins above this one
-      int incl = tot;
-      if (tid < 256) {
+        // suffix sums over the 256 bins: bins above this one
+        incl = tot;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
           const int v = __shfl_down_sync(0xffffffffu, incl, o);
@@ -475,17 +494,18 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
       prefix |= (unsigned)s_sel[0] << shift;
       remaining = s_sel[1];
       mask |= 255u << shift;
-      __syncthreads();
     }
     tau = prefix;
     need_eq = remaining;
   }
 
-  // ---- ordered compaction: positions with key > tau, plus the first need_eq with key == tau
+  // ---- ordered compaction: thread t owns the run [t*R, (t+1)*R) of the slice; it keeps the
+  // positions with key > tau, plus the first need_eq (in position order) with key == tau
   if (want > 0) {
+    const int r0 = min(tid * R, n), r1 = min(r0 + R, n);
     int gt = 0, eq = 0;
     if (all) {
-      gt = max(r1 - r0, 0);
+      gt = r1 - r0;
     } else {
       for (int j = r0; j < r1; ++j) {
         const unsigned key = key_at(j);
@@ -500,6 +520,7 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
       const int y = __shfl_up_sync(0xffffffffu, eq_inc, o);
       if (lane >= o) gt_inc += x, eq_inc += y;
     }
+    __syncthreads();   // the threshold search is done with s_scan
     if (lane == 31) s_scan[warp][0] = gt_inc, s_scan[warp][1] = eq_inc;
     __syncthreads();
     int gt_before = gt_inc - gt, eq_before = eq_inc - eq;
@@ -533,6 +554,13 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
   // the index list is complete (and visible to the cluster) after this barrier; it also keeps
   // every CTA's shared memory alive until its peers have read it
   cluster.sync();
+  if (FUSED && R <= 8) {
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const int j = e * kTailThreads + tid;
+      if (j < n) a.s_comp_out[poff + c0 + j] = held[e];
+    }
+  }
 
   // ---- gather: selected rows in ascending position order, then the W window rows
   if (a.K_out) {
@@ -626,8 +654,9 @@ cudaError_t launch_tail(const LaunchCtx& c, const TailArgs& t) {
   const bool fused = t.scores == nullptr;
   a.cached = chunk <= kTailCacheCap ? 1 : 0;
   if (fused && !a.cached) return cudaErrorInvalidValue;   // callers check tail_can_fuse() first
+  (void)R;
   size_t smem = 0;
-  if (a.cached) smem += (size_t)R * kTailThreads * 4;
+  if (a.cached) smem += ((size_t)chunk + (chunk >> 5) + 1) * 4;
   if (fused) smem += ((size_t)chunk + 64) * 4;
   static size_t set_fused[64] = {0}, set_plain[64] = {0};
   int dev = 0;

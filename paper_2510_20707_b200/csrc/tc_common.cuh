@@ -237,19 +237,48 @@ __host__ __device__ __forceinline__ int tile_owner(int t, int nt, int g) {
   return (int)((((long long)t + 1) * g - 1) / nt);
 }
 
-struct SegIter {
-  // enumerates the segments [start, end) (tile ids) of the range [T0, T1) of one (b, h)
-  // when nt tiles are split contiguously over g CTAs
-  int T0, T1, nt, g, c, start;
-  __device__ SegIter(int T0_, int T1_, int nt_, int g_) : T0(T0_), T1(T1_), nt(nt_), g(g_) {
-    c = (int)((((long long)T0 + 1) * g - 1) / nt);  // CTA that owns tile T0
-    start = T0;
+// Walks the tiles [lo, hi) of one CTA in (b, h, t) order without dividing per tile.
+struct TileIter {
+  int id, hi, b, h, t, per_head, H;
+  const int* tile_start;
+  __device__ TileIter(const int* tile_start_, int batch, int H_, int lo, int hi_)
+      : id(lo), hi(hi_), H(H_), tile_start(tile_start_) {
+    b = h = t = 0;
+    per_head = 1;
+    if (lo < hi_) {
+      const TileCoord c = tile_coord(tile_start_, batch, H_, lo);
+      b = c.b, h = c.h, t = c.t;
+      per_head = (tile_start_[b + 1] - tile_start_[b]) / H_;
+    }
   }
-  __device__ bool valid() const { return start < T1; }
-  __device__ void next() {
-    ++c;
-    start = c < g ? cta_first_tile(c, nt, g) : T1;
-    if (start > T1) start = T1;
+  __device__ __forceinline__ bool valid() const { return id < hi; }
+  __device__ __forceinline__ int bh() const { return b * H + h; }
+  // first / last tile of a segment: a run of tiles of one (b, h) inside this CTA's range
+  __device__ __forceinline__ bool seg_last() const { return id + 1 == hi || t + 1 == per_head; }
+  __device__ __forceinline__ void next() {
+    ++id;
+    if (++t == per_head) {
+      t = 0;
+      if (++h == H) {
+        h = 0;
+        ++b;
+        if (id < hi) per_head = (tile_start[b + 1] - tile_start[b]) / H;
+      }
+    }
+  }
+};
+
+// Segments of one (b, h) when its tiles [T0, T0 + per_head) lie in a list of nt tiles split
+// contiguously over g CTAs: segment e starts at T0 for e = 0 and at the first tile of CTA
+// c0 + e otherwise (c0 = CTA that owns T0).
+struct SegList {
+  int T0, c0, nseg, nt, g;
+  __device__ SegList(int T0_, int per_head, int nt_, int g_) : T0(T0_), nt(nt_), g(g_) {
+    c0 = tile_owner(T0_, nt_, g_);
+    nseg = tile_owner(T0_ + per_head - 1, nt_, g_) - c0 + 1;
+  }
+  __device__ __forceinline__ int start(int e) const {
+    return e == 0 ? T0 : cta_first_tile(c0 + e, nt, g);
   }
 };
 
