@@ -318,6 +318,10 @@ def run_mixkv(args):
     torch.cuda.synchronize()
     tr_c = [[(C.c_void_p * (n_stage + 1))(*[e.cuda_event for e in ly]) for ly in st_]
             for st_ in tr_ev]
+    # the GPU is kept busy while the host enqueues the traced steps, so that the events are
+    # reached back to back on the device and their differences are device times, not host
+    # enqueue times
+    torch.cuda._sleep(int(6e-3 * 1.9e9 * n_tr * wl.layers / 28))
     for s in range(n_tr):
         step(s, trace=tr_c[s])
     torch.cuda.synchronize()

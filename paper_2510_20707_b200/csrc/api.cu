@@ -64,6 +64,8 @@ int build_table(const mixkv_params* p, const int32_t* cu, int batch, int L, SeqT
   const int sms = device_sm_count();
   st->g1 = st->nt1 < sms ? st->nt1 : sms;
   st->g2 = st->nt2 < sms ? st->nt2 : sms;
+  st->q1 = st->nt1 / st->g1, st->r1 = st->nt1 % st->g1;
+  st->q2 = st->nt2 / st->g2, st->r2 = st->nt2 % st->g2;
   *max_len = mx;
   return MIXKV_OK;
 }
@@ -99,8 +101,6 @@ void carve(const mixkv_params* p, const SeqTable& st, unsigned char* base, Works
   ws->vstat = (float4*)take((size_t)st.nt2 * 16);
   ws->dstat = (float4*)take((size_t)st.nt2 * 16);
   ws->exsum = (float*)take(H * st.pchunks_total * 4);
-  ws->bq = (float*)take(BH * st.NQ * 4);
-  ws->kbar_rows = (__nv_bfloat16*)take(BH * kExtraRows * kHeadDim * 2);
   ws->rbar = (float*)take(BH * 4);
   ws->counts = (int*)take(BH * 4);
   ws->idx_offsets = (int*)take((BH + 1) * 4);
@@ -132,15 +132,13 @@ int make_ctx(const mixkv_params* p, const int32_t* cu, int batch, int L, void* w
   return MIXKV_OK;
 }
 
-// pass 1, merge, pass 2 (and the pooled-score sums max pooling needs): everything the mix reads.
+// pass 1, pass 2 (and the pooled-score sums max pooling needs): everything the mix reads.
 int enqueue_passes(const LaunchCtx& c, const void* K, const void* V, const void* Q, float* s_div,
                    float* rbar_out, int* status) {
   c.mark();
   if (launch_pass1(c, K, Q, status) != cudaSuccess) return MIXKV_ERR_CUDA;
   c.mark();
-  if (launch_merge(c, rbar_out) != cudaSuccess) return MIXKV_ERR_CUDA;
-  c.mark();
-  if (launch_pass2(c, K, V, Q, s_div, status) != cudaSuccess) return MIXKV_ERR_CUDA;
+  if (launch_pass2(c, K, V, Q, s_div, rbar_out, status) != cudaSuccess) return MIXKV_ERR_CUDA;
   if (c.p.pool_mode == MIXKV_POOL_MAX) {
     c.mark();
     if (launch_poolsum(c) != cudaSuccess) return MIXKV_ERR_CUDA;
@@ -179,7 +177,6 @@ int enqueue_select(const LaunchCtx& c, const float* scores, int* counts, TailArg
 int layer_stages(const mixkv_params* p, bool fused_ok, const char** names) {
   int n = 0;
   names[n++] = "pass1";
-  names[n++] = "merge";
   names[n++] = "pass2";
   if (p->pool_mode == MIXKV_POOL_MAX) names[n++] = "poolsum";
   if (p->budget_mode == MIXKV_BUDGET_ADAPTIVE || !fused_ok) names[n++] = "mixpool";

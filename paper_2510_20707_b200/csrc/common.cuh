@@ -26,10 +26,16 @@ struct SeqTable {
   int cu[kMaxBatch + 1];             // sequence offsets into Ltot
   int pchunk_start[kMaxBatch + 1];   // prefix sum of candidate chunks
   // persistent 128-key tile schedules of the two tensor-core passes, (b, h, t) order
-  int nt1, g1;                       // pass 1: tiles over all L keys, CTAs
-  int nt2, g2;                       // pass 2: tiles over the P candidate keys, CTAs
+  int nt1, g1, q1, r1;               // pass 1: tiles over all L keys, CTAs, nt1 = q1 * g1 + r1
+  int nt2, g2, q2, r2;               // pass 2: tiles over the P candidate keys, likewise
   int tile1_start[kMaxBatch + 1];    // prefix sum of H * ceil(L_b / 128)
   int tile2_start[kMaxBatch + 1];    // prefix sum of H * ceil(P_b / 128)
+};
+
+// nt tiles split contiguously over g CTAs (g <= nt): the first r CTAs take q + 1 tiles, the
+// others q.
+struct Split {
+  int nt, g, q, r;
 };
 
 // Device workspace carve-up (all pointers into the caller's workspace).
@@ -46,8 +52,6 @@ struct Workspace {
   float4* vstat;      // [nt2]         (min, max, sum, -) of |V_i| over candidates
   float4* dstat;      // [nt2]         (min, max, sum) of s_div, window-count-weighted sum of s_ex_raw
   float* exsum;       // [H, pchunks_total]   per-chunk sum of pooled s_ex (max pooling only)
-  float* bq;          // [batch*H, NQ]  log2 normaliser of each window row (incl. 1/W)
-  __nv_bfloat16* kbar_rows;  // [batch*H, 16, d]  mean unit key as bf16 hi/lo/lo2 rows, 13 zero rows
   float* rbar;        // [batch*H]
   int* counts;        // [batch*H]
   int* idx_offsets;   // [batch*H + 1]
@@ -77,9 +81,8 @@ struct LaunchCtx {
 
 // ---- kernels (defined in the .cu files) ------------------------------------------
 cudaError_t launch_pass1(const LaunchCtx& c, const void* K, const void* Q, int* status);
-cudaError_t launch_merge(const LaunchCtx& c, float* rbar_out);
 cudaError_t launch_pass2(const LaunchCtx& c, const void* K, const void* V, const void* Q,
-                         float* s_div_out, int* status);
+                         float* s_div_out, float* rbar_out, int* status);
 int device_sm_count();
 cudaError_t launch_poolsum(const LaunchCtx& c);
 cudaError_t launch_mixpool(const LaunchCtx& c, const float* s_div, const float* rbar_in,

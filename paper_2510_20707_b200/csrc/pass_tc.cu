@@ -1,15 +1,15 @@
 // The two passes over K of the MixKV scoring step as persistent, warp-specialised sm_100a
 // kernels: TMA tile loads into 128-byte-swizzled shared memory, tcgen05.mma (bf16 x bf16 ->
 // fp32) with accumulators in tensor memory, and epilogues that read the accumulators back with
-// tcgen05.ld.  A small merge kernel sits between them.
+// tcgen05.ld.
 //
 //   pass 1  K from HBM.  Logits with the window queries on the M side (one query row per TMEM
 //           lane), so the running softmax (max, sum) of a row is thread-local; alongside, key
 //           norms and the sum of unit keys from the shared-memory tile.
-//   merge   per (sequence, head): the per-CTA partial softmax statistics become one log2
-//           normaliser per window row, the partial unit-key sums become the mean unit key
-//           (written as bf16 hi / lo / lo2 rows) and the redundancy of Eq. 4.
-//   pass 2  K again (served by L2), V from HBM.  Logits with the keys on the M side (one key
+//   pass 2  K again (served by L2), V from HBM.  At the start of a (sequence, head) segment the
+//           CTA folds pass 1's per-CTA partials: the softmax statistics become one log2
+//           normaliser per window row, the unit-key sums become the mean unit key (bf16 hi /
+//           lo / lo2 rows) and the redundancy of Eq. 4.  Logits with the keys on the M side (one key
 //           per TMEM lane), normalised with the finished row statistics, so the column sum over
 //           window rows and query heads is thread-local -> s_ex_raw.  The mean unit key rides
 //           along as three extra bf16 "query" rows -> K_i . kbar -> s_div.  Value norms are
@@ -146,8 +146,8 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int NQ = st.NQ, W = st.W, H = st.H;
-  const int lo = cta_first_tile(blockIdx.x, st.nt1, st.g1);
-  const int hi = cta_first_tile(blockIdx.x + 1, st.nt1, st.g1);
+  const int lo = cta_first_tile(blockIdx.x, split1(st));
+  const int hi = cta_first_tile(blockIdx.x + 1, split1(st));
   volatile int* abort = &bars->abort;
 
   pdl_launch_dependents();
@@ -388,93 +388,6 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
   if (tid == 0 && bars->abort && status) atomicExch(status, MIXKV_ERR_TIMEOUT);
 }
 
-// ========================================================================= merge
-// One CTA per (sequence, head): folds the per-segment partials of pass 1.  Warps take segments
-// side by side so that the loads of different segments are in flight together.
-__global__ void __launch_bounds__(256)
-k_merge(const SeqTable st, const Workspace ws, float* __restrict__ rbar_out) {
-  __shared__ float2 part[8][256];
-  __shared__ float kpart[2][kHeadDim];
-  __shared__ int sstart[256];
-  __shared__ float sred[4];
-  pdl_launch_dependents();
-  pdl_wait();
-  const int bh = blockIdx.x, b = bh / st.H, h = bh % st.H;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int NQ = st.NQ;
-  const int L = st.cu[b + 1] - st.cu[b];
-  const int per_head = (st.tile1_start[b + 1] - st.tile1_start[b]) / st.H;
-  const SegList sl(st.tile1_start[b] + h * per_head, per_head, st.nt1, st.g1);
-  const int nunits = NQ <= 128 ? 2 : 1;
-  float M[8], Z[8];
-#pragma unroll
-  for (int r = 0; r < 8; ++r) M[r] = -1e30f, Z[r] = 0.f;
-  float ks = 0.f;
-  const int kd = tid & (kHeadDim - 1), kpar = tid >> 7;
-  for (int e0 = 0; e0 < sl.nseg; e0 += 256) {
-    const int ne = min(256, sl.nseg - e0);
-    __syncthreads();
-    if (tid < ne) sstart[tid] = sl.start(e0 + tid);
-    __syncthreads();
-#pragma unroll 2
-    for (int e = warp; e < ne; e += 8) {
-      for (int u = 0; u < nunits; ++u) {
-        const float2* src = ws.rowstat + ((size_t)sstart[e] * 2 + u) * NQ;
-#pragma unroll
-        for (int r = 0; r < 8; ++r) {
-          const int q = lane + 32 * r;
-          if (q < NQ) {
-            const float2 mz = src[q];
-            const float mn = fmaxf(M[r], mz.x);
-            Z[r] = Z[r] * ex2(M[r] - mn) + mz.y * ex2(mz.x - mn);
-            M[r] = mn;
-          }
-        }
-      }
-    }
-#pragma unroll 4
-    for (int e = kpar; e < ne; e += 2) ks += ws.ksum[(size_t)sstart[e] * kHeadDim + kd];
-  }
-#pragma unroll
-  for (int r = 0; r < 8; ++r) part[warp][lane + 32 * r] = make_float2(M[r], Z[r]);
-  kpart[kpar][kd] = ks;
-  __syncthreads();
-  if (tid < NQ) {
-    float Mx = -1e30f;
-#pragma unroll
-    for (int w = 0; w < 8; ++w) Mx = fmaxf(Mx, part[w][tid].x);
-    float Zs = 0.f;
-#pragma unroll
-    for (int w = 0; w < 8; ++w) Zs += part[w][tid].y * exp2f(part[w][tid].x - Mx);
-    // log2 of (Z * W): the 1/W of the window mean is folded into the normaliser
-    ws.bq[(size_t)bh * NQ + tid] = Mx + (log2f(Zs) + log2f((float)st.W));
-  }
-  __nv_bfloat16* rows = ws.kbar_rows + (size_t)bh * kExtraRows * kHeadDim;
-  if (tid < kHeadDim) {
-    const float s = kpart[0][tid] + kpart[1][tid];
-    const float n2 = warp_sum(s * s);
-    if (lane == 0) sred[warp] = n2;
-    const float kb = s / (float)L;
-    const __nv_bfloat16 p0 = __float2bfloat16_rn(kb);
-    const float r1 = kb - __bfloat162float(p0);
-    const __nv_bfloat16 p1 = __float2bfloat16_rn(r1);
-    const __nv_bfloat16 p2 = __float2bfloat16_rn(r1 - __bfloat162float(p1));
-    rows[tid] = p0;
-    rows[kHeadDim + tid] = p1;
-    rows[2 * kHeadDim + tid] = p2;
-  }
-  for (int i = tid; i < (kExtraRows - 3) * kHeadDim / 2; i += 256)
-    reinterpret_cast<uint32_t*>(rows + 3 * kHeadDim)[i] = 0u;
-  __syncthreads();
-  if (tid == 0) {
-    const double nn = ((double)sred[0] + (double)sred[1]) + ((double)sred[2] + (double)sred[3]);
-    const double T = (double)L;
-    const float r = (float)((nn - T) / (T * (T - 1.0)));   // Eq. 4
-    ws.rbar[bh] = r;
-    if (rbar_out) rbar_out[bh] = r;
-  }
-}
-
 // ======================================================================== pass 2
 constexpr int kP2KStages = 3;              // K tiles (32 KB each)
 constexpr int kP2VStagesMax = 4;           // V half tiles: 64 rows, 16 KB each
@@ -490,6 +403,7 @@ struct P2Bars {
   uint64_t tempty[2];
   uint64_t qfull;
   uint64_t qfree;
+  uint64_t kbready;
   uint32_t tmem_base;
   int abort;
   int vote[2][2];
@@ -515,10 +429,9 @@ __device__ __forceinline__ void colsum_chunk(const uint32_t (&r)[16], const floa
 // grid = g2 persistent CTAs: K producer, MMA, V producer, 1 idle, 8 epilogue, 4 value-norm warps.
 __global__ void __launch_bounds__(kThreads, 1)
 k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
-        const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKB,
-        const SeqTable st, const Workspace ws, float* __restrict__ s_div_out,
-        const float scale_log2e, const int use_vnorm, const int pool_half, const int vstages,
-        int* status) {
+        const __grid_constant__ CUtensorMap tmQ, const SeqTable st, const Workspace ws,
+        float* __restrict__ s_div_out, float* __restrict__ rbar_out, const float scale_log2e,
+        const int use_vnorm, const int pool_half, const int vstages, int* status) {
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* base =
       reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
@@ -530,11 +443,12 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
   float* sbq = reinterpret_cast<float*>(sV + vstages * kVSubBytes);  // [256] negated normalisers
   float* sx = sbq + 256;                      // [2][128] partial sums WG0 -> WG1
   float* sred = sx + 256;                     // [32]
-  P2Bars* bars = reinterpret_cast<P2Bars*>(sred + 32);
+  float2* part = reinterpret_cast<float2*>(sred + 32);   // [8][256] per-warp row statistics
+  P2Bars* bars = reinterpret_cast<P2Bars*>(part + 8 * 256);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int lo = cta_first_tile(blockIdx.x, st.nt2, st.g2);
-  const int hi = cta_first_tile(blockIdx.x + 1, st.nt2, st.g2);
+  const int lo = cta_first_tile(blockIdx.x, split2(st));
+  const int hi = cta_first_tile(blockIdx.x + 1, split2(st));
   volatile int* abort = &bars->abort;
   constexpr int kWarpTmaV = 2;
 
@@ -554,6 +468,7 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
     }
     mbar_init(&bars->qfull, 1);
     mbar_init(&bars->qfree, 1);
+    mbar_init(&bars->kbready, 4);          // the four warps that write the mean-key rows
     bars->abort = 0;
     mbar_init_fence();
   }
@@ -561,7 +476,6 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
   if (warp == kWarpTma && lane == 0) {
     tma_prefetch_desc(&tmK);
     tma_prefetch_desc(&tmQ);
-    tma_prefetch_desc(&tmKB);
   }
   if (warp == kWarpTmaV && lane == 0) tma_prefetch_desc(&tmV);
   tc_fence_before();
@@ -578,11 +492,9 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
       for (TileIter ti(st.tile2_start, st.batch, H, lo, hi); ti.valid(); ti.next()) {
         if (seg_start) {
           if (segn > 0 && !mbar_wait(&bars->qfree, (segn - 1) & 1, abort)) break;
-          mbar_expect_tx(&bars->qfull, NB * 256);
+          mbar_expect_tx(&bars->qfull, NQ * 256);
           tma_load_2d(sQ, &tmQ, 0, ti.bh() * NQ, &bars->qfull);
           tma_load_2d(sQ + NB * 128, &tmQ, 64, ti.bh() * NQ, &bars->qfull);
-          tma_load_2d(sQ + NQ * 128, &tmKB, 0, ti.bh() * kExtraRows, &bars->qfull);
-          tma_load_2d(sQ + NB * 128 + NQ * 128, &tmKB, 64, ti.bh() * kExtraRows, &bars->qfull);
           ++segn;
         }
         seg_start = ti.seg_last();
@@ -633,6 +545,7 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
       for (TileIter ti(st.tile2_start, st.batch, H, lo, hi); ti.valid(); ti.next()) {
         if (seg_start) {
           if (!mbar_wait(&bars->qfull, segn & 1, abort)) break;
+          if (!mbar_wait(&bars->kbready, segn & 1, abort)) break;
           ++segn;
         }
         seg_start = ti.seg_last();
@@ -670,8 +583,47 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
     for (TileIter ti(st.tile2_start, st.batch, H, lo, hi); ti.valid(); ti.next()) {
       const int L = st.cu[ti.b + 1] - st.cu[ti.b], P = L - W;
       if (seg_start) {
-        named_bar_sync(1, kEpiThreads);   // the previous segment's readers of sbq are done
-        if (et < NQ) sbq[et] = -ws.bq[(size_t)ti.bh() * NQ + et];
+        // fold pass 1's per-segment softmax statistics of this (b, h) into one log2 normaliser
+        // per window row (the 1/W of the window mean folded in); warps take segments side by side
+        named_bar_sync(1, kEpiThreads);   // the previous segment's readers of sbq / part are done
+        {
+          const int per_head = (st.tile1_start[ti.b + 1] - st.tile1_start[ti.b]) / H;
+          const SegList sl(st.tile1_start[ti.b] + ti.h * per_head, per_head, split1(st));
+          const int nunits = NQ <= 128 ? 2 : 1;
+          const int ew = warp - kEpiWarp0;
+          float M[8], Z[8];
+#pragma unroll
+          for (int r = 0; r < 8; ++r) M[r] = -1e30f, Z[r] = 0.f;
+#pragma unroll 2
+          for (int e = ew; e < sl.nseg; e += kEpiWarps) {
+            const int start = sl.start(e);
+            for (int u = 0; u < nunits; ++u) {
+              const float2* src = ws.rowstat + ((size_t)start * 2 + u) * NQ;
+#pragma unroll
+              for (int r = 0; r < 8; ++r) {
+                const int q = lane + 32 * r;
+                if (q < NQ) {
+                  const float2 mz = src[q];
+                  const float mn = fmaxf(M[r], mz.x);
+                  Z[r] = Z[r] * ex2(M[r] - mn) + mz.y * ex2(mz.x - mn);
+                  M[r] = mn;
+                }
+              }
+            }
+          }
+#pragma unroll
+          for (int r = 0; r < 8; ++r) part[ew * 256 + lane + 32 * r] = make_float2(M[r], Z[r]);
+          named_bar_sync(1, kEpiThreads);
+          if (et < NQ) {
+            float Mx = -1e30f;
+#pragma unroll
+            for (int w = 0; w < kEpiWarps; ++w) Mx = fmaxf(Mx, part[w * 256 + et].x);
+            float Zs = 0.f;
+#pragma unroll
+            for (int w = 0; w < kEpiWarps; ++w) Zs += part[w * 256 + et].y * exp2f(part[w * 256 + et].x - Mx);
+            sbq[et] = -(Mx + (log2f(Zs) + log2f((float)W)));
+          }
+        }
         dmin = INFINITY, dmax = -INFINITY, dsum = 0.f, exw = 0.f;
         seg_first = ti.id;
         named_bar_sync(1, kEpiThreads);
@@ -755,56 +707,111 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
       }
       ++it;
     }
-  } else if (warp >= kAuxWarp0 && use_vnorm) {
-    // ------------------------------------------------------------------ value norms
-    // Warps 12, 13 read the first 64 rows of a tile, warps 14, 15 the last 64; one row per
-    // thread from the swizzled half tile.
+  } else if (warp >= kAuxWarp0) {
+    // ------------------------------------------------------------------ mean key, value norms
+    // At the start of a segment: fold pass 1's unit-key sums of this (b, h) into the mean unit
+    // key, write its bf16 hi / lo / lo2 split into the three extra B rows and (once per head)
+    // publish the redundancy of Eq. 4.  Per tile: warps 12, 13 read the first 64 rows of the V
+    // tile, warps 14, 15 the last 64; one row per thread from the swizzled half tile.
     const int vt = tid - kAuxWarp0 * 32;         // 0..127
     const int sub = vt >> 6, vr = vt & 63;
     float vmin = INFINITY, vmax = -INFINITY, vsum = 0.f;
-    int it = 0, seg_first = lo;
+    int it = 0, segn = 0, seg_first = lo;
     bool seg_start = true;
     for (TileIter ti(st.tile2_start, st.batch, H, lo, hi); ti.valid(); ti.next()) {
       if (seg_start) {
+        const int L = st.cu[ti.b + 1] - st.cu[ti.b];
+        const int per_head = (st.tile1_start[ti.b + 1] - st.tile1_start[ti.b]) / H;
+        const SegList sl(st.tile1_start[ti.b] + ti.h * per_head, per_head, split1(st));
+        float s = 0.f;
+        for (int e0 = 0; e0 < sl.nseg; e0 += 16) {   // sixteen loads in flight per thread
+          float v[16];
+#pragma unroll
+          for (int e = 0; e < 16; ++e)
+            v[e] = e0 + e < sl.nseg ? ws.ksum[(size_t)sl.start(e0 + e) * kHeadDim + vt] : 0.f;
+#pragma unroll
+          for (int e = 0; e < 16; ++e) s += v[e];
+        }
+        const bool owner = ti.t == 0;   // the CTA that holds the head's first tile publishes rbar
+        if (owner) {
+          const float n2 = warp_sum(s * s);
+          if (lane == 0) sred[28 + (warp - kAuxWarp0)] = n2;
+        }
+        const float kb = s / (float)L;
+        __nv_bfloat16 parts[3];
+        parts[0] = __float2bfloat16_rn(kb);
+        const float r1 = kb - __bfloat162float(parts[0]);
+        parts[1] = __float2bfloat16_rn(r1);
+        parts[2] = __float2bfloat16_rn(r1 - __bfloat162float(parts[1]));
+        if (segn > 0) {   // the previous segment's MMAs must be done with the B rows
+          if (vt == 0) mbar_wait(&bars->qfree, (segn - 1) & 1, abort);
+          named_bar_sync(4, 128);
+        }
+        {
+          unsigned char* hb = sQ + (vt >> 6) * NB * 128 + (vt & 7) * 2;
+          const int chunk = (vt & 63) >> 3;
+#pragma unroll
+          for (int e = 0; e < kExtraRows; ++e) {
+            if (e < 3 || segn == 0)
+              *reinterpret_cast<__nv_bfloat16*>(hb + sw128_offset(NQ + e, chunk)) =
+                  e < 3 ? parts[e] : __float2bfloat16_rn(0.f);
+          }
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bars->kbready);
+        if (owner) {
+          named_bar_sync(4, 128);
+          if (vt == 0) {
+            const double nn = ((double)sred[28] + (double)sred[29]) + ((double)sred[30] + (double)sred[31]);
+            const double T = (double)L;
+            const float r = (float)((nn - T) / (T * (T - 1.0)));   // Eq. 4
+            ws.rbar[ti.bh()] = r;
+            if (rbar_out) rbar_out[ti.bh()] = r;
+          }
+        }
+        ++segn;
         vmin = INFINITY, vmax = -INFINITY, vsum = 0.f;
         seg_first = ti.id;
       }
       seg_start = ti.seg_last();
-      const int P = st.cu[ti.b + 1] - st.cu[ti.b] - W;
-      const int vit = 2 * it + sub;
-      const int vs = vit % vstages, vph = (vit / vstages) & 1;
-      const bool ok = mbar_wait(&bars->vfull[vs], vph, abort);
-      const unsigned char* tile = sV + vs * kVSubBytes;
-      float ss[4] = {0.f, 0.f, 0.f, 0.f};
-      if (ok) {
+      if (use_vnorm) {
+        const int P = st.cu[ti.b + 1] - st.cu[ti.b] - W;
+        const int vit = 2 * it + sub;
+        const int vs = vit % vstages, vph = (vit / vstages) & 1;
+        const bool ok = mbar_wait(&bars->vfull[vs], vph, abort);
+        const unsigned char* tile = sV + vs * kVSubBytes;
+        float ss[4] = {0.f, 0.f, 0.f, 0.f};
+        if (ok) {
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
+          for (int half = 0; half < 2; ++half) {
 #pragma unroll
-          for (int c = 0; c < 8; ++c) {
-            const uint4 u =
-                *reinterpret_cast<const uint4*>(tile + half * (kVSubBytes / 2) + sw128_offset(vr, c));
-            const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&u);
+            for (int c = 0; c < 8; ++c) {
+              const uint4 u =
+                  *reinterpret_cast<const uint4*>(tile + half * (kVSubBytes / 2) + sw128_offset(vr, c));
+              const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&u);
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const float2 f = __bfloat1622float2(p2[e]);
-              ss[e & 1] = fmaf(f.x, f.x, ss[e & 1]);
-              ss[2 + (e & 1)] = fmaf(f.y, f.y, ss[2 + (e & 1)]);
+              for (int e = 0; e < 4; ++e) {
+                const float2 f = __bfloat1622float2(p2[e]);
+                ss[e & 1] = fmaf(f.x, f.x, ss[e & 1]);
+                ss[2 + (e & 1)] = fmaf(f.y, f.y, ss[2 + (e & 1)]);
+              }
             }
           }
         }
-      }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&bars->vempty[vs]);
-      const int i = ti.t * kTile + sub * 64 + vr;
-      if (ok && i < P) {
-        const float n = sqrtf((ss[0] + ss[1]) + (ss[2] + ss[3]));
-        ws.vnorm[(size_t)ti.h * st.Ptot + (st.cu[ti.b] - ti.b * W) + i] = n;
-        vmin = fminf(vmin, n);
-        vmax = fmaxf(vmax, n);
-        vsum += n;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bars->vempty[vs]);
+        const int i = ti.t * kTile + sub * 64 + vr;
+        if (ok && i < P) {
+          const float n = sqrtf((ss[0] + ss[1]) + (ss[2] + ss[3]));
+          ws.vnorm[(size_t)ti.h * st.Ptot + (st.cu[ti.b] - ti.b * W) + i] = n;
+          vmin = fminf(vmin, n);
+          vmax = fmaxf(vmax, n);
+          vsum += n;
+        }
       }
       if (group_sync_stop(3, 128, vt == 0, abort, bars->vote[1], it)) break;
-      if (seg_start) {
+      if (seg_start && use_vnorm) {
         const float a = warp_min(vmin), b2 = warp_max(vmax), c2 = warp_sum(vsum);
         const int vw = warp - kAuxWarp0;
         if (lane == 0) {
@@ -880,7 +887,8 @@ size_t pass1_smem(int MB) {
 }
 size_t pass2_smem(int NQ, int vstages) {
   return 1024 + (size_t)2 * (NQ + kExtraRows) * 128 + kP2KStages * kTileBytes +
-         (size_t)vstages * kVSubBytes + 256 * 4 + 256 * 4 + 32 * 4 + sizeof(P2Bars) + 64;
+         (size_t)vstages * kVSubBytes + 256 * 4 + 256 * 4 + 32 * 4 + 8 * 256 * 8 + sizeof(P2Bars) +
+         64;
 }
 
 // cudaFuncSetAttribute once per (kernel, device).
@@ -932,18 +940,12 @@ cudaError_t launch_pass1(const LaunchCtx& c, const void* K, const void* Q, int* 
                     c.ws, c.scale_log2e, status);
 }
 
-cudaError_t launch_merge(const LaunchCtx& c, float* rbar_out) {
-  return launch_pdl(k_merge, dim3(c.st.batch * c.st.H), dim3(256), 0, c.stream, 1, c.st, c.ws,
-                    rbar_out);
-}
-
 cudaError_t launch_pass2(const LaunchCtx& c, const void* K, const void* V, const void* Q,
-                         float* s_div_out, int* status) {
-  CUtensorMap tmK, tmV, tmQ, tmKB;
+                         float* s_div_out, float* rbar_out, int* status) {
+  CUtensorMap tmK, tmV, tmQ;
   const void* Vsrc = c.p.use_vnorm ? V : K;   // the V map is never used without VNorm
   if (!map_rows3d(c, K, kTile, &tmK) || !map_rows3d(c, Vsrc, 64, &tmV) ||
-      !map_rows2d(Q, (long long)c.st.batch * c.st.H * c.st.NQ, c.st.NQ, &tmQ) ||
-      !map_rows2d(c.ws.kbar_rows, (long long)c.st.batch * c.st.H * kExtraRows, kExtraRows, &tmKB))
+      !map_rows2d(Q, (long long)c.st.batch * c.st.H * c.st.NQ, c.st.NQ, &tmQ))
     return cudaErrorInvalidValue;
   static bool done[64] = {false};
   cudaError_t e = ensure_smem(k_pass2, kSmemLimit, done);
@@ -951,8 +953,8 @@ cudaError_t launch_pass2(const LaunchCtx& c, const void* K, const void* V, const
   int vstages = kP2VStagesMax;
   while (vstages > 2 && pass2_smem(c.st.NQ, vstages) > kSmemLimit) --vstages;
   const size_t smem = pass2_smem(c.st.NQ, vstages);
-  return launch_pdl(k_pass2, dim3(c.st.g2), dim3(kThreads), smem, c.stream, 1, tmK, tmV, tmQ, tmKB,
-                    c.st, c.ws, s_div_out, c.scale_log2e, c.p.use_vnorm, c.p.pool_kernel >> 1,
+  return launch_pdl(k_pass2, dim3(c.st.g2), dim3(kThreads), smem, c.stream, 1, tmK, tmV, tmQ, c.st,
+                    c.ws, s_div_out, rbar_out, c.scale_log2e, c.p.use_vnorm, c.p.pool_kernel >> 1,
                     vstages, status);
 }
 

@@ -30,7 +30,7 @@ __device__ void head_scalars(const SeqTable& st, const Workspace& ws, const int 
   float vmin = INFINITY, vmax = -INFINITY, vsum = 0.f;
   {
     const int per_head = (st.tile2_start[b + 1] - st.tile2_start[b]) / st.H;
-    const SegList sl(st.tile2_start[b] + h * per_head, per_head, st.nt2, st.g2);
+    const SegList sl(st.tile2_start[b] + h * per_head, per_head, split2(st));
     for (int e = lane; e < sl.nseg; e += 32) {   // lanes take segments side by side
       const int start = sl.start(e);
       const float4 d4 = ws.dstat[start];

@@ -227,14 +227,20 @@ __device__ __forceinline__ TileCoord tile_coord(const int* tile_start, int batch
   c.bh = b * H + c.h;
   return c;
 }
-// First tile of CTA c when nt tiles are split over g CTAs (contiguous ranges).
-__host__ __device__ __forceinline__ int cta_first_tile(int c, int nt, int g) {
-  return (int)(((long long)c * nt) / g);
+__host__ __device__ __forceinline__ Split split1(const SeqTable& st) {
+  return Split{st.nt1, st.g1, st.q1, st.r1};
 }
-
+__host__ __device__ __forceinline__ Split split2(const SeqTable& st) {
+  return Split{st.nt2, st.g2, st.q2, st.r2};
+}
+// First tile of CTA c.
+__host__ __device__ __forceinline__ int cta_first_tile(int c, const Split& sp) {
+  return c * sp.q + (c < sp.r ? c : sp.r);
+}
 // CTA whose contiguous range contains tile t.
-__host__ __device__ __forceinline__ int tile_owner(int t, int nt, int g) {
-  return (int)((((long long)t + 1) * g - 1) / nt);
+__host__ __device__ __forceinline__ int tile_owner(int t, const Split& sp) {
+  const int big = sp.r * (sp.q + 1);
+  return t < big ? t / (sp.q + 1) : sp.r + (t - big) / sp.q;
 }
 
 // Walks the tiles [lo, hi) of one CTA in (b, h, t) order without dividing per tile.
@@ -268,17 +274,18 @@ struct TileIter {
   }
 };
 
-// Segments of one (b, h) when its tiles [T0, T0 + per_head) lie in a list of nt tiles split
-// contiguously over g CTAs: segment e starts at T0 for e = 0 and at the first tile of CTA
+// Segments of one (b, h) when its tiles [T0, T0 + per_head) lie in a tile list split
+// contiguously over CTAs: segment e starts at T0 for e = 0 and at the first tile of CTA
 // c0 + e otherwise (c0 = CTA that owns T0).
 struct SegList {
-  int T0, c0, nseg, nt, g;
-  __device__ SegList(int T0_, int per_head, int nt_, int g_) : T0(T0_), nt(nt_), g(g_) {
-    c0 = tile_owner(T0_, nt_, g_);
-    nseg = tile_owner(T0_ + per_head - 1, nt_, g_) - c0 + 1;
+  int T0, c0, nseg;
+  Split sp;
+  __device__ SegList(int T0_, int per_head, const Split& sp_) : T0(T0_), sp(sp_) {
+    c0 = tile_owner(T0_, sp_);
+    nseg = tile_owner(T0_ + per_head - 1, sp_) - c0 + 1;
   }
   __device__ __forceinline__ int start(int e) const {
-    return e == 0 ? T0 : cta_first_tile(c0 + e, nt, g);
+    return e == 0 ? T0 : cta_first_tile(c0 + e, sp);
   }
 };
 
