@@ -82,6 +82,10 @@ void mixkv_default_params(mixkv_params* p, int32_t kv_heads, int32_t gqa_ratio, 
 int mixkv_workspace_size(const mixkv_params* p, int32_t batch, int64_t total_tokens,
                          int32_t max_seq_len, size_t* bytes);
 
+/* The same for a call that handles n_layers layers at once (mixkv_compress_layers). */
+int mixkv_workspace_size_layers(const mixkv_params* p, int32_t n_layers, int32_t batch,
+                                int64_t total_tokens, int32_t max_seq_len, size_t* bytes);
+
 /* Scores of every candidate key (Sec. 3.2-3.3; Algorithm 1 step 1 and the mixing of step 2):
  *   s_ex   = pool_k( sum over the G query heads of the mean over the W window rows of the
  *            causal softmax attention weight on key i )             (extrinsic importance)
@@ -178,6 +182,35 @@ int mixkv_compress_layer_traced(const void* K, const void* V, const void* Qwin,
                                 int32_t* idx_offsets_opt, float* s_comp_opt,
                                 int32_t* status_dev, void* stream,
                                 void* const* events_host, int32_t n_events);
+
+/* mixkv_compress_layer for n_layers layers of identical shape in ONE set of kernel launches
+ * (Algorithm 1's "for each layer l and head h" loop taken whole): a serving engine that keeps the
+ * prefill KV of all layers resident can compress them together at the end of prefill, which
+ * spreads the per-launch costs over all layers and keeps every SM busy in the selection and
+ * gather step.  The layers are an outer batch dimension; each is processed exactly as
+ * mixkv_compress_layer would.
+ *   K, V              [n_layers, H, Ltot, d] bf16; kv_layer_stride = elements between the
+ *                     tensors of consecutive layers (0: packed, H * Ltot * d; otherwise a
+ *                     multiple of 8 and at least that)
+ *   Qwin              [n_layers, batch, H*G, W, d] bf16; q_layer_stride likewise (0: packed)
+ *   rbar_in_opt       optional, [n_layers, batch, H]
+ *   K_out, V_out      [n_layers, batch * H * B, d]: layer l starts at row l * batch * H * B and
+ *                     is packed inside its slice as mixkv_compress_layer packs it
+ *   out_row_offsets   [n_layers, batch * H + 1], rows relative to the layer's slice
+ *   idx_opt           [n_layers, cap], cap = sum over sequences of H * min(B - W, P_b)
+ *   counts_opt        [n_layers, batch * H];  idx_offsets_opt [n_layers, batch * H + 1]
+ *   s_comp_opt        [n_layers, H, Ptot]
+ *   workspace         mixkv_workspace_size_layers bytes
+ *   events_host       optional measurement hook as in mixkv_compress_layer_traced (NULL, 0: off)
+ * n_layers <= 1024. */
+int mixkv_compress_layers(const void* K, const void* V, const void* Qwin, int32_t n_layers,
+                          int64_t kv_layer_stride, int64_t q_layer_stride,
+                          const int32_t* cu_seqlens_host, int32_t batch, int32_t L,
+                          const mixkv_params* p, void* workspace, size_t workspace_bytes,
+                          const float* rbar_in_opt, void* K_out, void* V_out,
+                          int32_t* out_row_offsets, int32_t* idx_opt, int32_t* counts_opt,
+                          int32_t* idx_offsets_opt, float* s_comp_opt, int32_t* status_dev,
+                          void* stream, void* const* events_host, int32_t n_events);
 
 /* Number of kernels one mixkv_compress_layer call enqueues for these parameters, and the
  * name of the i-th of them (NULL when i is out of range). */

@@ -5,8 +5,8 @@ The product is ``libmixkv.so`` (hand-written sm_100a CUDA behind a C ABI declare
 that marshals torch tensors into pointers.  There is no CPU fallback: the binding raises
 if the library has not been built.
 """
-from .binding import (MixKVError, Params, compress_layer, launches_per_layer, load_library,
-                      scores, select, workspace_size)
+from .binding import (MixKVError, Params, compress_layer, compress_layers, launches_per_layer,
+                      load_library, scores, select, workspace_size, workspace_size_layers)
 
-__all__ = ["MixKVError", "Params", "compress_layer", "launches_per_layer", "load_library",
-           "scores", "select", "workspace_size"]
+__all__ = ["MixKVError", "Params", "compress_layer", "compress_layers", "launches_per_layer",
+           "load_library", "scores", "select", "workspace_size", "workspace_size_layers"]

@@ -19,7 +19,8 @@ LIB_PATH = os.path.join(_PKG, "libmixkv.so")
 
 EXPORTS = ("mixkv_default_params", "mixkv_workspace_size", "mixkv_scores", "mixkv_select",
            "mixkv_compress_layer", "mixkv_compress_layer_traced", "mixkv_launches_per_layer",
-           "mixkv_stage_name", "mixkv_status_string", "mixkv_scores_static")
+           "mixkv_stage_name", "mixkv_status_string", "mixkv_scores_static",
+           "mixkv_workspace_size_layers", "mixkv_compress_layers")
 
 
 class MixKVError(RuntimeError):
@@ -79,6 +80,8 @@ def load_library() -> C.CDLL:
         lib.mixkv_default_params.argtypes = [C.POINTER(_CParams), i32, i32, i32]
         lib.mixkv_workspace_size.argtypes = [C.POINTER(_CParams), i32, C.c_int64, i32,
                                              C.POINTER(sz)]
+        lib.mixkv_workspace_size_layers.argtypes = [C.POINTER(_CParams), i32, i32, C.c_int64, i32,
+                                                    C.POINTER(sz)]
         lib.mixkv_launches_per_layer.argtypes = [C.POINTER(_CParams)]
         lib.mixkv_scores.argtypes = [vp, vp, vp, C.POINTER(i32), i32, i32, C.POINTER(_CParams),
                                      vp, sz, vp, vp, vp, vp, vp, vp, vp]
@@ -91,6 +94,10 @@ def load_library() -> C.CDLL:
                                              vp, vp, vp, vp]
         lib.mixkv_compress_layer_traced.argtypes = lib.mixkv_compress_layer.argtypes + [
             C.POINTER(vp), i32]
+        lib.mixkv_compress_layers.argtypes = [vp, vp, vp, i32, C.c_int64, C.c_int64,
+                                              C.POINTER(i32), i32, i32, C.POINTER(_CParams), vp,
+                                              sz, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp,
+                                              C.POINTER(vp), i32]
         lib.mixkv_stage_name.restype = C.c_char_p
         lib.mixkv_stage_name.argtypes = [C.POINTER(_CParams), i32]
         _lib = lib
@@ -128,6 +135,17 @@ def workspace_size(params: Params, batch: int, total_tokens: int, max_seq_len: i
                                              C.byref(out))
     if rc != 0:
         raise MixKVError(rc, "mixkv_workspace_size")
+    return int(out.value)
+
+
+def workspace_size_layers(params: Params, n_layers: int, batch: int, total_tokens: int,
+                          max_seq_len: int) -> int:
+    out = C.c_size_t(0)
+    pc = params.c()
+    rc = load_library().mixkv_workspace_size_layers(C.byref(pc), n_layers, batch, total_tokens,
+                                                    max_seq_len, C.byref(out))
+    if rc != 0:
+        raise MixKVError(rc, "mixkv_workspace_size_layers")
     return int(out.value)
 
 
@@ -268,4 +286,54 @@ def compress_layer(K: torch.Tensor, V: torch.Tensor, Q: torch.Tensor, params: Pa
         rc = load_library().mixkv_compress_layer_traced(*args, trace_events, len(trace_events))
     if rc != 0:
         raise MixKVError(rc, "mixkv_compress_layer")
+    return out
+
+
+def compress_layers(K: torch.Tensor, V: torch.Tensor, Q: torch.Tensor, params: Params,
+                    cu_seqlens: Optional[Sequence[int]] = None,
+                    rbar_in: Optional[torch.Tensor] = None,
+                    workspace: Optional[torch.Tensor] = None, stream=None,
+                    out: Optional[Dict[str, torch.Tensor]] = None,
+                    want_aux: bool = True, trace_events=None) -> Dict[str, torch.Tensor]:
+    """mixkv_compress_layers: K, V [n_layers, H, Ltot, 128], Q [n_layers, batch, H*G, W, 128]
+    (bf16 device tensors; the layer dimension may be strided, the rest contiguous).  Returns
+    K_out / V_out [n_layers, batch*H*B, 128], out_row_offsets [n_layers, batch*H+1] and, if
+    want_aux, idx [n_layers, cap] / counts / idx_offsets / s_comp."""
+    NL, H, Ltot, d = K.shape
+    batch = 1 if cu_seqlens is None else len(cu_seqlens) - 1
+    max_len = Ltot if cu_seqlens is None else max(int(cu_seqlens[b + 1]) - int(cu_seqlens[b])
+                                                 for b in range(batch))
+    if workspace is None:
+        workspace = torch.empty(workspace_size_layers(params, NL, batch, Ltot, max_len),
+                                dtype=torch.uint8, device=K.device)
+    for t in (K, V, Q):
+        assert t[0].is_contiguous(), "each layer must be contiguous"
+    assert V.stride(0) == K.stride(0), "K and V must share their layer stride"
+    Ptot = Ltot - batch * params.window
+    lens = [Ltot] if cu_seqlens is None else [int(cu_seqlens[b + 1]) - int(cu_seqlens[b])
+                                              for b in range(batch)]
+    cap = max(sum(H * min(params.budget - params.window, L - params.window) for L in lens), 1)
+    if out is None:
+        i32 = dict(dtype=torch.int32, device=K.device)
+        rows = batch * H * params.budget
+        out = {"K_out": torch.empty((NL, rows, d), dtype=torch.bfloat16, device=K.device),
+               "V_out": torch.empty((NL, rows, d), dtype=torch.bfloat16, device=K.device),
+               "out_row_offsets": torch.empty((NL, batch * H + 1), **i32),
+               "status": torch.zeros(1, **i32)}
+        if want_aux:
+            out["idx"] = torch.empty((NL, cap), **i32)
+            out["counts"] = torch.empty((NL, batch * H), **i32)
+            out["idx_offsets"] = torch.empty((NL, batch * H + 1), **i32)
+            out["s_comp"] = torch.empty((NL, H, Ptot), dtype=torch.float32, device=K.device)
+    cu, _ = _cu_array(cu_seqlens)
+    pc = params.c()
+    ev, n_ev = (None, 0) if trace_events is None else (trace_events, len(trace_events))
+    rc = load_library().mixkv_compress_layers(
+        K.data_ptr(), V.data_ptr(), Q.data_ptr(), NL, K.stride(0), Q.stride(0), cu, batch, Ltot,
+        C.byref(pc), _ptr(workspace), workspace.numel(), _ptr(rbar_in), _ptr(out["K_out"]),
+        _ptr(out["V_out"]), _ptr(out["out_row_offsets"]), _ptr(out.get("idx")),
+        _ptr(out.get("counts")), _ptr(out.get("idx_offsets")), _ptr(out.get("s_comp")),
+        _ptr(out["status"]), _stream(stream), ev, n_ev)
+    if rc != 0:
+        raise MixKVError(rc, "mixkv_compress_layers")
     return out

@@ -32,12 +32,13 @@ int check_params(const mixkv_params* p) {
 }
 
 // Builds the sequence table from the host offsets (or a single length).
-int build_table(const mixkv_params* p, const int32_t* cu, int batch, int L, SeqTable* st,
-                int* max_len) {
-  if (batch < 1) return MIXKV_ERR_INVALID_ARG;
-  if (batch > kMaxBatch) return MIXKV_ERR_UNSUPPORTED;
+int build_table(const mixkv_params* p, const int32_t* cu, int batch, int L, int layers,
+                SeqTable* st, int* max_len) {
+  if (batch < 1 || layers < 1) return MIXKV_ERR_INVALID_ARG;
+  if (batch > kMaxBatch || layers > kMaxLayers) return MIXKV_ERR_UNSUPPORTED;
   if (!cu && batch != 1) return MIXKV_ERR_INVALID_ARG;
   memset(st, 0, sizeof(*st));
+  st->layers = layers;
   st->batch = batch;
   st->H = p->kv_heads;
   st->G = p->gqa_ratio;
@@ -61,11 +62,13 @@ int build_table(const mixkv_params* p, const int32_t* cu, int batch, int L, SeqT
   st->pchunks_total = st->pchunk_start[batch];
   st->nt1 = st->tile1_start[batch];
   st->nt2 = st->tile2_start[batch];
+  const long long t1 = (long long)layers * st->nt1, t2 = (long long)layers * st->nt2;
+  if (t1 > 0x3fffffffLL) return MIXKV_ERR_UNSUPPORTED;
   const int sms = device_sm_count();
-  st->g1 = st->nt1 < sms ? st->nt1 : sms;
-  st->g2 = st->nt2 < sms ? st->nt2 : sms;
-  st->q1 = st->nt1 / st->g1, st->r1 = st->nt1 % st->g1;
-  st->q2 = st->nt2 / st->g2, st->r2 = st->nt2 % st->g2;
+  st->g1 = t1 < sms ? (int)t1 : sms;
+  st->g2 = t2 < sms ? (int)t2 : sms;
+  st->q1 = (int)(t1 / st->g1), st->r1 = (int)(t1 % st->g1);
+  st->q2 = (int)(t2 / st->g2), st->r2 = (int)(t2 % st->g2);
   *max_len = mx;
   return MIXKV_OK;
 }
@@ -90,33 +93,44 @@ void carve(const mixkv_params* p, const SeqTable& st, unsigned char* base, Works
     off = align_up(off + bytes, 256);
     return ptr;
   };
-  const size_t H = st.H, BH = (size_t)st.batch * st.H;
-  ws->kinv = (float*)take(H * st.Ltot * 4);
-  ws->vnorm = (float*)take(H * st.Ptot * 4);
-  ws->s_ex_raw = (float*)take(H * st.Ptot * 4);
-  ws->s_div = (float*)take(H * st.Ptot * 4);
-  ws->s_comp = (float*)take(H * st.Ptot * 4);
-  ws->rowstat = (float2*)take((size_t)st.nt1 * 2 * st.NQ * 8);
-  ws->ksum = (float*)take((size_t)st.nt1 * kHeadDim * 4);
-  ws->vstat = (float4*)take((size_t)st.nt2 * 16);
-  ws->dstat = (float4*)take((size_t)st.nt2 * 16);
-  ws->exsum = (float*)take(H * st.pchunks_total * 4);
-  ws->rbar = (float*)take(BH * 4);
-  ws->counts = (int*)take(BH * 4);
-  ws->idx_offsets = (int*)take((BH + 1) * 4);
-  ws->idx = (int*)take((size_t)idx_capacity(p, st) * 4);
+  const size_t NL = st.layers, H = st.H, BH = (size_t)st.batch * st.H;
+  ws->kinv = (float*)take(NL * H * st.Ltot * 4);
+  ws->vnorm = (float*)take(NL * H * st.Ptot * 4);
+  ws->s_ex_raw = (float*)take(NL * H * st.Ptot * 4);
+  ws->s_div = (float*)take(NL * H * st.Ptot * 4);
+  ws->s_comp = (float*)take(NL * H * st.Ptot * 4);
+  ws->rowstat = (float2*)take(NL * st.nt1 * 2 * st.NQ * 8);
+  ws->ksum = (float*)take(NL * st.nt1 * kHeadDim * 4);
+  ws->vstat = (float4*)take(NL * st.nt2 * 16);
+  ws->dstat = (float4*)take(NL * st.nt2 * 16);
+  ws->exsum = (float*)take(NL * H * st.pchunks_total * 4);
+  ws->rbar = (float*)take(NL * BH * 4);
+  ws->counts = (int*)take(NL * BH * 4);
+  ws->idx_offsets = (int*)take(NL * (BH + 1) * 4);
+  ws->idx = (int*)take(NL * (size_t)idx_capacity(p, st) * 4);
   ws->bytes = off;
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 int make_ctx(const mixkv_params* p, const int32_t* cu, int batch, int L, void* workspace,
-             size_t workspace_bytes, void* stream, LaunchCtx* c) {
+             size_t workspace_bytes, void* stream, LaunchCtx* c, int layers = 1,
+             long long kv_layer_stride = 0, long long q_layer_stride = 0) {
   int rc = check_params(p);
   if (rc != MIXKV_OK) return rc;
   int max_len = 0;
-  rc = build_table(p, cu, batch, L, &c->st, &max_len);
+  rc = build_table(p, cu, batch, L, layers, &c->st, &max_len);
   if (rc != MIXKV_OK) return rc;
+  // layer strides in elements; 0 = the layers are packed back to back
+  const long long kv_dense = (long long)c->st.H * c->st.Ltot * kHeadDim;
+  const long long q_dense = (long long)batch * c->st.H * c->st.NQ * kHeadDim;
+  c->kv_layer_stride = kv_layer_stride ? kv_layer_stride : kv_dense;
+  c->q_layer_stride = q_layer_stride ? q_layer_stride : q_dense;
+  if (layers > 1 && (c->kv_layer_stride < kv_dense || c->q_layer_stride < q_dense ||
+                     (c->kv_layer_stride & 7) || (c->q_layer_stride & 7)))
+    return MIXKV_ERR_INVALID_ARG;   // layers must not overlap; TMA wants 16-byte strides
+  c->idx_cap = (int)idx_capacity(p, c->st);
+  c->out_rows_cap = batch * c->st.H * p->budget;
   if (!workspace || !aligned16(workspace)) return MIXKV_ERR_INVALID_ARG;
   carve(p, c->st, (unsigned char*)workspace, &c->ws);
   if (c->ws.bytes > workspace_bytes) return MIXKV_ERR_WORKSPACE_TOO_SMALL;
@@ -212,14 +226,21 @@ void mixkv_default_params(mixkv_params* p, int32_t kv_heads, int32_t gqa_ratio, 
 
 int mixkv_workspace_size(const mixkv_params* p, int32_t batch, int64_t total_tokens,
                          int32_t max_seq_len, size_t* bytes) {
+  return mixkv_workspace_size_layers(p, 1, batch, total_tokens, max_seq_len, bytes);
+}
+
+int mixkv_workspace_size_layers(const mixkv_params* p, int32_t n_layers, int32_t batch,
+                                int64_t total_tokens, int32_t max_seq_len, size_t* bytes) {
   int rc = check_params(p);
   if (rc != MIXKV_OK) return rc;
-  if (!bytes || batch < 1 || total_tokens < batch || max_seq_len < 1) return MIXKV_ERR_INVALID_ARG;
-  if (batch > kMaxBatch) return MIXKV_ERR_UNSUPPORTED;
+  if (!bytes || batch < 1 || n_layers < 1 || total_tokens < batch || max_seq_len < 1)
+    return MIXKV_ERR_INVALID_ARG;
+  if (batch > kMaxBatch || n_layers > kMaxLayers) return MIXKV_ERR_UNSUPPORTED;
   if (total_tokens > 0x7fffffffLL / 2) return MIXKV_ERR_UNSUPPORTED;
   // a table with the worst-case chunk counts for these totals
   SeqTable st;
   memset(&st, 0, sizeof(st));
+  st.layers = n_layers;
   st.batch = batch;
   st.H = p->kv_heads;
   st.G = p->gqa_ratio;
@@ -235,7 +256,8 @@ int mixkv_workspace_size(const mixkv_params* p, int32_t batch, int64_t total_tok
   Workspace ws;
   carve(p, st, nullptr, &ws);
   // idx_capacity() saw empty sequences above; add the true bound
-  const size_t idx_bytes = (size_t)batch * p->kv_heads * (size_t)(p->budget - p->window) * 4;
+  const size_t idx_bytes =
+      (size_t)n_layers * batch * p->kv_heads * (size_t)(p->budget - p->window) * 4;
   *bytes = ws.bytes + align_up(idx_bytes, 256) + 256;
   return MIXKV_OK;
 }
@@ -268,15 +290,18 @@ int mixkv_select(const float* scores, const int32_t* cu_seqlens_host, int32_t ba
   return enqueue_select(c, scores, counts, t);
 }
 
-int mixkv_compress_layer_traced(const void* K, const void* V, const void* Qwin,
-                                const int32_t* cu_seqlens_host, int32_t batch, int32_t L,
-                                const mixkv_params* p, void* workspace, size_t workspace_bytes,
-                                const float* rbar_in_opt, void* K_out, void* V_out,
-                                int32_t* out_row_offsets, int32_t* idx_opt, int32_t* counts_opt,
-                                int32_t* idx_offsets_opt, float* s_comp_opt, int32_t* status_dev,
-                                void* stream, void* const* events_host, int32_t n_events) {
+namespace {
+// Body of the layer calls: n_layers layers of identical shape in one set of launches.
+int compress_impl(const void* K, const void* V, const void* Qwin, int n_layers,
+                  long long kv_layer_stride, long long q_layer_stride,
+                  const int32_t* cu_seqlens_host, int32_t batch, int32_t L, const mixkv_params* p,
+                  void* workspace, size_t workspace_bytes, const float* rbar_in_opt, void* K_out,
+                  void* V_out, int32_t* out_row_offsets, int32_t* idx_opt, int32_t* counts_opt,
+                  int32_t* idx_offsets_opt, float* s_comp_opt, int32_t* status_dev, void* stream,
+                  void* const* events_host, int32_t n_events) {
   LaunchCtx c;
-  int rc = make_ctx(p, cu_seqlens_host, batch, L, workspace, workspace_bytes, stream, &c);
+  int rc = make_ctx(p, cu_seqlens_host, batch, L, workspace, workspace_bytes, stream, &c, n_layers,
+                    kv_layer_stride, q_layer_stride);
   if (rc != MIXKV_OK) return rc;
   if (events_host && n_events > 0) {
     c.trace_events = events_host;
@@ -315,6 +340,35 @@ int mixkv_compress_layer_traced(const void* K, const void* V, const void* Qwin,
   }
   c.mark();
   return MIXKV_OK;
+}
+}  // namespace
+
+int mixkv_compress_layer_traced(const void* K, const void* V, const void* Qwin,
+                                const int32_t* cu_seqlens_host, int32_t batch, int32_t L,
+                                const mixkv_params* p, void* workspace, size_t workspace_bytes,
+                                const float* rbar_in_opt, void* K_out, void* V_out,
+                                int32_t* out_row_offsets, int32_t* idx_opt, int32_t* counts_opt,
+                                int32_t* idx_offsets_opt, float* s_comp_opt, int32_t* status_dev,
+                                void* stream, void* const* events_host, int32_t n_events) {
+  return compress_impl(K, V, Qwin, 1, 0, 0, cu_seqlens_host, batch, L, p, workspace,
+                       workspace_bytes, rbar_in_opt, K_out, V_out, out_row_offsets, idx_opt,
+                       counts_opt, idx_offsets_opt, s_comp_opt, status_dev, stream, events_host,
+                       n_events);
+}
+
+int mixkv_compress_layers(const void* K, const void* V, const void* Qwin, int32_t n_layers,
+                          int64_t kv_layer_stride, int64_t q_layer_stride,
+                          const int32_t* cu_seqlens_host, int32_t batch, int32_t L,
+                          const mixkv_params* p, void* workspace, size_t workspace_bytes,
+                          const float* rbar_in_opt, void* K_out, void* V_out,
+                          int32_t* out_row_offsets, int32_t* idx_opt, int32_t* counts_opt,
+                          int32_t* idx_offsets_opt, float* s_comp_opt, int32_t* status_dev,
+                          void* stream, void* const* events_host, int32_t n_events) {
+  if (kv_layer_stride < 0 || q_layer_stride < 0) return MIXKV_ERR_INVALID_ARG;
+  return compress_impl(K, V, Qwin, n_layers, kv_layer_stride, q_layer_stride, cu_seqlens_host,
+                       batch, L, p, workspace, workspace_bytes, rbar_in_opt, K_out, V_out,
+                       out_row_offsets, idx_opt, counts_opt, idx_offsets_opt, s_comp_opt,
+                       status_dev, stream, events_host, n_events);
 }
 
 int mixkv_compress_layer(const void* K, const void* V, const void* Qwin,
@@ -367,7 +421,7 @@ int mixkv_scores_static(const void* K, const void* V, const void* Qwin,
     if (rc != MIXKV_OK) return rc;
     SeqTable st;
     int max_len = 0;
-    rc = build_table(p, cu_seqlens_host, batch, L, &st, &max_len);
+    rc = build_table(p, cu_seqlens_host, batch, L, 1, &st, &max_len);
     if (rc != MIXKV_OK) return rc;
     Workspace ws;
     carve(p, st, nullptr, &ws);

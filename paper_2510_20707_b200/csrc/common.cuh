@@ -12,6 +12,7 @@ namespace mixkv {
 
 constexpr int kHeadDim = 128;        // d, fixed
 constexpr int kMaxBatch = 64;        // sequences per call
+constexpr int kMaxLayers = 1024;     // layers per call
 constexpr int kMaxNQ = 240;          // G*W upper bound (16 spare rows carry the mean key)
 constexpr int kTile = 128;           // keys per tensor-core tile
 constexpr int kPChunk = 2048;        // candidate positions per CTA in pool / mix
@@ -20,14 +21,17 @@ constexpr float kLog2e = 1.4426950408889634f;
 
 // Everything a kernel needs to find its slice of the ragged batch.
 struct SeqTable {
+  int layers;                        // layers handled by one call (an outer batch dimension)
   int batch, H, G, W, NQ;
   int Ltot, Ptot;
   int pchunks_total;                 // sum over sequences of ceil(P_b / kPChunk)
   int cu[kMaxBatch + 1];             // sequence offsets into Ltot
   int pchunk_start[kMaxBatch + 1];   // prefix sum of candidate chunks
   // persistent 128-key tile schedules of the two tensor-core passes, (b, h, t) order
-  int nt1, g1, q1, r1;               // pass 1: tiles over all L keys, CTAs, nt1 = q1 * g1 + r1
-  int nt2, g2, q2, r2;               // pass 2: tiles over the P candidate keys, likewise
+  // Tiles of one layer: nt1 over all L keys (pass 1), nt2 over the P candidate keys (pass 2).
+  // layers * nt tiles are split over g CTAs: layers * nt = q * g + r.
+  int nt1, g1, q1, r1;
+  int nt2, g2, q2, r2;
   int tile1_start[kMaxBatch + 1];    // prefix sum of H * ceil(L_b / 128)
   int tile2_start[kMaxBatch + 1];    // prefix sum of H * ceil(P_b / 128)
 };
@@ -40,6 +44,7 @@ struct Split {
 
 // Device workspace carve-up (all pointers into the caller's workspace).
 struct Workspace {
+  // every array below has a leading [layers] dimension
   float* kinv;        // [H, Ltot]   1 / |K_i|  (0 for a zero key)
   float* vnorm;       // [H, Ptot]   |V_i|
   float* s_ex_raw;    // [H, Ptot]   window attention score before pooling
@@ -63,6 +68,10 @@ struct LaunchCtx {
   SeqTable st;
   Workspace ws;
   mixkv_params p;
+  long long kv_layer_stride;   // elements between the K (V) tensors of consecutive layers
+  long long q_layer_stride;    // elements between the window queries of consecutive layers
+  int idx_cap;                 // selected rows one layer can produce (capacity of its index list)
+  int out_rows_cap;            // output rows reserved per layer: batch * H * B
   float scale_log2e;   // softmax scale * log2(e)
   int max_seq_len;
   int max_prefix;
@@ -91,6 +100,17 @@ cudaError_t launch_budget(const LaunchCtx& c, const float* scores, int* counts);
 // Selection (and optionally the mix before it and the gather after it) by one CTA cluster per
 // (sequence, head).  scores != nullptr: select on them; else mix first (s_div, rbar_in) and
 // write the mixed scores to s_comp_out.  counts_dev == nullptr: fixed budgets.
+// Index of (layer, head h, sequence b, position i) in a [layers, H, Ltot] / [layers, H, Ptot]
+// array.
+__host__ __device__ __forceinline__ size_t kpos(const SeqTable& st, int layer, int h, int b,
+                                                int i) {
+  return ((size_t)layer * st.H + h) * st.Ltot + st.cu[b] + i;
+}
+__host__ __device__ __forceinline__ size_t ppos(const SeqTable& st, int layer, int h, int b,
+                                                int i) {
+  return ((size_t)layer * st.H + h) * st.Ptot + (st.cu[b] - b * st.W) + i;
+}
+
 struct TailArgs {
   const float* scores;
   const float* s_div;

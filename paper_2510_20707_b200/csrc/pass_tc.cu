@@ -188,12 +188,12 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
     if (lane == 0) {
       int it = 0, segn = 0;
       bool seg_start = true;
-      for (TileIter ti(st.tile1_start, st.batch, H, lo, hi); ti.valid(); ti.next()) {
+      for (TileIter ti(st.tile1_start, st.batch, H, st.nt1, lo, hi); ti.valid(); ti.next()) {
         if (seg_start) {
           if (segn > 0 && !mbar_wait(&bars->qfree, (segn - 1) & 1, abort)) break;
           mbar_expect_tx(&bars->qfull, NQ * 256);
-          tma_load_2d(sQ, &tmQ, 0, ti.bh() * NQ, &bars->qfull);
-          tma_load_2d(sQ + QR * 128, &tmQ, 64, ti.bh() * NQ, &bars->qfull);
+          tma_load_3d(sQ, &tmQ, 0, ti.bh() * NQ, ti.layer, &bars->qfull);
+          tma_load_3d(sQ + QR * 128, &tmQ, 64, ti.bh() * NQ, ti.layer, &bars->qfull);
           ++segn;
         }
         seg_start = ti.seg_last();
@@ -201,8 +201,8 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
         if (!mbar_wait(&bars->empty[s], ph ^ 1, abort)) break;
         mbar_expect_tx(&bars->full[s], kTileBytes);
         const int y = st.cu[ti.b] + ti.t * kTile;
-        tma_load_3d(sK + s * kTileBytes, &tmK, 0, y, ti.h, &bars->full[s]);
-        tma_load_3d(sK + s * kTileBytes + kHalfBytes, &tmK, 64, y, ti.h, &bars->full[s]);
+        tma_load_4d(sK + s * kTileBytes, &tmK, 0, y, ti.h, ti.layer, &bars->full[s]);
+        tma_load_4d(sK + s * kTileBytes + kHalfBytes, &tmK, 64, y, ti.h, ti.layer, &bars->full[s]);
         ++it;
       }
       if (*abort) {
@@ -216,7 +216,7 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
       constexpr uint32_t idesc = umma_idesc_bf16(128, kTile);
       int it = 0, segn = 0;
       bool seg_start = true;
-      for (TileIter ti(st.tile1_start, st.batch, H, lo, hi); ti.valid(); ti.next()) {
+      for (TileIter ti(st.tile1_start, st.batch, H, st.nt1, lo, hi); ti.valid(); ti.next()) {
         if (seg_start) {
           if (!mbar_wait(&bars->qfull, segn & 1, abort)) break;
           ++segn;
@@ -258,7 +258,7 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
     float m_run = -1e30f, z_run = 0.f;
     int it = 0, seg_first = lo;
     bool seg_start = true;
-    for (TileIter ti(st.tile1_start, st.batch, H, lo, hi); ti.valid(); ti.next()) {
+    for (TileIter ti(st.tile1_start, st.batch, H, st.nt1, lo, hi); ti.valid(); ti.next()) {
       if (seg_start) {
         m_run = -1e30f;
         z_run = 0.f;
@@ -307,7 +307,7 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
     for (int e = 0; e < 8; ++e) acc[e] = 0.f;
     int it = 0, seg_first = lo;
     bool seg_start = true;
-    for (TileIter ti(st.tile1_start, st.batch, H, lo, hi); ti.valid(); ti.next()) {
+    for (TileIter ti(st.tile1_start, st.batch, H, st.nt1, lo, hi); ti.valid(); ti.next()) {
       if (seg_start) {
 #pragma unroll
         for (int e = 0; e < 8; ++e) acc[e] = 0.f;
@@ -354,7 +354,7 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
         }
         const int i = ti.t * kTile + grp * 16 + bt * 8 + (c >> 1);   // the row this lane holds
         const float inv = (ok && i < L && p[0] > 0.f) ? rsqrtf(p[0]) : 0.f;
-        if (i < L && (c & 1) == 0) ws.kinv[(size_t)ti.h * st.Ltot + st.cu[ti.b] + i] = inv;
+        if (i < L && (c & 1) == 0) ws.kinv[kpos(st, ti.layer, ti.h, ti.b, i)] = inv;
 #pragma unroll
         for (int rr = 0; rr < 8; ++rr) {
           const float w = __shfl_sync(0xffffffffu, inv, (lane & 16) | (rr << 1));
@@ -489,12 +489,12 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
     if (lane == 0) {
       int it = 0, segn = 0;
       bool seg_start = true;
-      for (TileIter ti(st.tile2_start, st.batch, H, lo, hi); ti.valid(); ti.next()) {
+      for (TileIter ti(st.tile2_start, st.batch, H, st.nt2, lo, hi); ti.valid(); ti.next()) {
         if (seg_start) {
           if (segn > 0 && !mbar_wait(&bars->qfree, (segn - 1) & 1, abort)) break;
           mbar_expect_tx(&bars->qfull, NQ * 256);
-          tma_load_2d(sQ, &tmQ, 0, ti.bh() * NQ, &bars->qfull);
-          tma_load_2d(sQ + NB * 128, &tmQ, 64, ti.bh() * NQ, &bars->qfull);
+          tma_load_3d(sQ, &tmQ, 0, ti.bh() * NQ, ti.layer, &bars->qfull);
+          tma_load_3d(sQ + NB * 128, &tmQ, 64, ti.bh() * NQ, ti.layer, &bars->qfull);
           ++segn;
         }
         seg_start = ti.seg_last();
@@ -502,8 +502,8 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
         if (!mbar_wait(&bars->kempty[s], ph ^ 1, abort)) break;
         mbar_expect_tx(&bars->kfull[s], kTileBytes);
         const int y = st.cu[ti.b] + ti.t * kTile;
-        tma_load_3d(sK + s * kTileBytes, &tmK, 0, y, ti.h, &bars->kfull[s]);
-        tma_load_3d(sK + s * kTileBytes + kHalfBytes, &tmK, 64, y, ti.h, &bars->kfull[s]);
+        tma_load_4d(sK + s * kTileBytes, &tmK, 0, y, ti.h, ti.layer, &bars->kfull[s]);
+        tma_load_4d(sK + s * kTileBytes + kHalfBytes, &tmK, 64, y, ti.h, ti.layer, &bars->kfull[s]);
         ++it;
       }
       if (*abort) {
@@ -516,7 +516,7 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
     if (lane == 0 && use_vnorm) {
       int vit = 0;
       bool ok = true;
-      for (TileIter ti(st.tile2_start, st.batch, H, lo, hi); ti.valid() && ok; ti.next()) {
+      for (TileIter ti(st.tile2_start, st.batch, H, st.nt2, lo, hi); ti.valid() && ok; ti.next()) {
         const int y = st.cu[ti.b] + ti.t * kTile;
         for (int sub = 0; sub < 2; ++sub) {
           const int vs = vit % vstages, vph = (vit / vstages) & 1;
@@ -526,8 +526,8 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
           }
           mbar_expect_tx(&bars->vfull[vs], kVSubBytes);
           unsigned char* dst = sV + vs * kVSubBytes;
-          tma_load_3d(dst, &tmV, 0, y + sub * 64, ti.h, &bars->vfull[vs]);
-          tma_load_3d(dst + kVSubBytes / 2, &tmV, 64, y + sub * 64, ti.h, &bars->vfull[vs]);
+          tma_load_4d(dst, &tmV, 0, y + sub * 64, ti.h, ti.layer, &bars->vfull[vs]);
+          tma_load_4d(dst + kVSubBytes / 2, &tmV, 64, y + sub * 64, ti.h, ti.layer, &bars->vfull[vs]);
           ++vit;
         }
       }
@@ -542,7 +542,7 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
       const uint32_t idesc = umma_idesc_bf16(128, NB);
       int it = 0, segn = 0;
       bool seg_start = true;
-      for (TileIter ti(st.tile2_start, st.batch, H, lo, hi); ti.valid(); ti.next()) {
+      for (TileIter ti(st.tile2_start, st.batch, H, st.nt2, lo, hi); ti.valid(); ti.next()) {
         if (seg_start) {
           if (!mbar_wait(&bars->qfull, segn & 1, abort)) break;
           if (!mbar_wait(&bars->kbready, segn & 1, abort)) break;
@@ -580,7 +580,7 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
     float dmin = INFINITY, dmax = -INFINITY, dsum = 0.f, exw = 0.f;
     int it = 0, seg_first = lo;
     bool seg_start = true;
-    for (TileIter ti(st.tile2_start, st.batch, H, lo, hi); ti.valid(); ti.next()) {
+    for (TileIter ti(st.tile2_start, st.batch, H, st.nt2, lo, hi); ti.valid(); ti.next()) {
       const int L = st.cu[ti.b + 1] - st.cu[ti.b], P = L - W;
       if (seg_start) {
         // fold pass 1's per-segment softmax statistics of this (b, h) into one log2 normaliser
@@ -588,7 +588,8 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
         named_bar_sync(1, kEpiThreads);   // the previous segment's readers of sbq / part are done
         {
           const int per_head = (st.tile1_start[ti.b + 1] - st.tile1_start[ti.b]) / H;
-          const SegList sl(st.tile1_start[ti.b] + ti.h * per_head, per_head, split1(st));
+          const SegList sl(ti.layer * st.nt1 + st.tile1_start[ti.b] + ti.h * per_head, per_head,
+                           split1(st));
           const int nunits = NQ <= 128 ? 2 : 1;
           const int ew = warp - kEpiWarp0;
           float M[8], Z[8];
@@ -632,7 +633,7 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
       const int ts = it & 1, tph = (it >> 1) & 1;
       const int ikey = ti.t * kTile + key;
       float kinv_i = 0.f;
-      if (wg == 1 && ikey < P) kinv_i = ws.kinv[(size_t)ti.h * st.Ltot + st.cu[ti.b] + ikey];
+      if (wg == 1 && ikey < P) kinv_i = ws.kinv[kpos(st, ti.layer, ti.h, ti.b, ikey)];
       const bool ok = mbar_wait(&bars->tfull[ts], tph, abort);
       tc_fence_after();
       const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + ts * 256;
@@ -673,7 +674,7 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
       if (group_sync_stop(1, kEpiThreads, et == 0, abort, bars->vote[0], it)) break;
       if (wg == 1) {
         if (ikey < P) {
-          const size_t poff = (size_t)ti.h * st.Ptot + (st.cu[ti.b] - ti.b * W);
+          const size_t poff = ppos(st, ti.layer, ti.h, ti.b, 0);
           const float ex = (acc0 + acc1) + sx[ts * 128 + key];
           ws.s_ex_raw[poff + ikey] = ex;
           const float sd = -dot * kinv_i;
@@ -718,11 +719,12 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
     float vmin = INFINITY, vmax = -INFINITY, vsum = 0.f;
     int it = 0, segn = 0, seg_first = lo;
     bool seg_start = true;
-    for (TileIter ti(st.tile2_start, st.batch, H, lo, hi); ti.valid(); ti.next()) {
+    for (TileIter ti(st.tile2_start, st.batch, H, st.nt2, lo, hi); ti.valid(); ti.next()) {
       if (seg_start) {
         const int L = st.cu[ti.b + 1] - st.cu[ti.b];
         const int per_head = (st.tile1_start[ti.b + 1] - st.tile1_start[ti.b]) / H;
-        const SegList sl(st.tile1_start[ti.b] + ti.h * per_head, per_head, split1(st));
+        const SegList sl(ti.layer * st.nt1 + st.tile1_start[ti.b] + ti.h * per_head, per_head,
+                           split1(st));
         float s = 0.f;
         for (int e0 = 0; e0 < sl.nseg; e0 += 16) {   // sixteen loads in flight per thread
           float v[16];
@@ -766,8 +768,8 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
             const double nn = ((double)sred[28] + (double)sred[29]) + ((double)sred[30] + (double)sred[31]);
             const double T = (double)L;
             const float r = (float)((nn - T) / (T * (T - 1.0)));   // Eq. 4
-            ws.rbar[ti.bh()] = r;
-            if (rbar_out) rbar_out[ti.bh()] = r;
+            ws.rbar[ti.unit()] = r;
+            if (rbar_out) rbar_out[ti.unit()] = r;
           }
         }
         ++segn;
@@ -804,7 +806,7 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
         const int i = ti.t * kTile + sub * 64 + vr;
         if (ok && i < P) {
           const float n = sqrtf((ss[0] + ss[1]) + (ss[2] + ss[3]));
-          ws.vnorm[(size_t)ti.h * st.Ptot + (st.cu[ti.b] - ti.b * W) + i] = n;
+          ws.vnorm[ppos(st, ti.layer, ti.h, ti.b, i)] = n;
           vmin = fminf(vmin, n);
           vmax = fmaxf(vmax, n);
           vsum += n;
@@ -854,29 +856,32 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// X [H, Ltot, d] bf16 as a 3-D tensor (d, Ltot, H) with boxes of 64 x rows x 1.  Rows past the
-// end of the tensor read as zero.
-bool map_rows3d(const LaunchCtx& c, const void* X, int box_rows, CUtensorMap* tm) {
+// X [layers, H, Ltot, d] bf16 (layer stride given in elements) as a 4-D tensor (d, Ltot, H,
+// layers) with boxes of 64 x rows x 1 x 1.  Rows past the end of the tensor read as zero.
+bool map_kv(const LaunchCtx& c, const void* X, int box_rows, CUtensorMap* tm) {
   EncodeTiledFn enc = encode_fn();
   if (!enc) return false;
-  cuuint64_t dims[3] = {(cuuint64_t)kHeadDim, (cuuint64_t)c.st.Ltot, (cuuint64_t)c.st.H};
-  cuuint64_t strides[2] = {(cuuint64_t)kHeadDim * 2, (cuuint64_t)c.st.Ltot * kHeadDim * 2};
-  cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
-  cuuint32_t es[3] = {1, 1, 1};
-  return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(X), dims, strides, box, es,
+  cuuint64_t dims[4] = {(cuuint64_t)kHeadDim, (cuuint64_t)c.st.Ltot, (cuuint64_t)c.st.H,
+                        (cuuint64_t)c.st.layers};
+  cuuint64_t strides[3] = {(cuuint64_t)kHeadDim * 2, (cuuint64_t)c.st.Ltot * kHeadDim * 2,
+                           (cuuint64_t)c.kv_layer_stride * 2};
+  cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 1, 1};
+  cuuint32_t es[4] = {1, 1, 1, 1};
+  return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(X), dims, strides, box, es,
              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// X [rows, d] bf16 as a 2-D tensor (d, rows) with boxes of 64 x box_rows.
-bool map_rows2d(const void* X, long long rows, int box_rows, CUtensorMap* tm) {
+// Q [layers, batch * H * NQ, d] bf16 as a 3-D tensor (d, rows, layers) with boxes of 64 x NQ x 1.
+bool map_q(const LaunchCtx& c, const void* Q, CUtensorMap* tm) {
   EncodeTiledFn enc = encode_fn();
   if (!enc) return false;
-  cuuint64_t dims[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows};
-  cuuint64_t strides[1] = {(cuuint64_t)kHeadDim * 2};
-  cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
-  cuuint32_t es[2] = {1, 1};
-  return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(X), dims, strides, box, es,
+  cuuint64_t dims[3] = {(cuuint64_t)kHeadDim, (cuuint64_t)c.st.batch * c.st.H * c.st.NQ,
+                        (cuuint64_t)c.st.layers};
+  cuuint64_t strides[2] = {(cuuint64_t)kHeadDim * 2, (cuuint64_t)c.q_layer_stride * 2};
+  cuuint32_t box[3] = {64, (cuuint32_t)c.st.NQ, 1};
+  cuuint32_t es[3] = {1, 1, 1};
+  return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(Q), dims, strides, box, es,
              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -922,9 +927,7 @@ int device_sm_count() {
 
 cudaError_t launch_pass1(const LaunchCtx& c, const void* K, const void* Q, int* status) {
   CUtensorMap tmK, tmQ;
-  if (!map_rows3d(c, K, kTile, &tmK) ||
-      !map_rows2d(Q, (long long)c.st.batch * c.st.H * c.st.NQ, c.st.NQ, &tmQ))
-    return cudaErrorInvalidValue;
+  if (!map_kv(c, K, kTile, &tmK) || !map_q(c, Q, &tmQ)) return cudaErrorInvalidValue;
   static bool done1[64] = {false}, done2[64] = {false};
   if (c.st.NQ <= 128) {
     const size_t smem = pass1_smem(1);
@@ -944,8 +947,7 @@ cudaError_t launch_pass2(const LaunchCtx& c, const void* K, const void* V, const
                          float* s_div_out, float* rbar_out, int* status) {
   CUtensorMap tmK, tmV, tmQ;
   const void* Vsrc = c.p.use_vnorm ? V : K;   // the V map is never used without VNorm
-  if (!map_rows3d(c, K, kTile, &tmK) || !map_rows3d(c, Vsrc, 64, &tmV) ||
-      !map_rows2d(Q, (long long)c.st.batch * c.st.H * c.st.NQ, c.st.NQ, &tmQ))
+  if (!map_kv(c, K, kTile, &tmK) || !map_kv(c, Vsrc, 64, &tmV) || !map_q(c, Q, &tmQ))
     return cudaErrorInvalidValue;
   static bool done[64] = {false};
   cudaError_t e = ensure_smem(k_pass2, kSmemLimit, done);

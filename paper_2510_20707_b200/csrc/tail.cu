@@ -20,17 +20,17 @@ namespace {
 //   s_in_scaled  = (|V_i| - sc[0]) * sc[1]
 //   s_div_scaled = (s_div_i - sc[2]) * sc[3]
 //   sc[4]        = redundancy used by the mix
-__device__ void head_scalars(const SeqTable& st, const Workspace& ws, const int b, const int h,
-                             const int pool_k, const int pool_mode, const int use_vnorm,
+__device__ void head_scalars(const SeqTable& st, const Workspace& ws, const int layer, const int b,
+                             const int h, const int pool_k, const int pool_mode, const int use_vnorm,
                              const float eps, const float* __restrict__ rbar_in, const int lane,
                              float* sc) {
-  const int bh = b * st.H + h;
+  const int unit = (layer * st.batch + b) * st.H + h;
   const int P = st.cu[b + 1] - st.cu[b] - st.W;
   float dmin = INFINITY, dmax = -INFINITY, dsum = 0.f, exw = 0.f;
   float vmin = INFINITY, vmax = -INFINITY, vsum = 0.f;
   {
     const int per_head = (st.tile2_start[b + 1] - st.tile2_start[b]) / st.H;
-    const SegList sl(st.tile2_start[b] + h * per_head, per_head, split2(st));
+    const SegList sl(layer * st.nt2 + st.tile2_start[b] + h * per_head, per_head, split2(st));
     for (int e = lane; e < sl.nseg; e += 32) {   // lanes take segments side by side
       const int start = sl.start(e);
       const float4 d4 = ws.dstat[start];
@@ -53,7 +53,7 @@ __device__ void head_scalars(const SeqTable& st, const Workspace& ws, const int 
   } else {
     float e = 0.f;
     for (int c = st.pchunk_start[b] + lane; c < st.pchunk_start[b + 1]; c += 32)
-      e += ws.exsum[(size_t)h * st.pchunks_total + c];
+      e += ws.exsum[((size_t)layer * st.H + h) * st.pchunks_total + c];
     ex = warp_sum(e);
   }
   dmin = warp_min(dmin);
@@ -81,7 +81,7 @@ __device__ void head_scalars(const SeqTable& st, const Workspace& ws, const int 
     sc[1] = cin;
     sc[2] = dmin;
     sc[3] = dinv * a_div;
-    sc[4] = rbar_in ? rbar_in[bh] : ws.rbar[bh];
+    sc[4] = rbar_in ? rbar_in[unit] : ws.rbar[unit];
   }
 }
 
@@ -127,12 +127,12 @@ k_poolsum(const SeqTable st, const Workspace ws, const int k) {
   __shared__ float sred[8];
   pdl_launch_dependents();
   pdl_wait();
-  const int pcx = blockIdx.x, h = blockIdx.y;
+  const int pcx = blockIdx.x, h = blockIdx.y, layer = blockIdx.z;
   const int b = find_seq(st.pchunk_start, st.batch, pcx);
   const int P = st.cu[b + 1] - st.cu[b] - st.W;
   const int p0 = (pcx - st.pchunk_start[b]) * kPChunk;
   const int p1 = min(p0 + kPChunk, P);
-  const size_t poff = (size_t)h * st.Ptot + (st.cu[b] - b * st.W);
+  const size_t poff = ppos(st, layer, h, b, 0);
   const int half = k >> 1;
   for (int t = threadIdx.x; t < (p1 - p0) + 2 * half; t += 256) {
     const int i = p0 - half + t;
@@ -147,7 +147,7 @@ k_poolsum(const SeqTable st, const Workspace ws, const int k) {
   if (threadIdx.x == 0) {
     float s = 0.f;
     for (int w = 0; w < 8; ++w) s += sred[w];
-    ws.exsum[(size_t)h * st.pchunks_total + pcx] = s;
+    ws.exsum[((size_t)layer * st.H + h) * st.pchunks_total + pcx] = s;
   }
 }
 
@@ -161,16 +161,16 @@ k_mixpool(const SeqTable st, const Workspace ws, const float* __restrict__ s_div
   __shared__ float sc[8];
   pdl_launch_dependents();
   pdl_wait();
-  const int pcx = blockIdx.x, h = blockIdx.y;
+  const int pcx = blockIdx.x, h = blockIdx.y, layer = blockIdx.z;
   const int b = find_seq(st.pchunk_start, st.batch, pcx);
   const int P = st.cu[b + 1] - st.cu[b] - st.W;
   const int p0 = (pcx - st.pchunk_start[b]) * kPChunk;
   const int p1 = min(p0 + kPChunk, P);
-  const size_t poff = (size_t)h * st.Ptot + (st.cu[b] - b * st.W);
+  const size_t poff = ppos(st, layer, h, b, 0);
   const int half = mp.pool_k >> 1;
   const float pad = mp.pool_mode == MIXKV_POOL_AVG ? 0.f : -INFINITY;
   if (threadIdx.x < 32)
-    head_scalars(st, ws, b, h, mp.pool_k, mp.pool_mode, mp.use_vnorm, mp.eps, rbar_in,
+    head_scalars(st, ws, layer, b, h, mp.pool_k, mp.pool_mode, mp.use_vnorm, mp.eps, rbar_in,
                  threadIdx.x, sc);
   for (int t = threadIdx.x; t < (p1 - p0) + 2 * half; t += 256) {
     const int i = p0 - half + t;
@@ -251,12 +251,13 @@ k_budget(const SeqTable st, const float* __restrict__ scores, int* __restrict__ 
   __shared__ int s_gt[64], s_eq[64];
   pdl_launch_dependents();
   pdl_wait();
-  const int b = blockIdx.x, H = st.H;
+  const int b = blockIdx.x, layer = blockIdx.y, H = st.H;
+  counts += (size_t)layer * st.batch * H;
   const int P = st.cu[b + 1] - st.cu[b] - st.W;
   const long long total = (long long)H * P;
   long long N = (long long)H * (Bp - floor_slots);
   if (N > total) N = total;
-  const float* base = scores + (st.cu[b] - b * st.W);
+  const float* base = scores + ppos(st, layer, 0, b, 0);
   if (N <= 0) {
     for (int h = threadIdx.x; h < H; h += blockDim.x) counts[b * H + h] = min(floor_slots, P);
     return;
@@ -315,6 +316,9 @@ struct TailKernelArgs {
   __nv_bfloat16* V_out;
   int Bp;                     // B - W
   int cached;                 // keys of the slice fit the shared-memory cache
+  long long kv_layer_stride;  // elements between consecutive layers of K (V)
+  int idx_cap;                // index-list entries reserved per layer
+  int out_rows_cap;           // output rows reserved per layer
   MixParams mp;
 };
 
@@ -343,12 +347,18 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
   __shared__ float sc[8];
   cg::cluster_group cluster = cg::this_cluster();
   const int crank = (int)cluster.block_rank();
-  const int bh = blockIdx.x / kTailCluster, b = bh / st.H, h = bh % st.H;
   const int BH = st.batch * st.H;
+  const int unit = blockIdx.x / kTailCluster;          // (layer, sequence, head)
+  const int layer = unit / BH, bh = unit % BH, b = bh / st.H, h = bh % st.H;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int W = st.W;
   const int P = st.cu[b + 1] - st.cu[b] - W;
-  const size_t poff = (size_t)h * st.Ptot + (st.cu[b] - b * W);
+  const size_t poff = ppos(st, layer, h, b, 0);
+  // this layer's slices of the per-layer arrays
+  const int* counts_dev = a.counts_dev ? a.counts_dev + (size_t)layer * BH : nullptr;
+  int* counts_out = a.counts_out ? a.counts_out + (size_t)layer * BH : nullptr;
+  int* idx_offsets = a.idx_offsets + (size_t)layer * (BH + 1);
+  int* out_row_offsets = a.out_row_offsets ? a.out_row_offsets + (size_t)layer * (BH + 1) : nullptr;
   // slice of this CTA: positions [c0, c0 + n)
   const int chunk = (P + kTailCluster - 1) / kTailCluster;
   const int R = (chunk + kTailThreads - 1) / kTailThreads;   // positions per thread
@@ -363,10 +373,10 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
   // ---- budget and output offsets of this (b, h)
   if (tid < 32) {
     int off = 0, cnt;
-    if (a.counts_dev) {
-      for (int t = lane; t < bh; t += 32) off += a.counts_dev[t];
+    if (counts_dev) {
+      for (int t = lane; t < bh; t += 32) off += counts_dev[t];
       for (int o = 16; o > 0; o >>= 1) off += __shfl_xor_sync(0xffffffffu, off, o);
-      cnt = a.counts_dev[bh];
+      cnt = counts_dev[bh];
     } else {
       off = fixed_offset(st, bh, a.Bp);
       cnt = min(a.Bp, P);
@@ -375,12 +385,12 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
       s_off = off;
       s_sel[1] = cnt;
       if (crank == 0) {
-        a.idx_offsets[bh] = off;
-        if (a.counts_out) a.counts_out[bh] = cnt;
-        if (a.out_row_offsets) a.out_row_offsets[bh] = off + bh * W;
+        idx_offsets[bh] = off;
+        if (counts_out) counts_out[bh] = cnt;
+        if (out_row_offsets) out_row_offsets[bh] = off + bh * W;
         if (bh == BH - 1) {
-          a.idx_offsets[BH] = off + cnt;
-          if (a.out_row_offsets) a.out_row_offsets[BH] = off + cnt + BH * W;
+          idx_offsets[BH] = off + cnt;
+          if (out_row_offsets) out_row_offsets[BH] = off + cnt + BH * W;
         }
       }
     }
@@ -393,8 +403,8 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
     const int half = a.mp.pool_k >> 1;
     const float pad = a.mp.pool_mode == MIXKV_POOL_AVG ? 0.f : -INFINITY;
     if (warp == 1)
-      head_scalars(st, ws, b, h, a.mp.pool_k, a.mp.pool_mode, a.mp.use_vnorm, a.mp.eps, a.rbar_in,
-                   lane, sc);
+      head_scalars(st, ws, layer, b, h, a.mp.pool_k, a.mp.pool_mode, a.mp.use_vnorm, a.mp.eps,
+                   a.rbar_in, lane, sc);
     for (int t = tid; t < n + 2 * half; t += kTailThreads) {
       const int i = c0 - half + t;
       sraw[t] = (i >= 0 && i < P) ? ws.s_ex_raw[poff + i] : pad;
@@ -437,7 +447,7 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
   for (int t = tid; t < 256; t += kTailThreads) hist[0][t] = 0;
   __syncthreads();
   const int want = s_sel[1];
-  int* out = a.idx + s_off;
+  int* out = a.idx + (size_t)layer * a.idx_cap + s_off;
   auto key_at = [&](int j) -> unsigned {
     return cached ? skeys[kslot(j)] : order_key(src[poff + c0 + j]);
   };
@@ -566,20 +576,22 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
   if (a.K_out) {
     const int n_sel = max(want, 0) < P ? max(want, 0) : P;
     const int rows = n_sel + W;
+    const __nv_bfloat16* Ksrc = a.K + (size_t)layer * a.kv_layer_stride;
+    const __nv_bfloat16* Vsrc = a.V + (size_t)layer * a.kv_layer_stride;
     const size_t srow0 = (size_t)h * st.Ltot + st.cu[b];
-    const size_t drow0 = (size_t)(s_off + bh * W);
+    const size_t drow0 = (size_t)layer * a.out_rows_cap + (size_t)(s_off + bh * W);
     const int hw = tid >> 4, l = tid & 15;                       // 32 half-warps, 16 B per lane
     constexpr int kRowsPerSweep = kTailCluster * (kTailThreads / 16);
     for (int rb = crank * (kTailThreads / 16) + hw; rb < rows; rb += 2 * kRowsPerSweep) {
       const int ra = rb + kRowsPerSweep;
       const int sa = rb < n_sel ? __ldcg(out + rb) : P + (rb - n_sel);
       const int sb = ra < rows ? (ra < n_sel ? __ldcg(out + ra) : P + (ra - n_sel)) : -1;
-      const uint4 k0 = __ldg(reinterpret_cast<const uint4*>(a.K + (srow0 + sa) * kHeadDim) + l);
-      const uint4 v0 = __ldg(reinterpret_cast<const uint4*>(a.V + (srow0 + sa) * kHeadDim) + l);
+      const uint4 k0 = __ldg(reinterpret_cast<const uint4*>(Ksrc + (srow0 + sa) * kHeadDim) + l);
+      const uint4 v0 = __ldg(reinterpret_cast<const uint4*>(Vsrc + (srow0 + sa) * kHeadDim) + l);
       uint4 k1 = make_uint4(0, 0, 0, 0), v1 = k1;
       if (sb >= 0) {
-        k1 = __ldg(reinterpret_cast<const uint4*>(a.K + (srow0 + sb) * kHeadDim) + l);
-        v1 = __ldg(reinterpret_cast<const uint4*>(a.V + (srow0 + sb) * kHeadDim) + l);
+        k1 = __ldg(reinterpret_cast<const uint4*>(Ksrc + (srow0 + sb) * kHeadDim) + l);
+        v1 = __ldg(reinterpret_cast<const uint4*>(Vsrc + (srow0 + sb) * kHeadDim) + l);
       }
       reinterpret_cast<uint4*>(a.K_out + (drow0 + rb) * kHeadDim)[l] = k0;
       reinterpret_cast<uint4*>(a.V_out + (drow0 + rb) * kHeadDim)[l] = v0;
@@ -612,18 +624,21 @@ MixParams mix_params(const mixkv_params& p) {
 }  // namespace
 
 cudaError_t launch_poolsum(const LaunchCtx& c) {
-  return launch_pdl(k_poolsum, dim3(c.st.pchunks_total, c.st.H), dim3(256), 0, c.stream, 1, c.st,
+  return launch_pdl(k_poolsum, dim3(c.st.pchunks_total, c.st.H, c.st.layers), dim3(256), 0,
+                    c.stream, 1, c.st,
                     c.ws, c.p.pool_kernel);
 }
 
 cudaError_t launch_mixpool(const LaunchCtx& c, const float* s_div, const float* rbar_in,
                            float* s_ex_out, float* s_comp) {
-  return launch_pdl(k_mixpool, dim3(c.st.pchunks_total, c.st.H), dim3(256), 0, c.stream, 1, c.st,
+  return launch_pdl(k_mixpool, dim3(c.st.pchunks_total, c.st.H, c.st.layers), dim3(256), 0,
+                    c.stream, 1, c.st,
                     c.ws, s_div, rbar_in, s_ex_out, s_comp, mix_params(c.p));
 }
 
 cudaError_t launch_budget(const LaunchCtx& c, const float* scores, int* counts) {
-  return launch_pdl(k_budget, dim3(c.st.batch), dim3(1024), 0, c.stream, 1, c.st, scores, counts,
+  return launch_pdl(k_budget, dim3(c.st.batch, c.st.layers), dim3(1024), 0, c.stream, 1, c.st,
+                    scores, counts,
                     c.p.budget - c.p.window, floor_slots(c.p));
 }
 
@@ -648,6 +663,9 @@ cudaError_t launch_tail(const LaunchCtx& c, const TailArgs& t) {
   a.K_out = (__nv_bfloat16*)t.K_out;
   a.V_out = (__nv_bfloat16*)t.V_out;
   a.Bp = c.p.budget - c.p.window;
+  a.kv_layer_stride = c.kv_layer_stride;
+  a.idx_cap = c.idx_cap;
+  a.out_rows_cap = c.out_rows_cap;
   a.mp = mix_params(c.p);
   const int chunk = (c.max_prefix + kTailCluster - 1) / kTailCluster;
   const int R = (chunk + kTailThreads - 1) / kTailThreads;
@@ -670,7 +688,7 @@ cudaError_t launch_tail(const LaunchCtx& c, const TailArgs& t) {
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64) have[dev] = ask;
   }
-  const dim3 grid(c.st.batch * c.st.H * kTailCluster);
+  const dim3 grid(c.st.layers * c.st.batch * c.st.H * kTailCluster);
   if (fused)
     return launch_pdl(k_tail<true>, grid, dim3(kTailThreads), smem, c.stream, kTailCluster, c.st,
                       c.ws, a);

@@ -84,6 +84,14 @@ __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* tm, in
       "l"(tm), "r"(x), "r"(y), "r"(z), "r"(smem_u32(bar))
       : "memory");
 }
+__device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* tm, int x, int y, int z,
+                                            int w, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], "
+      "[%1, {%2, %3, %4, %5}], [%6];" ::"r"(smem_u32(dst)),
+      "l"(tm), "r"(x), "r"(y), "r"(z), "r"(w), "r"(smem_u32(bar))
+      : "memory");
+}
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* tm) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(tm) : "memory");
 }
@@ -228,10 +236,10 @@ __device__ __forceinline__ TileCoord tile_coord(const int* tile_start, int batch
   return c;
 }
 __host__ __device__ __forceinline__ Split split1(const SeqTable& st) {
-  return Split{st.nt1, st.g1, st.q1, st.r1};
+  return Split{st.layers * st.nt1, st.g1, st.q1, st.r1};
 }
 __host__ __device__ __forceinline__ Split split2(const SeqTable& st) {
-  return Split{st.nt2, st.g2, st.q2, st.r2};
+  return Split{st.layers * st.nt2, st.g2, st.q2, st.r2};
 }
 // First tile of CTA c.
 __host__ __device__ __forceinline__ int cta_first_tile(int c, const Split& sp) {
@@ -243,23 +251,27 @@ __host__ __device__ __forceinline__ int tile_owner(int t, const Split& sp) {
   return t < big ? t / (sp.q + 1) : sp.r + (t - big) / sp.q;
 }
 
-// Walks the tiles [lo, hi) of one CTA in (b, h, t) order without dividing per tile.
+// Walks the tiles [lo, hi) of one CTA in (layer, b, h, t) order without dividing per tile.
+// Tile ids run over all layers: id = layer * nt + (tile of the layer).
 struct TileIter {
-  int id, hi, b, h, t, per_head, H;
+  int id, hi, layer, b, h, t, per_head, H, batch, nt;
   const int* tile_start;
-  __device__ TileIter(const int* tile_start_, int batch, int H_, int lo, int hi_)
-      : id(lo), hi(hi_), H(H_), tile_start(tile_start_) {
-    b = h = t = 0;
+  __device__ TileIter(const int* tile_start_, int batch_, int H_, int nt_, int lo, int hi_)
+      : id(lo), hi(hi_), H(H_), batch(batch_), nt(nt_), tile_start(tile_start_) {
+    layer = b = h = t = 0;
     per_head = 1;
     if (lo < hi_) {
-      const TileCoord c = tile_coord(tile_start_, batch, H_, lo);
+      layer = lo / nt_;
+      const TileCoord c = tile_coord(tile_start_, batch_, H_, lo - layer * nt_);
       b = c.b, h = c.h, t = c.t;
       per_head = (tile_start_[b + 1] - tile_start_[b]) / H_;
     }
   }
   __device__ __forceinline__ bool valid() const { return id < hi; }
+  // (sequence, head) of the tile inside its layer, and over all layers
   __device__ __forceinline__ int bh() const { return b * H + h; }
-  // first / last tile of a segment: a run of tiles of one (b, h) inside this CTA's range
+  __device__ __forceinline__ int unit() const { return (layer * batch + b) * H + h; }
+  // last tile of a segment: a run of tiles of one (layer, b, h) inside this CTA's range
   __device__ __forceinline__ bool seg_last() const { return id + 1 == hi || t + 1 == per_head; }
   __device__ __forceinline__ void next() {
     ++id;
@@ -267,7 +279,10 @@ struct TileIter {
       t = 0;
       if (++h == H) {
         h = 0;
-        ++b;
+        if (++b == batch) {
+          b = 0;
+          ++layer;
+        }
         if (id < hi) per_head = (tile_start[b + 1] - tile_start[b]) / H;
       }
     }

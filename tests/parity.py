@@ -132,3 +132,43 @@ def run_layer_parity(wl: synth.Workload, layer: int = 0, variant: str = "literal
     check_gather(x["K"], to_bits(out["K_out"]), ro, idx, offs, cu, W, H)
     check_gather(x["V"], to_bits(out["V_out"]), ro, idx, offs, cu, W, H)
     return out, ref, ref_s
+
+
+def run_layers_parity(wl: synth.Workload, layers, variant: str = "calibrated", pad_rows: int = 0,
+                      **kw):
+    """mixkv_compress_layers over several layers at once against the oracle, layer by layer.
+    pad_rows > 0 leaves a gap between the layers of K / V (a strided layer dimension)."""
+    po, pg = params_pair(wl, **kw)
+    cu = wl.cu_seqlens
+    cu_arg = None if wl.batch == 1 else cu
+    cu_list = None if wl.batch == 1 else [int(c) for c in cu]
+    xs = [synth.make_layer(wl, l, variant) for l in layers]
+    H, W, NL = wl.kv_heads, wl.window, len(xs)
+    Ltot = wl.total_tokens
+
+    def stack(name):
+        t = torch.stack([to_dev(x[name]) for x in xs])
+        if pad_rows and name != "Q":
+            buf = torch.zeros((NL, H * Ltot + pad_rows, 128), dtype=torch.bfloat16, device="cuda")
+            buf[:, :H * Ltot] = t.reshape(NL, H * Ltot, 128)
+            t = buf[:, :H * Ltot].view(NL, H, Ltot, 128)
+        return t
+
+    K, V, Q = stack("K"), stack("V"), stack("Q")
+    out = binding.compress_layers(K, V, Q, pg, cu_seqlens=cu_list)
+    torch.cuda.synchronize()
+    assert int(out["status"].item()) == 0
+    for n, x in enumerate(xs):
+        ref_s = oracle.scores(x["K"], x["V"], x["Q"], po, cu=cu_arg)
+        ref = oracle.select(ref_s["s_comp"], po, cu=cu_arg)
+        check_scores(f"s_comp[layer {n}]", out["s_comp"][n].cpu().numpy(), ref_s["s_comp"], cu, W)
+        offs = out["idx_offsets"][n].cpu().numpy()
+        idx = out["idx"][n].cpu().numpy()
+        counts = out["counts"][n].cpu().numpy()
+        slack = None if po.budget_mode == 0 else 2
+        check_selection(idx, offs, counts, ref, ref_s["s_comp"], cu, W, H, counts_slack=slack)
+        ro = out["out_row_offsets"][n].cpu().numpy()
+        assert np.array_equal(ro, offs + np.arange(wl.batch * H + 1) * W)
+        check_gather(x["K"], to_bits(out["K_out"][n]), ro, idx, offs, cu, W, H)
+        check_gather(x["V"], to_bits(out["V_out"][n]), ro, idx, offs, cu, W, H)
+    return out

@@ -7,7 +7,7 @@ import torch
 import oracle
 from paper_2510_20707_b200 import binding, synth
 from parity import (check_rbar, check_scores, check_selection, params_pair, run_layer_parity,
-                    to_bits, to_dev)
+                    run_layers_parity, to_bits, to_dev)
 
 pytestmark = pytest.mark.gpu
 
@@ -116,3 +116,26 @@ def test_c4_ragged_adaptive_layer():
 @pytest.mark.parametrize("name", ["C3", "C3b"])
 def test_c3_long_video_layer(name):
     run_layer_parity(synth.CONFIGS[name], 13, "calibrated")
+
+
+# ---- several layers in one call (mixkv_compress_layers)
+def test_layers_batched_small_ragged():
+    wl = synth.small_workload(H=3, G=2, W=16, seq_lens=(300, 1025, 47), pool_kernel=7, budget=48,
+                              seed=9)
+    wl = synth.replace(wl, layers=5)
+    run_layers_parity(wl, range(5))
+    run_layers_parity(synth.with_budget(wl, 48, budget_mode=1), range(5))
+    run_layers_parity(wl, range(3), pad_rows=24, pool_mode=1)
+
+
+def test_layers_batched_c2():
+    run_layers_parity(synth.CONFIGS["C2"], (0, 13, 27, 5))
+
+
+def test_layers_batched_c4_adaptive():
+    run_layers_parity(synth.CONFIGS["C4"], (0, 1))
+
+
+def test_layers_batched_c3_c5():
+    run_layers_parity(synth.CONFIGS["C3"], (3, 20))
+    run_layers_parity(synth.CONFIGS["C5"], (0, 31))
