@@ -1,8 +1,8 @@
 #!/usr/bin/env python
 """Benchmark of the MixKV per-layer KV-cache compression step on B200.
 
-A step is one pass of the whole hot path (score -> mix -> select -> gather, i.e. one
-mixkv_compress_layer call per layer) over all layers of one synthetic prefill.  The metric
+A step is one pass of the whole hot path (score -> mix -> select -> gather) over all layers of
+one synthetic prefill: one mixkv_compress_layers call.  The metric
 is KV tokens compressed per second: tokens of the batch / time of one step (every layer
 compresses the same tokens), whole job over all GPUs.  Each GPU runs an independent replica
 (the step has no cross-GPU exchange), so scaling is weak.
@@ -44,6 +44,7 @@ def parse_args():
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (debug)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-per-layer", action="store_true")
     return ap.parse_args()
 
 
@@ -220,37 +221,42 @@ def run_mixkv(args):
                         pool_kernel=wl.pool_kernel, budget=wl.budget, budget_mode=wl.budget_mode,
                         ada_floor=wl.ada_floor)
     cu_list = None if wl.batch == 1 else [int(c) for c in wl.cu_seqlens]
-    H, Ltot = wl.kv_heads, wl.total_tokens
+    H, Ltot, NL = wl.kv_heads, wl.total_tokens, wl.layers
     n_stage = binding.launches_per_layer(pg)
     stage_names = binding.stage_names(pg)
 
-    # ---- inputs: every layer has its own buffers; enough sets that the inputs cycled
-    # through between two uses of the same buffer exceed L2 several times
-    host = []
-    for layer in range(wl.layers):
+    # ---- inputs: K, V [layers, H, Ltot, d] and Q [layers, batch, H*G, W, d] in pinned host
+    # memory; enough device copies ("sets") that the bytes streamed between two uses of a
+    # buffer exceed L2 several times
+    host = {k: torch.empty((NL,) + shp, dtype=torch.bfloat16).pin_memory()
+            for k, shp in (("K", (H, Ltot, 128)), ("V", (H, Ltot, 128)),
+                           ("Q", (wl.batch, H * wl.gqa_ratio, wl.window, 128)))}
+    for layer in range(NL):
         x = synth.make_layer(wl, layer, args.variant)
-        host.append({k: torch.from_numpy(v.view(np.int16)).view(torch.bfloat16).pin_memory()
-                     for k, v in x.items()})
-    set_bytes = sum(t.numel() * 2 for h in host for t in h.values())
+        for k, v in x.items():
+            host[k][layer].copy_(torch.from_numpy(v.view(np.int16)).view(torch.bfloat16))
+    set_bytes = sum(t.numel() * 2 for t in host.values())
     n_sets = max(1, int(np.ceil(4 * L2_BYTES / set_bytes)))
-    dev_in = [[{k: t.to(dev) for k, t in h.items()} for h in host] for _ in range(n_sets)]
-    ws_bytes = binding.workspace_size(pg, wl.batch, Ltot, max(wl.seq_lens))
+    dev_in = [{k: t.to(dev) for k, t in host.items()} for _ in range(n_sets)]
+    ws_bytes = binding.workspace_size_layers(pg, NL, wl.batch, Ltot, max(wl.seq_lens))
     workspace = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
     rows_cap = wl.batch * H * wl.budget
-    outs = [{"K_out": torch.empty((rows_cap, 128), dtype=torch.bfloat16, device=dev),
-             "V_out": torch.empty((rows_cap, 128), dtype=torch.bfloat16, device=dev),
-             "out_row_offsets": torch.empty(wl.batch * H + 1, dtype=torch.int32, device=dev),
-             "status": torch.zeros(1, dtype=torch.int32, device=dev)} for _ in range(wl.layers)]
+
+    def new_out():
+        return {"K_out": torch.empty((NL, rows_cap, 128), dtype=torch.bfloat16, device=dev),
+                "V_out": torch.empty((NL, rows_cap, 128), dtype=torch.bfloat16, device=dev),
+                "out_row_offsets": torch.empty((NL, wl.batch * H + 1), dtype=torch.int32, device=dev),
+                "status": torch.zeros(1, dtype=torch.int32, device=dev)}
+
+    out = new_out()
     stream = torch.cuda.current_stream()
 
     def step(s, trace=None):
-        bufs = dev_in[s % n_sets]
-        for layer in range(wl.layers):
-            b = bufs[layer]
-            binding.compress_layer(b["K"], b["V"], b["Q"], pg, cu_seqlens=cu_list,
-                                   workspace=workspace, stream=torch.cuda.current_stream(),
-                                   out=outs[layer], want_aux=False,
-                                   trace_events=None if trace is None else trace[layer])
+        """One step = the whole hot path over all layers: ONE mixkv_compress_layers call."""
+        b = dev_in[s % n_sets]
+        binding.compress_layers(b["K"], b["V"], b["Q"], pg, cu_seqlens=cu_list,
+                                workspace=workspace, stream=stream, out=out, want_aux=False,
+                                trace_events=trace)
 
     def barrier():
         torch.cuda.synchronize()
@@ -259,20 +265,9 @@ def run_mixkv(args):
             torch.cuda.synchronize()
 
     def check_status():
-        bad = [int(o["status"].item()) for o in outs if int(o["status"].item()) != 0]
-        if bad:
-            raise SystemExit(f"device status {bad[0]} reported by a kernel")
-
-    # ---- one CUDA graph per input set: a whole step (all layers) captured from the C-ABI calls
-    step(0)                      # first call outside capture (one-time function attributes)
-    torch.cuda.synchronize()
-    graphs = []
-    for i in range(n_sets):
-        g = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g):
-            step(i)
-        graphs.append(g)
-    stream = torch.cuda.current_stream()
+        st_ = int(out["status"].item())
+        if st_ != 0:
+            raise SystemExit(f"device status {st_} reported by a kernel")
 
     def timed(run, n_warm, n_steps):
         for s in range(n_warm):
@@ -290,50 +285,58 @@ def run_mixkv(args):
             dist.all_reduce(t, op=dist.ReduceOp.MAX)
         return float(t.item()) / n_steps
 
-    # ---- timed region: K replays of the captured step (device-resident inputs)
+    # ---- timed region: K steps, device-resident inputs, CUDA events on the launching stream
     for s in range(args.warmup):
-        graphs[s % n_sets].replay()
+        step(s)
     barrier()
+    check_status()
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
         time.sleep(0.25)
-    ms_per_step = timed(lambda s: graphs[s % n_sets].replay(), 0, args.steps)
+    ms_per_step = timed(step, 0, args.steps)
     clocks = sampler.stop() if rank == 0 else None
     check_status()
     value = world * wl.total_tokens / (ms_per_step * 1e-3)
 
-    # ---- the same step issued call by call from Python (host launch cost included)
-    direct_ms = timed(lambda s: step(s), 1, max(3, min(args.steps, 10)))
-
-    # ---- per-kernel CUDA-event times: every kernel of every layer bracketed by events on the
-    # launching stream, over args.steps traced steps
-    n_tr = max(1, min(args.steps, 5))
-    tr_ev = [[[torch.cuda.Event(enable_timing=True) for _ in range(n_stage + 1)]
-              for _ in range(wl.layers)] for _ in range(n_tr)]
+    # ---- per-kernel CUDA-event times: every kernel of a step bracketed by events on the
+    # launching stream
+    n_tr = max(1, min(args.steps, 10))
+    tr_ev = [[torch.cuda.Event(enable_timing=True) for _ in range(n_stage + 1)] for _ in range(n_tr)]
     for st_ in tr_ev:
-        for ly in st_:
-            for e in ly:
-                e.record(stream)          # forces creation of the underlying CUDA event
+        for e in st_:
+            e.record(stream)          # forces creation of the underlying CUDA event
     torch.cuda.synchronize()
-    tr_c = [[(C.c_void_p * (n_stage + 1))(*[e.cuda_event for e in ly]) for ly in st_]
-            for st_ in tr_ev]
-    # the GPU is kept busy while the host enqueues the traced steps, so that the events are
-    # reached back to back on the device and their differences are device times, not host
-    # enqueue times
-    torch.cuda._sleep(int(6e-3 * 1.9e9 * n_tr * wl.layers / 28))
+    tr_c = [(C.c_void_p * (n_stage + 1))(*[e.cuda_event for e in st_]) for st_ in tr_ev]
     for s in range(n_tr):
         step(s, trace=tr_c[s])
     torch.cuda.synchronize()
     check_status()
-    stage_us = {name: 1e3 * statistics.mean(ly[i].elapsed_time(ly[i + 1])
-                                            for st_ in tr_ev for ly in st_)
+    stage_ms = {name: statistics.mean(st_[i].elapsed_time(st_[i + 1]) for st_ in tr_ev)
                 for i, name in enumerate(stage_names)}
+
+    # ---- the same layers through the one-layer entry point, one call per layer (context)
+    per_layer_ms = None
+    if not args.no_per_layer:
+        ws1 = torch.empty(binding.workspace_size(pg, wl.batch, Ltot, max(wl.seq_lens)),
+                          dtype=torch.uint8, device=dev)
+        o1 = {"K_out": out["K_out"][0], "V_out": out["V_out"][0],
+              "out_row_offsets": out["out_row_offsets"][0], "status": out["status"]}
+
+        def step_per_layer(s):
+            b = dev_in[s % n_sets]
+            for layer in range(NL):
+                binding.compress_layer(b["K"][layer], b["V"][layer], b["Q"][layer], pg,
+                                       cu_seqlens=cu_list, workspace=ws1, stream=stream, out=o1,
+                                       want_aux=False)
+
+        per_layer_ms = timed(step_per_layer, 1, max(3, min(args.steps, 5)))
+        check_status()
 
     # ---- end to end: host buffers in, compact cache out, copies inside the timed region
     e2e = None
     if not args.no_e2e:
-        e2e = run_e2e(args, wl, pg, cu_list, host, workspace, dev, world, barrier, binding)
+        e2e = run_e2e(args, wl, pg, cu_list, host, dev, world, barrier, binding)
 
     if world > 1:
         dist.barrier()
@@ -343,26 +346,23 @@ def run_mixkv(args):
         return
     peak, peak_kind = peaks()
     ab = algorithmic_bytes(wl)
-    dom = max(("pass1", "pass2"), key=lambda k: stage_us[k])
-    dom_us = stage_us[dom]
-    achieved = ab[dom] / (dom_us * 1e-6) / 1e9
-    layer_ms = ms_per_step / wl.layers
+    dom = max(("pass1", "pass2"), key=lambda k: stage_ms[k])
+    dom_ms = stage_ms[dom]
+    achieved = NL * ab[dom] / (dom_ms * 1e-3) / 1e9
+    layer_ms = ms_per_step / NL
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16 in, f32 accumulate",
         "data": "synthetic",
         "config": workload_config(wl, args.variant, {
-            "l2": f"{n_sets} set(s) of per-layer inputs, {n_sets * set_bytes / 2**20:.0f} MiB cycled "
+            "l2": f"{n_sets} set(s) of inputs, {n_sets * set_bytes / 2**20:.0f} MiB cycled "
                   f"(> 126 MB L2) between two uses of a buffer",
-            "launch": "one CUDA graph per input set, captured from the per-layer C-ABI calls "
-                      "and replayed once per step",
+            "launch": "one mixkv_compress_layers call per step (all layers in one set of kernels)",
             "parallelism": "replicas only" if world > 1 else "single GPU"}),
         "per_layer_latency_us": layer_ms * 1e3,
-        "token_layers_per_s": world * wl.total_tokens * wl.layers / (ms_per_step * 1e-3),
-        "direct_call": {"ms_per_step": direct_ms, "per_layer_latency_us": direct_ms / wl.layers * 1e3,
-                        "note": "same step, one ctypes call per layer from Python, no graph"},
-        "stage_us": stage_us,
+        "token_layers_per_s": world * wl.total_tokens * NL / (ms_per_step * 1e-3),
+        "stage_ms": stage_ms,
         "layer_roofline": {"bound": "hbm", "achieved": ab["layer"] / (layer_ms * 1e-3) / 1e9,
                            "peak": peak, "unit": "GB/s",
                            "frac": ab["layer"] / (layer_ms * 1e-3) / 1e9 / peak,
@@ -371,11 +371,15 @@ def run_mixkv(args):
         "roofline": {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "traffic": None,
                      "peak_source": f"{peak_kind} copy bandwidth",
-                     "algorithmic_bytes_per_launch": ab[dom],
-                     "kernel_us": dom_us},
+                     "algorithmic_bytes_per_launch": NL * ab[dom],
+                     "kernel_ms": dom_ms},
         "clocks": clocks,
-        "gpu_launches": n_stage * wl.layers * args.steps,
+        "gpu_launches": n_stage * args.steps,
     }
+    if per_layer_ms is not None:
+        line["one_layer_per_call"] = {
+            "ms_per_step": per_layer_ms, "per_layer_latency_us": per_layer_ms / NL * 1e3,
+            "note": "same step as one mixkv_compress_layer call per layer, issued from Python"}
     if e2e is not None:
         line["e2e"] = e2e
     if not args.no_cpu_baseline:
@@ -385,44 +389,50 @@ def run_mixkv(args):
         dist.destroy_process_group()
 
 
-def run_e2e(args, wl, pg, cu_list, host, workspace, dev, world, barrier, binding):
-    """Same metric through the public call with HOST buffers: every layer's K, V, Q are copied
-    from pinned host memory, compressed, and the compact cache is copied back, all inside the
-    timed region.  Two streams alternate layers so copies overlap compute."""
+def run_e2e(args, wl, pg, cu_list, host, dev, world, barrier, binding):
+    """Same metric through the public call with HOST buffers: the layers are cut into groups;
+    each group's K, V, Q are copied from pinned host memory, compressed with one
+    mixkv_compress_layers call, and its compact cache is copied back, all inside the timed
+    region.  Two streams alternate groups so copies overlap compute."""
     import torch
     import torch.distributed as dist
 
-    H = wl.kv_heads
+    H, NL = wl.kv_heads, wl.layers
     rows_cap = wl.batch * H * wl.budget
+    grp = max(1, min(NL, 4))
+    groups = [(g0, min(g0 + grp, NL)) for g0 in range(0, NL, grp)]
     streams = [torch.cuda.Stream(device=dev) for _ in range(2)]
+    ws_bytes = binding.workspace_size_layers(pg, grp, wl.batch, wl.total_tokens, max(wl.seq_lens))
     slots = []
     for i in range(2):
-        ws = torch.empty_like(workspace)
         slots.append({
-            "in": {k: torch.empty_like(t, device=dev) for k, t in host[0].items()},
-            "ws": ws,
-            "out": {"K_out": torch.empty((rows_cap, 128), dtype=torch.bfloat16, device=dev),
-                    "V_out": torch.empty((rows_cap, 128), dtype=torch.bfloat16, device=dev),
-                    "out_row_offsets": torch.empty(wl.batch * H + 1, dtype=torch.int32, device=dev),
+            "in": {k: torch.empty((grp,) + tuple(t.shape[1:]), dtype=t.dtype, device=dev)
+                   for k, t in host.items()},
+            "ws": torch.empty(ws_bytes, dtype=torch.uint8, device=dev),
+            "out": {"K_out": torch.empty((grp, rows_cap, 128), dtype=torch.bfloat16, device=dev),
+                    "V_out": torch.empty((grp, rows_cap, 128), dtype=torch.bfloat16, device=dev),
+                    "out_row_offsets": torch.empty((grp, wl.batch * H + 1), dtype=torch.int32,
+                                                   device=dev),
                     "status": torch.zeros(1, dtype=torch.int32, device=dev)}})
-    host_out = [{"K_out": torch.empty((rows_cap, 128), dtype=torch.bfloat16).pin_memory(),
-                 "V_out": torch.empty((rows_cap, 128), dtype=torch.bfloat16).pin_memory(),
-                 "out_row_offsets": torch.empty(wl.batch * H + 1, dtype=torch.int32).pin_memory()}
-                for _ in range(wl.layers)]
-    h2d = sum(t.numel() * t.element_size() for t in host[0].values()) * wl.layers
-    d2h = sum(t.numel() * t.element_size() for t in host_out[0].values()) * wl.layers
+    host_out = {"K_out": torch.empty((NL, rows_cap, 128), dtype=torch.bfloat16).pin_memory(),
+                "V_out": torch.empty((NL, rows_cap, 128), dtype=torch.bfloat16).pin_memory(),
+                "out_row_offsets": torch.empty((NL, wl.batch * H + 1), dtype=torch.int32).pin_memory()}
+    h2d = sum(t.numel() * t.element_size() for t in host.values())
+    d2h = sum(t.numel() * t.element_size() for t in host_out.values())
 
     def step():
-        for layer in range(wl.layers):
-            sl, st = slots[layer % 2], streams[layer % 2]
+        for gi, (g0, g1) in enumerate(groups):
+            sl, st = slots[gi % 2], streams[gi % 2]
+            n = g1 - g0
             with torch.cuda.stream(st):
-                for k, t in host[layer].items():
-                    sl["in"][k].copy_(t, non_blocking=True)
-                binding.compress_layer(sl["in"]["K"], sl["in"]["V"], sl["in"]["Q"], pg,
-                                       cu_seqlens=cu_list, workspace=sl["ws"], stream=st,
-                                       out=sl["out"], want_aux=False)
-                for k, t in host_out[layer].items():
-                    t.copy_(sl["out"][k], non_blocking=True)
+                for k, t in host.items():
+                    sl["in"][k][:n].copy_(t[g0:g1], non_blocking=True)
+                o = {k: (v if k == "status" else v[:n]) for k, v in sl["out"].items()}
+                binding.compress_layers(sl["in"]["K"][:n], sl["in"]["V"][:n], sl["in"]["Q"][:n], pg,
+                                        cu_seqlens=cu_list, workspace=sl["ws"], stream=st, out=o,
+                                        want_aux=False)
+                for k, t in host_out.items():
+                    t[g0:g1].copy_(sl["out"][k][:n], non_blocking=True)
 
     steps = max(3, min(args.steps, 10))
     for _ in range(3):
@@ -439,16 +449,19 @@ def run_e2e(args, wl, pg, cu_list, host, workspace, dev, world, barrier, binding
         e.record(s)
     torch.cuda.synchronize()
     wall_ms = (time.perf_counter() - t0) * 1e3
+    bad = [int(sl["out"]["status"].item()) for sl in slots if int(sl["out"]["status"].item()) != 0]
+    if bad:
+        raise SystemExit(f"device status {bad[0]} reported by a kernel (e2e)")
     dev_ms = max(b.elapsed_time(e) for b in beg for e in end)
-    ms = max(dev_ms, 0.0)
-    t = torch.tensor([ms], dtype=torch.float64, device=dev)
+    t = torch.tensor([dev_ms], dtype=torch.float64, device=dev)
     if world > 1:
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
     ms = float(t.item()) / steps
     return {"value": world * wl.total_tokens / (ms * 1e-3), "unit": UNIT,
             "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms,
             "steps": steps, "wall_ms_per_step": wall_ms / steps,
-            "note": "pinned host K/V/Q -> device, compress, compact cache -> pinned host"}
+            "note": f"pinned host K/V/Q -> device in groups of {grp} layers, "
+                    "mixkv_compress_layers per group, compact cache -> pinned host"}
 
 
 def main():
