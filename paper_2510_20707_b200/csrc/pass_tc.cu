@@ -276,8 +276,8 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
         const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + ts * (MB * 128) + col0;
         uint32_t ra[32], rb[32];
         tmem_ld32(taddr, ra);
-#pragma unroll
-        for (int c0 = 0; c0 < NC; c0 += 64) {
+#pragma unroll 1
+        for (int c0 = 0; c0 < NC; c0 += 64) {   // kept rolled: the body must stay in the i-cache
           tmem_ld_wait();
           tmem_ld_fence(ra);
           tmem_ld32(taddr + c0 + 32, rb);
@@ -319,7 +319,7 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
       const bool ok = mbar_wait(&bars->full[s], ph, abort);
       const unsigned char* tile = sK + s * kTileBytes + chalf * kHalfBytes;
       // two batches of eight rows keep the register footprint small
-#pragma unroll
+#pragma unroll 1
       for (int bt = 0; bt < 2; ++bt) {
         uint4 u[8];
         float p[8];
@@ -645,8 +645,8 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
         // 16-column chunks, the next one in flight while this one is reduced
         uint32_t ra[16], rb[16];
         if (nch > 0) tmem_ld16(taddr + cbeg, ra);
-#pragma unroll
-        for (int ci = 0; ci < kMaxNQ / 32 + 1; ci += 2) {
+#pragma unroll 1
+        for (int ci = 0; ci < nch; ci += 2) {   // kept rolled: the body must stay in the i-cache
           if (ci < nch) {
             tmem_ld_wait();
             tmem_ld_fence(ra);
