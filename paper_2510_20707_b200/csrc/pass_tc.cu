@@ -80,12 +80,17 @@ __device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
   return d;
 }
 
+constexpr size_t kSmemLimit = 227 * 1024;   // dynamic shared memory a CTA may ask for
+
 // ======================================================================== pass 1
-constexpr int kP1Stages = 4;   // K tile ring
+constexpr int kP1MaxStages = 6;
+// K tile ring: as deep as shared memory allows next to the query tile (the deeper the ring, the
+// more bytes in flight towards HBM)
+__host__ __device__ constexpr int p1_stages(int MB) { return MB == 2 ? 5 : 6; }
 
 struct P1Bars {
-  uint64_t full[kP1Stages];
-  uint64_t empty[kP1Stages];
+  uint64_t full[kP1MaxStages];
+  uint64_t empty[kP1MaxStages];
   uint64_t tfull[2];
   uint64_t tempty[2];
   uint64_t qfull;
@@ -139,10 +144,20 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
   unsigned char* base =
       reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
   constexpr int QR = MB * 128;                 // query rows the MMA reads
+  constexpr int kP1Stages = p1_stages(MB);
   unsigned char* sQ = base;                    // 2 halves x [QR x 128 B]
   unsigned char* sK = sQ + 2 * QR * 128;       // kP1Stages x 32 KB
-  float* sks = reinterpret_cast<float*>(sK + kP1Stages * kTileBytes);  // [8][128] key-sum exchange
-  P1Bars* bars = reinterpret_cast<P1Bars*>(sks + 1024);
+  float* sks = reinterpret_cast<float*>(sK + kP1Stages * kTileBytes);  // [4][128] key-sum exchange
+  P1Bars* bars = reinterpret_cast<P1Bars*>(sks + 512);
+  {
+    // the carve-up above must fit behind the (1 KB aligned) base
+    unsigned dyn;
+    asm("mov.u32 %0, %%dynamic_smem_size;" : "=r"(dyn));
+    if ((size_t)(reinterpret_cast<unsigned char*>(bars + 1) - smem_dyn) > dyn) {
+      if (threadIdx.x == 0 && status) atomicExch(status, MIXKV_ERR_CUDA);
+      return;
+    }
+  }
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int NQ = st.NQ, W = st.W, H = st.H;
@@ -369,14 +384,16 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
       }
       if (group_sync_stop(2, 128, kt == 0, abort, bars->vote, it)) break;
       if (seg_start) {
-        // fold the eight row groups: sks[grp][dim]
+        // fold the eight row groups: the two of a warp by shuffle, the four warps through sks
+        const int aw = warp - kAuxWarp0;
 #pragma unroll
-        for (int e = 0; e < 8; ++e) sks[grp * 128 + c * 8 + e] = acc[e];
+        for (int e = 0; e < 8; ++e) {
+          const float v = acc[e] + __shfl_xor_sync(0xffffffffu, acc[e], 16);
+          if (lane < 16) sks[aw * 128 + c * 8 + e] = v;
+        }
         named_bar_sync(2, 128);
-        float t = 0.f;
-#pragma unroll
-        for (int g2 = 0; g2 < 8; ++g2) t += sks[g2 * 128 + kt];
-        ws.ksum[(size_t)seg_first * kHeadDim + kt] = t;
+        ws.ksum[(size_t)seg_first * kHeadDim + kt] =
+            (sks[kt] + sks[128 + kt]) + (sks[256 + kt] + sks[384 + kt]);
         named_bar_sync(2, 128);
       }
       ++it;
@@ -392,8 +409,6 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
 constexpr int kP2KStages = 3;              // K tiles (32 KB each)
 constexpr int kP2VStagesMax = 4;           // V half tiles: 64 rows, 16 KB each
 constexpr int kVSubBytes = 64 * 256;
-constexpr size_t kSmemLimit = 227 * 1024;
-
 struct P2Bars {
   uint64_t kfull[kP2KStages];
   uint64_t kempty[kP2KStages];
@@ -887,8 +902,12 @@ bool map_q(const LaunchCtx& c, const void* Q, CUtensorMap* tm) {
 }
 
 size_t pass1_smem(int MB) {
-  return 1024 + (size_t)2 * MB * 128 * 128 + kP1Stages * kTileBytes + 1024 * 4 + sizeof(P1Bars) +
-         64;
+  // up to 1023 bytes of alignment slack in front of the carve-up; never beyond the limit (the
+  // kernel checks that its carve-up fits behind the aligned base)
+  const size_t need = (size_t)2 * MB * 128 * 128 + (size_t)p1_stages(MB) * kTileBytes + 512 * 4 +
+                      sizeof(P1Bars);
+  const size_t want = need + 1024;
+  return want < kSmemLimit ? want : kSmemLimit;
 }
 size_t pass2_smem(int NQ, int vstages) {
   return 1024 + (size_t)2 * (NQ + kExtraRows) * 128 + kP2KStages * kTileBytes +
