@@ -336,7 +336,7 @@ __device__ __forceinline__ int fixed_offset(const SeqTable& st, int bh, int Bp) 
 __device__ __forceinline__ int kslot(int j) { return j + (j >> 5); }
 
 template <bool FUSED>
-__global__ void __launch_bounds__(kTailThreads, 1)
+__global__ void __launch_bounds__(kTailThreads, 2)
 k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
   extern __shared__ __align__(16) unsigned char tail_smem[];
   __shared__ int hist[2][256];
@@ -421,13 +421,27 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
     __syncthreads();
     const float invk = 1.0f / (float)a.mp.pool_k;
     if (R <= 8) {
+      // the eight pooling windows advance together (same order of additions as pool_window),
+      // so their shared-memory loads overlap instead of forming eight serial chains
+      float ex[8];
+      const bool avg = a.mp.pool_mode == MIXKV_POOL_AVG;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) ex[e] = avg ? 0.f : -INFINITY;
+      for (int u = 0; u < a.mp.pool_k; ++u) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const int j = min(e * kTailThreads + tid, n - 1 > 0 ? n - 1 : 0);
+          const float w = sraw[j + u];
+          ex[e] = avg ? ex[e] + w : fmaxf(ex[e], w);
+        }
+      }
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
         const int j = e * kTailThreads + tid;
         held[e] = 0.f;
         if (j < n) {
-          const float ex = pool_window(sraw + j, a.mp.pool_k, a.mp.pool_mode, invk);
-          held[e] = mix_one(ex, vn[e], dv[e], sc, a.mp.use_vnorm, a.mp.mix_mode);
+          held[e] = mix_one(avg ? ex[e] * invk : ex[e], vn[e], dv[e], sc, a.mp.use_vnorm,
+                            a.mp.mix_mode);
           skeys[kslot(j)] = order_key(held[e]);
         }
       }
@@ -470,9 +484,15 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
           const unsigned key = key_at(j);
           if ((key & mask) == prefix) digit = (key >> shift) & 255u;
         }
-        const unsigned peers = __match_any_sync(0xffffffffu, digit);
-        if (digit != 0xffffffffu && (int)(__ffs(peers) - 1) == lane)
-          atomicAdd(&hist[buf][digit], __popc(peers));
+        // most warps see one digit only (always in the first passes): one vote, one add
+        const unsigned first = __shfl_sync(0xffffffffu, digit, 0);
+        if (__all_sync(0xffffffffu, digit == first)) {
+          if (lane == 0 && digit != 0xffffffffu) atomicAdd(&hist[buf][digit], 32);
+        } else {
+          const unsigned peers = __match_any_sync(0xffffffffu, digit);
+          if (digit != 0xffffffffu && (int)(__ffs(peers) - 1) == lane)
+            atomicAdd(&hist[buf][digit], __popc(peers));
+        }
       }
       cluster.sync();
       // every CTA adds up the cluster's histograms and finds the digit itself
