@@ -102,7 +102,7 @@ void carve(const mixkv_params* p, const SeqTable& st, unsigned char* base, Works
   ws->rowstat = (float2*)take(NL * st.nt1 * 2 * st.NQ * 8);
   ws->ksum = (float*)take(NL * st.nt1 * kHeadDim * 4);
   ws->vstat = (float4*)take(NL * st.nt2 * 16);
-  ws->dstat = (float4*)take(NL * st.nt2 * 16);
+  ws->dstat = (float4*)take(NL * st.nt2 * 2 * 16);
   ws->exsum = (float*)take(NL * H * st.pchunks_total * 4);
   ws->rbar = (float*)take(NL * BH * 4);
   ws->counts = (int*)take(NL * BH * 4);

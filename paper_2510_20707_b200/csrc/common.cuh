@@ -55,7 +55,7 @@ struct Workspace {
   float2* rowstat;    // [nt1, 2, NQ]  softmax (max, sum) of each window row, log2 units
   float* ksum;        // [nt1, d]      sum of unit keys
   float4* vstat;      // [nt2]         (min, max, sum, -) of |V_i| over candidates
-  float4* dstat;      // [nt2]         (min, max, sum) of s_div, window-count-weighted sum of s_ex_raw
+  float4* dstat;      // [nt2, 2]      per epilogue warpgroup: (min, max, sum) of s_div, window-count-weighted sum of s_ex_raw
   float* exsum;       // [H, pchunks_total]   per-chunk sum of pooled s_ex (max pooling only)
   float* rbar;        // [batch*H]
   int* counts;        // [batch*H]

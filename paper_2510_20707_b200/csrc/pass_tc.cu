@@ -421,7 +421,7 @@ struct P2Bars {
   uint64_t kbready;
   uint32_t tmem_base;
   int abort;
-  int vote[2][2];
+  int vote[3][2];
 };
 
 // Sixteen logit columns of one key: adds exp2(logit * scale - normaliser of the column).
@@ -455,10 +455,9 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
   unsigned char* sQ = base;                   // 2 halves x [NB x 128 B]
   unsigned char* sK = sQ + 2 * NB * 128;      // kP2KStages x 32 KB
   unsigned char* sV = sK + kP2KStages * kTileBytes;   // vstages x 16 KB
-  float* sbq = reinterpret_cast<float*>(sV + vstages * kVSubBytes);  // [256] negated normalisers
-  float* sx = sbq + 256;                      // [2][128] partial sums WG0 -> WG1
-  float* sred = sx + 256;                     // [32]
-  float2* part = reinterpret_cast<float2*>(sred + 32);   // [8][256] per-warp row statistics
+  float* sbq = reinterpret_cast<float*>(sV + vstages * kVSubBytes);  // [2][256] negated normalisers
+  float* sred = sbq + 512;                    // [64]: 2 x 16 epilogue, 16 value norms + 4 mean key
+  float2* part = reinterpret_cast<float2*>(sred + 64);   // [2][4][256] per-warp row statistics
   P2Bars* bars = reinterpret_cast<P2Bars*>(part + 8 * 256);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -479,7 +478,7 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(&bars->tfull[s], 1);
-      mbar_init(&bars->tempty[s], kEpiThreads);
+      mbar_init(&bars->tempty[s], 128);    // the warpgroup that owns the accumulator stage
     }
     mbar_init(&bars->qfull, 1);
     mbar_init(&bars->qfree, 1);
@@ -584,13 +583,18 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
     }
   } else if (warp >= kEpiWarp0 && warp < kEpiWarp0 + kEpiWarps) {
     // ------------------------------------------------------------------ epilogue
+    // The two warpgroups take alternate tiles (warpgroup g owns accumulator stage g), one key
+    // per thread and all G*W columns of it, so a tile needs no exchange between warpgroups and
+    // the groups never wait for each other: each folds the segment's row statistics into its
+    // own normaliser table and leaves its own partial score statistics.
     const int quarter = warp & 3, wg = (warp - kEpiWarp0) >> 2;
-    const int et = tid - kEpiWarp0 * 32;        // 0..255
+    const int gt = (tid - kEpiWarp0 * 32) & 127;   // thread inside the warpgroup
+    const int gw = gt >> 5;                        // warp inside the warpgroup
     const int key = quarter * 32 + lane;
-    // warpgroup 0 takes the first half of the 16-column chunks, warpgroup 1 the rest
-    const int CA = ((NQ / 16 + 1) >> 1) * 16;
-    const int cbeg = wg == 0 ? 0 : CA;
-    const int nch = (wg == 0 ? CA : NQ - CA) / 16;
+    const int nch = NQ / 16;
+    float* mybq = sbq + wg * 256;
+    float2* mypart = part + wg * 4 * 256;
+    const int barid = 1 + wg;                      // named barriers 1, 2: one per warpgroup
     const f32x2 sc2 = pack2(scale_log2e, scale_log2e);
     float dmin = INFINITY, dmax = -INFINITY, dsum = 0.f, exw = 0.f;
     int it = 0, seg_first = lo;
@@ -598,20 +602,20 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
     for (TileIter ti(st.tile2_start, st.batch, H, st.nt2, lo, hi); ti.valid(); ti.next()) {
       const int L = st.cu[ti.b + 1] - st.cu[ti.b], P = L - W;
       if (seg_start) {
-        // fold pass 1's per-segment softmax statistics of this (b, h) into one log2 normaliser
-        // per window row (the 1/W of the window mean folded in); warps take segments side by side
-        named_bar_sync(1, kEpiThreads);   // the previous segment's readers of sbq / part are done
+        // fold pass 1's per-segment softmax statistics of this (layer, b, h) into one log2
+        // normaliser per window row (the 1/W of the window mean folded in); the four warps
+        // take segments side by side
+        named_bar_sync(barid, 128);   // the previous segment's readers of mybq / mypart are done
         {
           const int per_head = (st.tile1_start[ti.b + 1] - st.tile1_start[ti.b]) / H;
           const SegList sl(ti.layer * st.nt1 + st.tile1_start[ti.b] + ti.h * per_head, per_head,
                            split1(st));
           const int nunits = NQ <= 128 ? 2 : 1;
-          const int ew = warp - kEpiWarp0;
           float M[8], Z[8];
 #pragma unroll
           for (int r = 0; r < 8; ++r) M[r] = -1e30f, Z[r] = 0.f;
 #pragma unroll 2
-          for (int e = ew; e < sl.nseg; e += kEpiWarps) {
+          for (int e = gw; e < sl.nseg; e += 4) {
             const int start = sl.start(e);
             for (int u = 0; u < nunits; ++u) {
               const float2* src = ws.rowstat + ((size_t)start * 2 + u) * NQ;
@@ -628,69 +632,64 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
             }
           }
 #pragma unroll
-          for (int r = 0; r < 8; ++r) part[ew * 256 + lane + 32 * r] = make_float2(M[r], Z[r]);
-          named_bar_sync(1, kEpiThreads);
-          if (et < NQ) {
+          for (int r = 0; r < 8; ++r) mypart[gw * 256 + lane + 32 * r] = make_float2(M[r], Z[r]);
+          named_bar_sync(barid, 128);
+          for (int q = gt; q < NQ; q += 128) {
             float Mx = -1e30f;
 #pragma unroll
-            for (int w = 0; w < kEpiWarps; ++w) Mx = fmaxf(Mx, part[w * 256 + et].x);
+            for (int w = 0; w < 4; ++w) Mx = fmaxf(Mx, mypart[w * 256 + q].x);
             float Zs = 0.f;
 #pragma unroll
-            for (int w = 0; w < kEpiWarps; ++w) Zs += part[w * 256 + et].y * exp2f(part[w * 256 + et].x - Mx);
-            sbq[et] = -(Mx + (log2f(Zs) + log2f((float)W)));
+            for (int w = 0; w < 4; ++w) Zs += mypart[w * 256 + q].y * exp2f(mypart[w * 256 + q].x - Mx);
+            mybq[q] = -(Mx + (log2f(Zs) + log2f((float)W)));
           }
         }
         dmin = INFINITY, dmax = -INFINITY, dsum = 0.f, exw = 0.f;
         seg_first = ti.id;
-        named_bar_sync(1, kEpiThreads);
+        named_bar_sync(barid, 128);
       }
       seg_start = ti.seg_last();
-      const int ts = it & 1, tph = (it >> 1) & 1;
-      const int ikey = ti.t * kTile + key;
-      float kinv_i = 0.f;
-      if (wg == 1 && ikey < P) kinv_i = ws.kinv[kpos(st, ti.layer, ti.h, ti.b, ikey)];
-      const bool ok = mbar_wait(&bars->tfull[ts], tph, abort);
-      tc_fence_after();
-      const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + ts * 256;
-      f32x2 acc = pack2(0.f, 0.f);
-      float dot = 0.f;
-      if (ok) {
-        uint32_t rd[4];
-        if (wg == 1) tmem_ld4(taddr + NQ, rd);
-        // 16-column chunks, the next one in flight while this one is reduced
-        uint32_t ra[16], rb[16];
-        if (nch > 0) tmem_ld16(taddr + cbeg, ra);
+      const int ts = it & 1;
+      if (ts == wg) {   // this warpgroup's tile
+        const int tph = (it >> 1) & 1;
+        const int ikey = ti.t * kTile + key;
+        float kinv_i = 0.f;
+        if (ikey < P) kinv_i = ws.kinv[kpos(st, ti.layer, ti.h, ti.b, ikey)];
+        const bool ok = mbar_wait(&bars->tfull[ts], tph, abort);
+        tc_fence_after();
+        const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + ts * 256;
+        f32x2 acc = pack2(0.f, 0.f);
+        float dot = 0.f;
+        if (ok) {
+          uint32_t rd[4];
+          tmem_ld4(taddr + NQ, rd);
+          // 16-column chunks, the next one in flight while this one is reduced
+          uint32_t ra[16], rb[16];
+          tmem_ld16(taddr, ra);
 #pragma unroll 1
-        for (int ci = 0; ci < nch; ci += 2) {   // kept rolled: the body must stay in the i-cache
-          if (ci < nch) {
+          for (int ci = 0; ci < nch; ci += 2) {   // kept rolled: the body must stay in the i-cache
             tmem_ld_wait();
             tmem_ld_fence(ra);
-            if (ci + 1 < nch) tmem_ld16(taddr + cbeg + (ci + 1) * 16, rb);
-            colsum_chunk(ra, sbq + cbeg + ci * 16, sc2, acc);
+            if (ci + 1 < nch) tmem_ld16(taddr + (ci + 1) * 16, rb);
+            colsum_chunk(ra, mybq + ci * 16, sc2, acc);
+            if (ci + 1 < nch) {
+              tmem_ld_wait();
+              tmem_ld_fence(rb);
+              if (ci + 2 < nch) tmem_ld16(taddr + (ci + 2) * 16, ra);
+              colsum_chunk(rb, mybq + (ci + 1) * 16, sc2, acc);
+            }
           }
-          if (ci + 1 < nch) {
-            tmem_ld_wait();
-            tmem_ld_fence(rb);
-            if (ci + 2 < nch) tmem_ld16(taddr + cbeg + (ci + 2) * 16, ra);
-            colsum_chunk(rb, sbq + cbeg + (ci + 1) * 16, sc2, acc);
-          }
-        }
-        if (wg == 1) {
           tmem_ld_wait();
           tmem_ld_fence(rd);
           dot = (__uint_as_float(rd[0]) + __uint_as_float(rd[1])) + __uint_as_float(rd[2]);
         }
-      }
-      tc_fence_before();
-      mbar_arrive(&bars->tempty[ts]);
-      float acc0, acc1;
-      unpack2(acc, acc0, acc1);
-      if (wg == 0) sx[ts * 128 + key] = acc0 + acc1;
-      if (group_sync_stop(1, kEpiThreads, et == 0, abort, bars->vote[0], it)) break;
-      if (wg == 1) {
-        if (ikey < P) {
+        tc_fence_before();
+        mbar_arrive(&bars->tempty[ts]);
+        if (ok && ikey < P) {
+          float acc0, acc1;
+          unpack2(acc, acc0, acc1);
           const size_t poff = ppos(st, ti.layer, ti.h, ti.b, 0);
-          const float ex = (acc0 + acc1) + sx[ts * 128 + key];
+          const float ex = acc0 + acc1;
           ws.s_ex_raw[poff + ikey] = ex;
           const float sd = -dot * kinv_i;
           s_div_out[poff + ikey] = sd;
@@ -701,24 +700,25 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
           const int cover = min(ikey, pool_half) + min(P - 1 - ikey, pool_half) + 1;
           exw = fmaf(ex, (float)cover, exw);
         }
-        if (seg_start) {
-          const float a = warp_min(dmin), b2 = warp_max(dmax), c2 = warp_sum(dsum),
-                      d2 = warp_sum(exw);
-          if (lane == 0) {
-            sred[quarter] = a;
-            sred[4 + quarter] = b2;
-            sred[8 + quarter] = c2;
-            sred[12 + quarter] = d2;
-          }
-          named_bar_sync(5, 128);
-          if (quarter == 0 && lane == 0) {
-            ws.dstat[seg_first] = make_float4(
-                fminf(fminf(sred[0], sred[1]), fminf(sred[2], sred[3])),
-                fmaxf(fmaxf(sred[4], sred[5]), fmaxf(sred[6], sred[7])),
-                (sred[8] + sred[9]) + (sred[10] + sred[11]),
-                (sred[12] + sred[13]) + (sred[14] + sred[15]));
-          }
-          named_bar_sync(5, 128);
+      }
+      if (group_sync_stop(barid, 128, gt == 0, abort, bars->vote[wg], it)) break;
+      if (seg_start) {
+        // this warpgroup's share of the segment's score statistics (neutral if it had no tile)
+        const float a = warp_min(dmin), b2 = warp_max(dmax), c2 = warp_sum(dsum),
+                    d2 = warp_sum(exw);
+        float* sr = sred + wg * 16;
+        if (lane == 0) {
+          sr[gw] = a;
+          sr[4 + gw] = b2;
+          sr[8 + gw] = c2;
+          sr[12 + gw] = d2;
+        }
+        named_bar_sync(barid, 128);
+        if (gt == 0) {
+          ws.dstat[(size_t)seg_first * 2 + wg] = make_float4(
+              fminf(fminf(sr[0], sr[1]), fminf(sr[2], sr[3])),
+              fmaxf(fmaxf(sr[4], sr[5]), fmaxf(sr[6], sr[7])),
+              (sr[8] + sr[9]) + (sr[10] + sr[11]), (sr[12] + sr[13]) + (sr[14] + sr[15]));
         }
       }
       ++it;
@@ -752,7 +752,7 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
         const bool owner = ti.t == 0;   // the CTA that holds the head's first tile publishes rbar
         if (owner) {
           const float n2 = warp_sum(s * s);
-          if (lane == 0) sred[28 + (warp - kAuxWarp0)] = n2;
+          if (lane == 0) sred[48 + (warp - kAuxWarp0)] = n2;
         }
         const float kb = s / (float)L;
         __nv_bfloat16 parts[3];
@@ -780,7 +780,7 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
         if (owner) {
           named_bar_sync(4, 128);
           if (vt == 0) {
-            const double nn = ((double)sred[28] + (double)sred[29]) + ((double)sred[30] + (double)sred[31]);
+            const double nn = ((double)sred[48] + (double)sred[49]) + ((double)sred[50] + (double)sred[51]);
             const double T = (double)L;
             const float r = (float)((nn - T) / (T * (T - 1.0)));   // Eq. 4
             ws.rbar[ti.unit()] = r;
@@ -827,21 +827,21 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
           vsum += n;
         }
       }
-      if (group_sync_stop(3, 128, vt == 0, abort, bars->vote[1], it)) break;
+      if (group_sync_stop(3, 128, vt == 0, abort, bars->vote[2], it)) break;
       if (seg_start && use_vnorm) {
         const float a = warp_min(vmin), b2 = warp_max(vmax), c2 = warp_sum(vsum);
         const int vw = warp - kAuxWarp0;
         if (lane == 0) {
-          sred[16 + vw] = a;
-          sred[20 + vw] = b2;
-          sred[24 + vw] = c2;
+          sred[32 + vw] = a;
+          sred[36 + vw] = b2;
+          sred[40 + vw] = c2;
         }
         named_bar_sync(4, 128);
         if (vt == 0) {
           ws.vstat[seg_first] = make_float4(
-              fminf(fminf(sred[16], sred[17]), fminf(sred[18], sred[19])),
-              fmaxf(fmaxf(sred[20], sred[21]), fmaxf(sred[22], sred[23])),
-              (sred[24] + sred[25]) + (sred[26] + sred[27]), 0.f);
+              fminf(fminf(sred[32], sred[33]), fminf(sred[34], sred[35])),
+              fmaxf(fmaxf(sred[36], sred[37]), fmaxf(sred[38], sred[39])),
+              (sred[40] + sred[41]) + (sred[42] + sred[43]), 0.f);
         }
         named_bar_sync(4, 128);
       }
@@ -911,8 +911,7 @@ size_t pass1_smem(int MB) {
 }
 size_t pass2_smem(int NQ, int vstages) {
   return 1024 + (size_t)2 * (NQ + kExtraRows) * 128 + kP2KStages * kTileBytes +
-         (size_t)vstages * kVSubBytes + 256 * 4 + 256 * 4 + 32 * 4 + 8 * 256 * 8 + sizeof(P2Bars) +
-         64;
+         (size_t)vstages * kVSubBytes + 512 * 4 + 64 * 4 + 8 * 256 * 8 + sizeof(P2Bars) + 64;
 }
 
 // cudaFuncSetAttribute once per (kernel, device).

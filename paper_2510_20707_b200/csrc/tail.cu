@@ -33,11 +33,11 @@ __device__ void head_scalars(const SeqTable& st, const Workspace& ws, const int 
     const SegList sl(layer * st.nt2 + st.tile2_start[b] + h * per_head, per_head, split2(st));
     for (int e = lane; e < sl.nseg; e += 32) {   // lanes take segments side by side
       const int start = sl.start(e);
-      const float4 d4 = ws.dstat[start];
-      dmin = fminf(dmin, d4.x);
-      dmax = fmaxf(dmax, d4.y);
-      dsum += d4.z;
-      exw += d4.w;
+      const float4 d4 = ws.dstat[(size_t)start * 2], e4 = ws.dstat[(size_t)start * 2 + 1];
+      dmin = fminf(dmin, fminf(d4.x, e4.x));
+      dmax = fmaxf(dmax, fmaxf(d4.y, e4.y));
+      dsum += d4.z + e4.z;
+      exw += d4.w + e4.w;
       if (use_vnorm) {
         const float4 v4 = ws.vstat[start];
         vmin = fminf(vmin, v4.x);
