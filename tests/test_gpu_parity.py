@@ -139,3 +139,48 @@ def test_layers_batched_c4_adaptive():
 def test_layers_batched_c3_c5():
     run_layers_parity(synth.CONFIGS["C3"], (3, 20))
     run_layers_parity(synth.CONFIGS["C5"], (0, 31))
+
+
+def test_bench_launch_configuration_sampled():
+    # the call bench.py times: all 28 layers of C3 in one mixkv_compress_layers call; the oracle
+    # checks three sampled layers (first, middle, last), the rest by properties that hold at any
+    # size: counts, ascending in-range indices, offsets, and the window rows at the end of
+    # every (layer, head) block being bit-exact copies
+    wl = synth.CONFIGS["C3"]
+    NL, H, W, B = wl.layers, wl.kv_heads, wl.window, wl.budget
+    L = wl.total_tokens
+    po, pg = params_pair(wl)
+    K = torch.empty((NL, H, L, 128), dtype=torch.bfloat16, device="cuda")
+    V = torch.empty_like(K)
+    Q = torch.empty((NL, 1, H * wl.gqa_ratio, W, 128), dtype=torch.bfloat16, device="cuda")
+    sampled = {}
+    for layer in range(NL):
+        x = synth.make_layer(wl, layer, "calibrated")
+        K[layer], V[layer], Q[layer] = to_dev(x["K"]), to_dev(x["V"]), to_dev(x["Q"])
+        if layer in (0, NL // 2, NL - 1):
+            sampled[layer] = x
+    out = binding.compress_layers(K, V, Q, pg)
+    torch.cuda.synchronize()
+    assert int(out["status"].item()) == 0
+    P = L - W
+    counts = out["counts"].cpu().numpy()
+    offs = out["idx_offsets"].cpu().numpy()
+    ro = out["out_row_offsets"].cpu().numpy()
+    idx = out["idx"].cpu().numpy()
+    assert (counts == B - W).all()
+    assert (offs == np.arange(H + 1) * (B - W)).all() and (ro == np.arange(H + 1) * B).all()
+    sel = idx.reshape(NL, H, B - W)
+    assert (np.diff(sel, axis=2) > 0).all() and sel.min() >= 0 and sel.max() < P
+    Ko = out["K_out"].view(NL, H, B, 128)
+    Vo = out["V_out"].view(NL, H, B, 128)
+    assert torch.equal(Ko[:, :, B - W:], K[:, :, P:]) and torch.equal(Vo[:, :, B - W:], V[:, :, P:])
+    gidx = torch.from_numpy(sel).cuda().long()[..., None].expand(-1, -1, -1, 128)
+    assert torch.equal(Ko[:, :, :B - W], torch.gather(K, 2, gidx))
+    assert torch.equal(Vo[:, :, :B - W], torch.gather(V, 2, gidx))
+    cu = wl.cu_seqlens
+    for layer, x in sampled.items():
+        ref_s = oracle.scores(x["K"], x["V"], x["Q"], po)
+        ref = oracle.select(ref_s["s_comp"], po)
+        check_scores(f"s_comp[layer {layer}]", out["s_comp"][layer].cpu().numpy(), ref_s["s_comp"],
+                     cu, W)
+        check_selection(idx[layer], offs[layer], counts[layer], ref, ref_s["s_comp"], cu, W, H)
