@@ -298,7 +298,8 @@ k_budget(const SeqTable st, const float* __restrict__ scores, int* __restrict__ 
 // ------------------------------------------------------------------------------ tail
 constexpr int kTailCluster = 8;
 constexpr int kTailThreads = 512;
-constexpr int kTailCacheCap = 16384;   // positions one CTA keeps in shared memory
+constexpr int kTailCacheCap = 16384;       // positions a CTA of a cluster keeps in shared memory
+constexpr int kTailCacheCapSolo = 40960;   // positions a CTA that owns a whole head keeps
 
 struct TailKernelArgs {
   const float* scores;        // select on these (FUSED == false)
@@ -335,20 +336,24 @@ __device__ __forceinline__ int fixed_offset(const SeqTable& st, int bh, int Bp) 
 // (thread t, t + 512, ...) and the contiguous runs of the compaction free of bank conflicts.
 __device__ __forceinline__ int kslot(int j) { return j + (j >> 5); }
 
-template <bool FUSED>
-__global__ void __launch_bounds__(kTailThreads, 2)
+// T threads per CTA; the cluster size (1 or kTailCluster CTAs per (layer, sequence, head)) is read
+// from the launch: many independent heads fill the GPU with one CTA each and need no cluster
+// traffic at all, a call with few heads spreads each head over a cluster.
+template <bool FUSED, int T>
+__global__ void __launch_bounds__(T, T == 512 ? 2 : 1)
 k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
   extern __shared__ __align__(16) unsigned char tail_smem[];
   __shared__ int hist[2][256];
-  __shared__ int s_scan[16][2];
+  __shared__ int s_scan[32][2];
   __shared__ int s_tot[2];
   __shared__ int s_sel[2];      // digit, remaining
   __shared__ int s_off;
   __shared__ float sc[8];
   cg::cluster_group cluster = cg::this_cluster();
   const int crank = (int)cluster.block_rank();
+  const int cs = (int)cluster.num_blocks();
   const int BH = st.batch * st.H;
-  const int unit = blockIdx.x / kTailCluster;          // (layer, sequence, head)
+  const int unit = blockIdx.x / cs;                    // (layer, sequence, head)
   const int layer = unit / BH, bh = unit % BH, b = bh / st.H, h = bh % st.H;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int W = st.W;
@@ -360,12 +365,12 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
   int* idx_offsets = a.idx_offsets + (size_t)layer * (BH + 1);
   int* out_row_offsets = a.out_row_offsets ? a.out_row_offsets + (size_t)layer * (BH + 1) : nullptr;
   // slice of this CTA: positions [c0, c0 + n)
-  const int chunk = (P + kTailCluster - 1) / kTailCluster;
-  const int R = (chunk + kTailThreads - 1) / kTailThreads;   // positions per thread
+  const int chunk = (P + cs - 1) / cs;
+  const int R = (chunk + T - 1) / T;   // positions per thread
   const int c0 = min(crank * chunk, P);
   const int n = min(chunk, P - c0);
   unsigned* skeys = reinterpret_cast<unsigned*>(tail_smem);            // [kslot(chunk) + 1]
-  float* sraw = reinterpret_cast<float*>(skeys + kslot(chunk) + 1);    // FUSED: staged raw scores
+  float* sraw = reinterpret_cast<float*>(skeys + kslot(chunk) + 1);    // FUSED: [8 T + 64] stage
 
   pdl_launch_dependents();
   pdl_wait();
@@ -399,66 +404,60 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
   const bool cached = FUSED || a.cached;
   float held[8];   // FUSED, R <= 8: mixed scores kept until the selection is done
   if (FUSED) {
-    // ---- pooling and mix of this slice (Eq. 2, Eq. 5), thread t takes positions t, t + 512, ...
+    // ---- pooling and mix of this slice (Eq. 2, Eq. 5) in blocks of 8 T consecutive positions:
+    // thread t takes positions t, t + T, ... of the block
     const int half = a.mp.pool_k >> 1;
-    const float pad = a.mp.pool_mode == MIXKV_POOL_AVG ? 0.f : -INFINITY;
+    const bool avg = a.mp.pool_mode == MIXKV_POOL_AVG;
+    const float pad = avg ? 0.f : -INFINITY;
+    const float invk = 1.0f / (float)a.mp.pool_k;
     if (warp == 1)
       head_scalars(st, ws, layer, b, h, a.mp.pool_k, a.mp.pool_mode, a.mp.use_vnorm, a.mp.eps,
                    a.rbar_in, lane, sc);
-    for (int t = tid; t < n + 2 * half; t += kTailThreads) {
-      const int i = c0 - half + t;
-      sraw[t] = (i >= 0 && i < P) ? ws.s_ex_raw[poff + i] : pad;
-    }
-    float vn[8], dv[8];
-    if (R <= 8) {   // issue every load of the slice before the first use
+    for (int j0 = 0; j0 < n; j0 += 8 * T) {
+      const int nb = min(8 * T, n - j0);   // positions of this block
+      __syncthreads();                     // the previous block's readers of sraw are done
+      for (int t = tid; t < nb + 2 * half; t += T) {
+        const int i = c0 + j0 - half + t;
+        sraw[t] = (i >= 0 && i < P) ? ws.s_ex_raw[poff + i] : pad;
+      }
+      float vn[8], dv[8];   // every load of the block is issued before the first use
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
-        const int j = e * kTailThreads + tid;
-        vn[e] = (a.mp.use_vnorm && j < n) ? ws.vnorm[poff + c0 + j] : 0.f;
-        dv[e] = j < n ? a.s_div[poff + c0 + j] : 0.f;
+        const int jb = e * T + tid;
+        vn[e] = (a.mp.use_vnorm && jb < nb) ? ws.vnorm[poff + c0 + j0 + jb] : 0.f;
+        dv[e] = jb < nb ? a.s_div[poff + c0 + j0 + jb] : 0.f;
       }
-    }
-    __syncthreads();
-    const float invk = 1.0f / (float)a.mp.pool_k;
-    if (R <= 8) {
+      __syncthreads();
       // the eight pooling windows advance together (same order of additions as pool_window),
       // so their shared-memory loads overlap instead of forming eight serial chains
       float ex[8];
-      const bool avg = a.mp.pool_mode == MIXKV_POOL_AVG;
 #pragma unroll
       for (int e = 0; e < 8; ++e) ex[e] = avg ? 0.f : -INFINITY;
       for (int u = 0; u < a.mp.pool_k; ++u) {
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
-          const int j = min(e * kTailThreads + tid, n - 1 > 0 ? n - 1 : 0);
-          const float w = sraw[j + u];
+          const int jb = min(e * T + tid, nb - 1);
+          const float w = sraw[jb + u];
           ex[e] = avg ? ex[e] + w : fmaxf(ex[e], w);
         }
       }
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
-        const int j = e * kTailThreads + tid;
+        const int jb = e * T + tid;
         held[e] = 0.f;
-        if (j < n) {
+        if (jb < nb) {
           held[e] = mix_one(avg ? ex[e] * invk : ex[e], vn[e], dv[e], sc, a.mp.use_vnorm,
                             a.mp.mix_mode);
-          skeys[kslot(j)] = order_key(held[e]);
+          skeys[kslot(j0 + jb)] = order_key(held[e]);
+          if (R > 8) a.s_comp_out[poff + c0 + j0 + jb] = held[e];
         }
-      }
-    } else {
-      for (int j = tid; j < n; j += kTailThreads) {
-        const float ex = pool_window(sraw + j, a.mp.pool_k, a.mp.pool_mode, invk);
-        const float v = a.mp.use_vnorm ? ws.vnorm[poff + c0 + j] : 0.f;
-        const float c = mix_one(ex, v, a.s_div[poff + c0 + j], sc, a.mp.use_vnorm, a.mp.mix_mode);
-        a.s_comp_out[poff + c0 + j] = c;
-        skeys[kslot(j)] = order_key(c);
       }
     }
     src = a.s_comp_out;
   } else if (a.cached) {
-    for (int j = tid; j < n; j += kTailThreads) skeys[kslot(j)] = order_key(src[poff + c0 + j]);
+    for (int j = tid; j < n; j += T) skeys[kslot(j)] = order_key(src[poff + c0 + j]);
   }
-  for (int t = tid; t < 256; t += kTailThreads) hist[0][t] = 0;
+  for (int t = tid; t < 256; t += T) hist[0][t] = 0;
   __syncthreads();
   const int want = s_sel[1];
   int* out = a.idx + (size_t)layer * a.idx_cap + s_off;
@@ -478,7 +477,7 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
     for (int pass = 0; pass < 4; ++pass) {
       const int shift = 24 - 8 * pass, buf = pass & 1;
       for (int e = 0; e < R; ++e) {   // same trip count in every lane: full-warp votes
-        const int j = e * kTailThreads + tid;
+        const int j = e * T + tid;
         unsigned digit = 0xffffffffu;
         if (j < n) {
           const unsigned key = key_at(j);
@@ -498,9 +497,7 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
       // every CTA adds up the cluster's histograms and finds the digit itself
       int tot = 0, incl = 0;
       if (tid < 256) {
-#pragma unroll
-        for (int r = 0; r < kTailCluster; ++r)
-          tot += *cluster.map_shared_rank(&hist[buf][tid], r);
+        for (int r = 0; r < cs; ++r) tot += *cluster.map_shared_rank(&hist[buf][tid], r);
         hist[buf ^ 1][tid] = 0;   // every CTA is past its reads of the other buffer
         // suffix sums over the 256 bins: bins above this one
         incl = tot;
@@ -555,7 +552,7 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
     __syncthreads();
     int gt_before = gt_inc - gt, eq_before = eq_inc - eq;
     for (int w = 0; w < warp; ++w) gt_before += s_scan[w][0], eq_before += s_scan[w][1];
-    if (tid == kTailThreads - 1) {
+    if (tid == T - 1) {
       s_tot[0] = gt_before + gt;
       s_tot[1] = eq_before + eq;
     }
@@ -587,7 +584,7 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
   if (FUSED && R <= 8) {
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
-      const int j = e * kTailThreads + tid;
+      const int j = e * T + tid;
       if (j < n) a.s_comp_out[poff + c0 + j] = held[e];
     }
   }
@@ -600,10 +597,10 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
     const __nv_bfloat16* Vsrc = a.V + (size_t)layer * a.kv_layer_stride;
     const size_t srow0 = (size_t)h * st.Ltot + st.cu[b];
     const size_t drow0 = (size_t)layer * a.out_rows_cap + (size_t)(s_off + bh * W);
-    const int hw = tid >> 4, l = tid & 15;                       // 32 half-warps, 16 B per lane
-    constexpr int kRowsPerSweep = kTailCluster * (kTailThreads / 16);
-    for (int rb = crank * (kTailThreads / 16) + hw; rb < rows; rb += 2 * kRowsPerSweep) {
-      const int ra = rb + kRowsPerSweep;
+    const int hw = tid >> 4, l = tid & 15;                       // half-warps, 16 B per lane
+    const int rows_per_sweep = cs * (T / 16);
+    for (int rb = crank * (T / 16) + hw; rb < rows; rb += 2 * rows_per_sweep) {
+      const int ra = rb + rows_per_sweep;
       const int sa = rb < n_sel ? __ldcg(out + rb) : P + (rb - n_sel);
       const int sb = ra < rows ? (ra < n_sel ? __ldcg(out + ra) : P + (ra - n_sel)) : -1;
       const uint4 k0 = __ldg(reinterpret_cast<const uint4*>(Ksrc + (srow0 + sa) * kHeadDim) + l);
@@ -662,9 +659,46 @@ cudaError_t launch_budget(const LaunchCtx& c, const float* scores, int* counts) 
                     c.p.budget - c.p.window, floor_slots(c.p));
 }
 
-bool tail_can_fuse(const LaunchCtx& c) {
-  const int chunk = (c.max_prefix + kTailCluster - 1) / kTailCluster;
-  return chunk <= kTailCacheCap;
+// Launch shape of k_tail: many (layer, sequence, head) units -> one 1024-thread CTA each; few ->
+// a cluster of kTailCluster 512-thread CTAs each.  Returns false when the keys of a slice do not
+// fit the shared-memory cache under either shape.
+struct TailShape {
+  int cs, threads, chunk;
+  bool cached;
+};
+
+TailShape tail_shape(const LaunchCtx& c) {
+  const int units = c.st.layers * c.st.batch * c.st.H;
+  TailShape t;
+  t.cs = 1, t.threads = 1024, t.chunk = c.max_prefix;
+  if (units >= device_sm_count() / 2 && t.chunk <= kTailCacheCapSolo) {
+    t.cached = true;
+    return t;
+  }
+  t.cs = kTailCluster, t.threads = kTailThreads;
+  t.chunk = (c.max_prefix + kTailCluster - 1) / kTailCluster;
+  t.cached = t.chunk <= kTailCacheCap;
+  return t;
+}
+
+bool tail_can_fuse(const LaunchCtx& c) { return tail_shape(c).cached; }
+
+template <bool FUSED, int T>
+cudaError_t launch_tail_t(const LaunchCtx& c, const TailKernelArgs& a, const TailShape& sh,
+                          size_t smem) {
+  static size_t have[64] = {0};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (smem > 48 * 1024 && (dev < 0 || dev >= 64 || have[dev] < smem)) {
+    const size_t ask = 216 * 1024;
+    e = cudaFuncSetAttribute(k_tail<FUSED, T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)ask);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64) have[dev] = ask;
+  }
+  const dim3 grid(c.st.layers * c.st.batch * c.st.H * sh.cs);
+  return launch_pdl(k_tail<FUSED, T>, grid, dim3(T), smem, c.stream, sh.cs, c.st, c.ws, a);
 }
 
 cudaError_t launch_tail(const LaunchCtx& c, const TailArgs& t) {
@@ -687,33 +721,16 @@ cudaError_t launch_tail(const LaunchCtx& c, const TailArgs& t) {
   a.idx_cap = c.idx_cap;
   a.out_rows_cap = c.out_rows_cap;
   a.mp = mix_params(c.p);
-  const int chunk = (c.max_prefix + kTailCluster - 1) / kTailCluster;
-  const int R = (chunk + kTailThreads - 1) / kTailThreads;
+  const TailShape sh = tail_shape(c);
   const bool fused = t.scores == nullptr;
-  a.cached = chunk <= kTailCacheCap ? 1 : 0;
+  a.cached = sh.cached ? 1 : 0;
   if (fused && !a.cached) return cudaErrorInvalidValue;   // callers check tail_can_fuse() first
-  (void)R;
   size_t smem = 0;
-  if (a.cached) smem += ((size_t)chunk + (chunk >> 5) + 1) * 4;
-  if (fused) smem += ((size_t)chunk + 64) * 4;
-  static size_t set_fused[64] = {0}, set_plain[64] = {0};
-  int dev = 0;
-  cudaError_t e = cudaGetDevice(&dev);
-  if (e != cudaSuccess) return e;
-  size_t* have = fused ? set_fused : set_plain;
-  if (smem > 48 * 1024 && (dev < 0 || dev >= 64 || have[dev] < smem)) {
-    const size_t ask = 2 * ((size_t)kTailCacheCap + 512) * 4 + 256;
-    e = fused ? cudaFuncSetAttribute(k_tail<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ask)
-              : cudaFuncSetAttribute(k_tail<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ask);
-    if (e != cudaSuccess) return e;
-    if (dev >= 0 && dev < 64) have[dev] = ask;
-  }
-  const dim3 grid(c.st.layers * c.st.batch * c.st.H * kTailCluster);
-  if (fused)
-    return launch_pdl(k_tail<true>, grid, dim3(kTailThreads), smem, c.stream, kTailCluster, c.st,
-                      c.ws, a);
-  return launch_pdl(k_tail<false>, grid, dim3(kTailThreads), smem, c.stream, kTailCluster, c.st,
-                    c.ws, a);
+  if (a.cached) smem += ((size_t)sh.chunk + (sh.chunk >> 5) + 1) * 4;
+  if (fused) smem += ((size_t)8 * sh.threads + 64) * 4;
+  if (sh.threads == 1024)
+    return fused ? launch_tail_t<true, 1024>(c, a, sh, smem) : launch_tail_t<false, 1024>(c, a, sh, smem);
+  return fused ? launch_tail_t<true, 512>(c, a, sh, smem) : launch_tail_t<false, 512>(c, a, sh, smem);
 }
 
 }  // namespace mixkv
