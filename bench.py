@@ -60,6 +60,25 @@ def peaks():
     return 6650.0, "fallback"
 
 
+def measured_traffic(workload, kernel, layers):
+    """DRAM bytes per launch of `kernel` from the committed ncu capture, scaled to `layers`
+    layers; None when there is no capture for this workload or the kernel source has changed
+    since the counters were taken."""
+    import hashlib
+    path = os.path.join(ROOT, "profiles", f"dram_traffic_{workload}.json")
+    if not os.path.exists(path):
+        return None
+    with open(path) as f:
+        rec = json.load(f)
+    try:
+        with open(os.path.join(ROOT, rec["kernel_source"]), "rb") as f:
+            if hashlib.sha256(f.read()).hexdigest() != rec["sha256"]:
+                return None
+        return rec[kernel]["dram_bytes_per_layer"] * layers
+    except (KeyError, OSError):
+        return None
+
+
 def workload_config(wl, variant, extra=None):
     cfg = {"workload": f"{wl.name}: {wl.layers} layers, H={wl.kv_heads}, G={wl.gqa_ratio}, d=128, "
                        f"batch {wl.batch}, L={list(wl.seq_lens) if wl.batch > 1 else wl.seq_lens[0]}, "
@@ -386,7 +405,8 @@ def run_mixkv(args):
                            "frac_of_8TBs_nominal": ab["layer"] / (layer_ms * 1e-3) / 8e12,
                            "algorithmic_bytes_per_layer": ab["layer"]},
         "roofline": {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak,
-                     "unit": "GB/s", "frac": achieved / peak, "traffic": None,
+                     "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": measured_traffic(wl.name, dom, NL),
                      "peak_source": f"{peak_kind} copy bandwidth",
                      "algorithmic_bytes_per_launch": NL * ab[dom],
                      "kernel_ms": dom_ms},
