@@ -156,6 +156,24 @@ def run_reference(args):
 
 
 # ------------------------------------------------------------------------------ helpers
+def max_over_ranks(ms, world, device):
+    """The step time of the whole job is the slowest rank's (replicas run side by side)."""
+    import torch
+    import torch.distributed as dist
+
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(tokens_per_replica, world, ms_per_step):
+    """KV tokens compressed per second over all replicas (weak scaling: every rank compresses
+    its own copy of the workload)."""
+    return world * tokens_per_replica / (ms_per_step * 1e-3)
+
+
+
 class ClockSampler:
     """nvidia-smi clocks / throttle reasons sampled every 200 ms while the timed region runs."""
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
@@ -316,10 +334,7 @@ def run_mixkv(args):
             run(n_warm + s)
         t1.record(stream)
         barrier()
-        t = torch.tensor([t0.elapsed_time(t1)], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item()) / n_steps
+        return max_over_ranks(t0.elapsed_time(t1), world, dev) / n_steps
 
     # ---- timed region: K steps, device-resident inputs, CUDA events on the launching stream
     for s in range(args.warmup):
@@ -333,7 +348,7 @@ def run_mixkv(args):
     ms_per_step = timed(step, 0, args.steps)
     clocks = sampler.stop() if rank == 0 else None
     check_status()
-    value = world * wl.total_tokens / (ms_per_step * 1e-3)
+    value = whole_job_value(wl.total_tokens, world, ms_per_step)
 
     # ---- per-kernel CUDA-event times: every kernel of a step bracketed by events on the
     # launching stream
