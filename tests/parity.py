@@ -135,9 +135,10 @@ def run_layer_parity(wl: synth.Workload, layer: int = 0, variant: str = "literal
 
 
 def run_layers_parity(wl: synth.Workload, layers, variant: str = "calibrated", pad_rows: int = 0,
-                      **kw):
-    """mixkv_compress_layers over several layers at once against the oracle, layer by layer.
-    pad_rows > 0 leaves a gap between the layers of K / V (a strided layer dimension)."""
+                      check=None, **kw):
+    """mixkv_compress_layers over several layers at once against the oracle, layer by layer
+    (only the positions listed in `check`, if given).  pad_rows > 0 leaves a gap between the
+    layers of K / V (a strided layer dimension)."""
     po, pg = params_pair(wl, **kw)
     cu = wl.cu_seqlens
     cu_arg = None if wl.batch == 1 else cu
@@ -159,6 +160,8 @@ def run_layers_parity(wl: synth.Workload, layers, variant: str = "calibrated", p
     torch.cuda.synchronize()
     assert int(out["status"].item()) == 0
     for n, x in enumerate(xs):
+        if check is not None and n not in check:
+            continue
         ref_s = oracle.scores(x["K"], x["V"], x["Q"], po, cu=cu_arg)
         ref = oracle.select(ref_s["s_comp"], po, cu=cu_arg)
         check_scores(f"s_comp[layer {n}]", out["s_comp"][n].cpu().numpy(), ref_s["s_comp"], cu, W)

@@ -184,3 +184,19 @@ def test_bench_launch_configuration_sampled():
         check_scores(f"s_comp[layer {layer}]", out["s_comp"][layer].cpu().numpy(), ref_s["s_comp"],
                      cu, W)
         check_selection(idx[layer], offs[layer], counts[layer], ref, ref_s["s_comp"], cu, W, H)
+
+
+def test_long_sequence_cluster_tail():
+    # 65536 keys per head: the cluster shape of the tail kernel with 16 positions per thread
+    wl = synth.small_workload(H=2, G=4, W=32, seq_lens=(65536,), pool_kernel=7, budget=512,
+                              seed=31, centroids=32)
+    run_layer_parity(wl, variant="calibrated")
+
+
+def test_many_units_long_prefix_and_widest_query_tile():
+    # 80 (layer, head) units of 45000 candidates: too long for one CTA per head, so the call
+    # falls back to clusters; G*W = 240 is the widest supported query tile
+    wl = synth.small_workload(H=2, G=15, W=16, seq_lens=(45016,), pool_kernel=5, budget=300,
+                              seed=32, centroids=16)
+    wl = synth.replace(wl, layers=40)
+    run_layers_parity(wl, range(40), check=(0, 17, 39))
