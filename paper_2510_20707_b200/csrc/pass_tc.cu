@@ -289,18 +289,13 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
         const bool need_mask = ti.t * kTile + kTile > P;
         const int lim = P + jrow;   // last key this row may see
         const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + ts * (MB * 128) + col0;
-        uint32_t ra[32], rb[32];
-        tmem_ld32(taddr, ra);
 #pragma unroll 1
-        for (int c0 = 0; c0 < NC; c0 += 64) {   // kept rolled: the body must stay in the i-cache
+        for (int c0 = 0; c0 < NC; c0 += 32) {   // kept rolled: the body must stay in the i-cache
+          uint32_t ra[32];
+          tmem_ld32(taddr + c0, ra);
           tmem_ld_wait();
           tmem_ld_fence(ra);
-          tmem_ld32(taddr + c0 + 32, rb);
           softmax_chunk(ra, need_mask, k0 + c0, lim, scale_log2e, m_run, z_run);
-          tmem_ld_wait();
-          tmem_ld_fence(rb);
-          if (c0 + 64 < NC) tmem_ld32(taddr + c0 + 64, ra);
-          softmax_chunk(rb, need_mask, k0 + c0 + 32, lim, scale_log2e, m_run, z_run);
         }
       }
       tc_fence_before();
@@ -424,11 +419,13 @@ struct P2Bars {
   int vote[3][2];
 };
 
-// Sixteen logit columns of one key: adds exp2(logit * scale - normaliser of the column).
-__device__ __forceinline__ void colsum_chunk(const uint32_t (&r)[16], const float* nb_smem,
+// N logit columns of one key (registers r[0..N)): adds exp2(logit * scale - normaliser of the
+// column) to acc; nb_smem holds the negated normalisers of these columns.
+template <int N>
+__device__ __forceinline__ void colsum_chunk(const uint32_t (&r)[N], const float* nb_smem,
                                              const f32x2 sc2, f32x2& acc) {
 #pragma unroll
-  for (int j = 0; j < 16; j += 4) {
+  for (int j = 0; j < N; j += 4) {
     const float4 nb = *reinterpret_cast<const float4*>(nb_smem + j);   // negated normalisers
     float a0, a1, b0, b1;
     unpack2(fma2(pack2(__uint_as_float(r[j]), __uint_as_float(r[j + 1])), sc2, pack2(nb.x, nb.y)),
@@ -663,21 +660,23 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
         if (ok) {
           uint32_t rd[4];
           tmem_ld4(taddr + NQ, rd);
-          // 16-column chunks, the next one in flight while this one is reduced
-          uint32_t ra[16], rb[16];
-          tmem_ld16(taddr, ra);
+          // 32-column chunks (the other warpgroup's tile keeps the SM busy while this load is
+          // in flight), then a 16-column rest; kept rolled: the body must stay in the i-cache
+          const int n32 = nch >> 1;
 #pragma unroll 1
-          for (int ci = 0; ci < nch; ci += 2) {   // kept rolled: the body must stay in the i-cache
+          for (int ci = 0; ci < n32; ++ci) {
+            uint32_t ra[32];
+            tmem_ld32(taddr + ci * 32, ra);
             tmem_ld_wait();
             tmem_ld_fence(ra);
-            if (ci + 1 < nch) tmem_ld16(taddr + (ci + 1) * 16, rb);
-            colsum_chunk(ra, mybq + ci * 16, sc2, acc);
-            if (ci + 1 < nch) {
-              tmem_ld_wait();
-              tmem_ld_fence(rb);
-              if (ci + 2 < nch) tmem_ld16(taddr + (ci + 2) * 16, ra);
-              colsum_chunk(rb, mybq + (ci + 1) * 16, sc2, acc);
-            }
+            colsum_chunk<32>(ra, mybq + ci * 32, sc2, acc);
+          }
+          if (nch & 1) {
+            uint32_t rb[16];
+            tmem_ld16(taddr + n32 * 32, rb);
+            tmem_ld_wait();
+            tmem_ld_fence(rb);
+            colsum_chunk<16>(rb, mybq + n32 * 32, sc2, acc);
           }
           tmem_ld_wait();
           tmem_ld_fence(rd);
