@@ -83,10 +83,15 @@ __device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
 constexpr size_t kSmemLimit = 227 * 1024;   // dynamic shared memory a CTA may ask for
 
 // ======================================================================== pass 1
+// Key-statistics warps (from warp 12 on): 8 for one 128-row query block, where their latency
+// chains set the pace, 4 for two blocks, where the epilogue does.  One tile = 8 pairs of 8-row
+// batches, spread evenly over the warps.
+__host__ __device__ constexpr int p1_aux_warps(int MB) { return MB == 2 ? 4 : 8; }
+__host__ __device__ constexpr int p1_threads(int MB) { return (kAuxWarp0 + p1_aux_warps(MB)) * 32; }
 constexpr int kP1MaxStages = 6;
 // K tile ring: as deep as shared memory allows next to the query tile (the deeper the ring, the
 // more bytes in flight towards HBM)
-__host__ __device__ constexpr int p1_stages(int MB) { return MB == 2 ? 5 : 6; }
+__host__ __device__ constexpr int p1_stages(int MB) { return 5; }
 
 struct P1Bars {
   uint64_t full[kP1MaxStages];
@@ -135,9 +140,9 @@ __device__ __forceinline__ void softmax_chunk(uint32_t (&r)[32], const bool need
   z_run += z0 + z1;
 }
 
-// grid = g1 persistent CTAs: TMA, MMA, 2 idle, 8 epilogue, 4 key-statistics warps.
+// grid = g1 persistent CTAs: TMA, MMA, 2 idle, 8 epilogue, 4 or 8 key-statistics warps.
 template <int MB>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(p1_threads(MB), 1)
 k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ,
         const SeqTable st, const Workspace ws, const float scale_log2e, int* status) {
   extern __shared__ unsigned char smem_dyn[];
@@ -145,10 +150,12 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
       reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
   constexpr int QR = MB * 128;                 // query rows the MMA reads
   constexpr int kP1Stages = p1_stages(MB);
+  constexpr int kP1AuxWarps = p1_aux_warps(MB);
+  constexpr int kP1Threads = p1_threads(MB);
   unsigned char* sQ = base;                    // 2 halves x [QR x 128 B]
   unsigned char* sK = sQ + 2 * QR * 128;       // kP1Stages x 32 KB
-  float* sks = reinterpret_cast<float*>(sK + kP1Stages * kTileBytes);  // [4][128] key-sum exchange
-  P1Bars* bars = reinterpret_cast<P1Bars*>(sks + 512);
+  float* sks = reinterpret_cast<float*>(sK + kP1Stages * kTileBytes);  // [aux warps][128] key-sum exchange
+  P1Bars* bars = reinterpret_cast<P1Bars*>(sks + kP1AuxWarps * 128);
   {
     // the carve-up above must fit behind the (1 KB aligned) base
     unsigned dyn;
@@ -169,7 +176,7 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
   if (tid == 0) {
     for (int s = 0; s < kP1Stages; ++s) {
       mbar_init(&bars->full[s], 1);
-      mbar_init(&bars->empty[s], 1 + 4);   // MMA commit + 4 key-statistics warps
+      mbar_init(&bars->empty[s], 1 + kP1AuxWarps);   // MMA commit + the key-statistics warps
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(&bars->tfull[s], 1);
@@ -181,7 +188,7 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
     mbar_init_fence();
   }
   // rows of the query tile beyond NQ are never loaded: clear them once
-  for (int i = tid; i < 2 * (QR - NQ) * 8; i += kThreads) {
+  for (int i = tid; i < 2 * (QR - NQ) * 8; i += kP1Threads) {
     const int half = i / ((QR - NQ) * 8), rem = i % ((QR - NQ) * 8);
     const int r = NQ + rem / 8, c = rem % 8;
     *reinterpret_cast<uint4*>(sQ + half * QR * 128 + sw128_offset(r, c)) = make_uint4(0, 0, 0, 0);
@@ -306,12 +313,16 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
     }
   } else if (warp >= kAuxWarp0) {
     // ------------------------------------------------------------------ key statistics
-    // Sixteen lanes share a key row (one 16-byte chunk each); a 16-lane group owns 16 rows of
-    // the tile.  Sweep 1 squares, a butterfly leaves the squared norm of row c with lane c,
-    // sweep 2 adds the rows scaled by 1/|k| into eight per-thread sums (dims 8c .. 8c+7).
-    const int kt = tid - kAuxWarp0 * 32;         // 0..127
-    const int grp = kt >> 4, c = kt & 15;
+    // Sixteen lanes share a key row (one 16-byte chunk each); a pair of 8-row batches is one
+    // warp-wide step (one batch per 16-lane group).  Sweep 1 squares, a butterfly leaves the
+    // squared norm of row r with lanes 2r and 2r+1, sweep 2 adds the rows scaled by 1/|k| into
+    // eight per-thread sums (dims 8c .. 8c+7).
+    const int aux_w = warp - kAuxWarp0;
+    constexpr int kPairs = 8 / kP1AuxWarps;      // pairs of 8-row batches per warp and tile
+    const int c = lane & 15, lg = lane >> 4;
     const int chalf = c >> 3, cc = c & 7;
+    constexpr int aux_threads = kP1AuxWarps * 32;
+    const int kt = tid - kAuxWarp0 * 32;
     float acc[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) acc[e] = 0.f;
@@ -328,14 +339,14 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
       const int s = it % kP1Stages, ph = (it / kP1Stages) & 1;
       const bool ok = mbar_wait(&bars->full[s], ph, abort);
       const unsigned char* tile = sK + s * kTileBytes + chalf * kHalfBytes;
-      // two batches of eight rows keep the register footprint small
 #pragma unroll 1
-      for (int bt = 0; bt < 2; ++bt) {
+      for (int bp = 0; bp < kPairs; ++bp) {   // kept rolled: the body must stay in the i-cache
+        const int row0 = (2 * (aux_w * kPairs + bp) + lg) * 8;
         uint4 u[8];
         float p[8];
 #pragma unroll
         for (int rr = 0; rr < 8; ++rr) {
-          u[rr] = *reinterpret_cast<const uint4*>(tile + sw128_offset(grp * 16 + bt * 8 + rr, cc));
+          u[rr] = *reinterpret_cast<const uint4*>(tile + sw128_offset(row0 + rr, cc));
           const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&u[rr]);
           float s0 = 0.f, s1 = 0.f;
 #pragma unroll
@@ -346,7 +357,10 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
           }
           p[rr] = s0 + s1;
         }
-        // butterfly over the 16 lanes of the group: lanes 2r and 2r+1 end with the total of row r
+        if (bp == kPairs - 1) {   // the tile now lives in registers: hand the stage back
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&bars->empty[s]);
+        }
 #pragma unroll
         for (int o = 8; o >= 2; o >>= 1) {
           const bool up = (c & o) != 0;
@@ -358,11 +372,7 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
           }
         }
         p[0] += __shfl_xor_sync(0xffffffffu, p[0], 1);
-        if (bt == 1) {   // the tile now lives in registers: hand the stage back to the producer
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&bars->empty[s]);
-        }
-        const int i = ti.t * kTile + grp * 16 + bt * 8 + (c >> 1);   // the row this lane holds
+        const int i = ti.t * kTile + row0 + (c >> 1);
         const float inv = (ok && i < L && p[0] > 0.f) ? rsqrtf(p[0]) : 0.f;
         if (i < L && (c & 1) == 0) ws.kinv[kpos(st, ti.layer, ti.h, ti.b, i)] = inv;
 #pragma unroll
@@ -377,19 +387,21 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
           }
         }
       }
-      if (group_sync_stop(2, 128, kt == 0, abort, bars->vote, it)) break;
+      if (group_sync_stop(2, aux_threads, kt == 0, abort, bars->vote, it)) break;
       if (seg_start) {
-        // fold the eight row groups: the two of a warp by shuffle, the four warps through sks
-        const int aw = warp - kAuxWarp0;
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
           const float v = acc[e] + __shfl_xor_sync(0xffffffffu, acc[e], 16);
-          if (lane < 16) sks[aw * 128 + c * 8 + e] = v;
+          if (lane < 16) sks[aux_w * 128 + c * 8 + e] = v;
         }
-        named_bar_sync(2, 128);
-        ws.ksum[(size_t)seg_first * kHeadDim + kt] =
-            (sks[kt] + sks[128 + kt]) + (sks[256 + kt] + sks[384 + kt]);
-        named_bar_sync(2, 128);
+        named_bar_sync(2, aux_threads);
+        if (kt < kHeadDim) {
+          float t = 0.f;
+#pragma unroll
+          for (int w = 0; w < kP1AuxWarps; ++w) t += sks[w * 128 + kt];
+          ws.ksum[(size_t)seg_first * kHeadDim + kt] = t;
+        }
+        named_bar_sync(2, aux_threads);
       }
       ++it;
     }
@@ -903,7 +915,7 @@ bool map_q(const LaunchCtx& c, const void* Q, CUtensorMap* tm) {
 size_t pass1_smem(int MB) {
   // up to 1023 bytes of alignment slack in front of the carve-up; never beyond the limit (the
   // kernel checks that its carve-up fits behind the aligned base)
-  const size_t need = (size_t)2 * MB * 128 * 128 + (size_t)p1_stages(MB) * kTileBytes + 512 * 4 +
+  const size_t need = (size_t)2 * MB * 128 * 128 + (size_t)p1_stages(MB) * kTileBytes + p1_aux_warps(MB) * 128 * 4 +
                       sizeof(P1Bars);
   const size_t want = need + 1024;
   return want < kSmemLimit ? want : kSmemLimit;
@@ -950,13 +962,13 @@ cudaError_t launch_pass1(const LaunchCtx& c, const void* K, const void* Q, int* 
     const size_t smem = pass1_smem(1);
     cudaError_t e = ensure_smem(k_pass1<1>, smem, done1);
     if (e != cudaSuccess) return e;
-    return launch_pdl(k_pass1<1>, dim3(c.st.g1), dim3(kThreads), smem, c.stream, 1, tmK, tmQ, c.st,
+    return launch_pdl(k_pass1<1>, dim3(c.st.g1), dim3(p1_threads(1)), smem, c.stream, 1, tmK, tmQ, c.st,
                       c.ws, c.scale_log2e, status);
   }
   const size_t smem = pass1_smem(2);
   cudaError_t e = ensure_smem(k_pass1<2>, smem, done2);
   if (e != cudaSuccess) return e;
-  return launch_pdl(k_pass1<2>, dim3(c.st.g1), dim3(kThreads), smem, c.stream, 1, tmK, tmQ, c.st,
+  return launch_pdl(k_pass1<2>, dim3(c.st.g1), dim3(p1_threads(2)), smem, c.stream, 1, tmK, tmQ, c.st,
                     c.ws, c.scale_log2e, status);
 }
 
