@@ -44,6 +44,33 @@ __device__ __forceinline__ bool group_sync_stop(int id, int n, bool leader, vola
   return slots[it & 1] != 0;
 }
 
+// Counts a delivered segment of a (layer, sequence, head) whose partial results come from
+// `nseg` CTAs; true in the CTA that delivers the last one.  Called by one thread after a CTA
+// barrier that follows the writes of the partial results: the release half of the atomic
+// publishes them, the acquire half lets the last arrival read everybody's.  The word holds
+// (tag << 16 | arrivals).  A word with another tag is left over from an earlier call, or was
+// never written, and the first arrival of this call replaces it: the caller's workspace needs
+// no clearing between calls.  Once the word carries the tag an arrival is one atomic add (no
+// retries when the CTAs of a head finish together).
+__device__ __forceinline__ bool arrive_last(unsigned long long* word, const unsigned long long tag,
+                                            const int nseg) {
+  unsigned long long cur = *reinterpret_cast<volatile unsigned long long*>(word);
+  for (;;) {
+    if ((cur >> 16) == tag) {
+      unsigned long long old;
+      asm volatile("atom.add.acq_rel.gpu.global.u64 %0, [%1], %2;"
+                   : "=l"(old)
+                   : "l"(word), "l"(1ull)
+                   : "memory");
+      return (int)((old + 1ull) & 0xffffull) == nseg;
+    }
+    __threadfence();   // release for the plain compare-and-swap below
+    const unsigned long long seen = atomicCAS(word, cur, (tag << 16) | 1ull);
+    if (seen == cur) return nseg == 1;
+    cur = seen;   // another CTA replaced the stale word first (or it changed): look again
+  }
+}
+
 __device__ __forceinline__ void raise(int* status, volatile int* abort) {
   *abort = 1;
   if (status) atomicExch(status, MIXKV_ERR_TIMEOUT);
@@ -103,7 +130,96 @@ struct P1Bars {
   uint32_t tmem_base;
   int abort;
   int vote[2];
+  int last;   // this CTA delivered the last segment of the head at hand
 };
+
+// ---- per-head folds at the end of pass 1 (once per (layer, sequence, head), in the CTA that
+// delivers the head's last segment)
+//
+// All segments' softmax (max, sum) of window row q -> minus the log2 of the row's normaliser.
+// NU partial results per segment and row.
+template <int NU>
+__device__ __forceinline__ float fold_row_stats(const float2* rowstat, const SegList& sl,
+                                                const int NQ, const int q) {
+  const int total = sl.nseg * NU;
+  float Mx = -1e30f, Zs = 0.f;
+#pragma unroll 1
+  for (int i0 = 0; i0 < total; i0 += 20) {   // twenty loads in flight
+    float2 v[20];
+#pragma unroll
+    for (int k = 0; k < 20; ++k) {
+      const int i = i0 + k;
+      v[k] = make_float2(-1e30f, 0.f);
+      if (i < total) v[k] = __ldcg(rowstat + ((size_t)sl.start(i / NU) * 2 + (i % NU)) * NQ + q);
+    }
+#pragma unroll
+    for (int k = 0; k < 20; ++k) {
+      const float mn = fmaxf(Mx, v[k].x);
+      Zs = Zs * ex2(Mx - mn) + v[k].y * ex2(v[k].x - mn);
+      Mx = mn;
+    }
+  }
+  return -(Mx + log2f(Zs));
+}
+// Sum over the head's segments of component kt of their unit-key sums.
+__device__ __forceinline__ float fold_key_sums(const float* ksum, const SegList& sl, const int kt) {
+  float sum = 0.f;
+#pragma unroll 1
+  for (int e0 = 0; e0 < sl.nseg; e0 += 20) {   // twenty loads in flight
+    float v[20];
+#pragma unroll
+    for (int e = 0; e < 20; ++e)
+      v[e] = e0 + e < sl.nseg ? __ldcg(ksum + (size_t)sl.start(e0 + e) * kHeadDim + kt) : 0.f;
+#pragma unroll
+    for (int e = 0; e < 20; ++e) sum += v[e];
+  }
+  return sum;
+}
+// Walks the segments of the CTA's tile range [lo, hi); every thread of the CTA calls it after
+// the barrier that ends the tile loops.  Threads 0 .. NQ-1 fold the row statistics, threads
+// 256 .. 383 the key sums.  `red` is shared scratch of four floats, `flag` a shared int.
+template <int MB>
+__device__ __forceinline__ void finish_heads(const SeqTable& st, const Workspace& ws, const int lo,
+                                             const int hi, const unsigned long long call_tag,
+                                             float* __restrict__ rbar_out, float* red, int* flag) {
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int NQ = st.NQ, H = st.H;
+  int id = lo;
+  while (id < hi) {
+    const TileIter ti(st.tile1_start, st.batch, H, st.nt1, id, hi);
+    const int per_head = (st.tile1_start[ti.b + 1] - st.tile1_start[ti.b]) / H;
+    const int L = st.cu[ti.b + 1] - st.cu[ti.b];
+    const int unit = ti.unit();
+    const SegList sl(ti.layer * st.nt1 + st.tile1_start[ti.b] + ti.h * per_head, per_head,
+                     split1(st));
+    if (tid == 0) *flag = arrive_last(ws.headcnt + unit, call_tag, sl.nseg);
+    __syncthreads();
+    const bool last = *flag != 0;
+    if (last) {
+      if (tid < NQ)
+        ws.bq[(size_t)unit * NQ + tid] =
+            fold_row_stats<MB == 1 ? 2 : 1>(ws.rowstat, sl, NQ, tid) - log2f((float)st.W);
+      const int kt = tid - 256;
+      float sum = 0.f;
+      if (kt >= 0 && kt < kHeadDim) {
+        sum = fold_key_sums(ws.ksum, sl, kt);
+        ws.kbar[(size_t)unit * kHeadDim + kt] = sum / (float)L;
+        const float n2 = warp_sum(sum * sum);
+        if (lane == 0) red[kt >> 5] = n2;
+      }
+    }
+    __syncthreads();   // `flag` may be rewritten; the four partial norms are in `red`
+    if (last && tid == 256) {
+      const double nn = ((double)red[0] + (double)red[1]) + ((double)red[2] + (double)red[3]);
+      const double T = (double)L;
+      const float r = (float)((nn - T) / (T * (T - 1.0)));   // Eq. 4
+      ws.rbar[unit] = r;
+      if (rbar_out) rbar_out[unit] = r;
+    }
+    __syncthreads();   // `red` is free again
+    id += min(hi - id, per_head - ti.t);
+  }
+}
 
 // One 32-column chunk of a logit row: running (max, sum) of the softmax in log2 units.
 __device__ __forceinline__ void softmax_chunk(uint32_t (&r)[32], const bool need_mask,
@@ -144,7 +260,8 @@ __device__ __forceinline__ void softmax_chunk(uint32_t (&r)[32], const bool need
 template <int MB>
 __global__ void __launch_bounds__(p1_threads(MB), 1)
 k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ,
-        const SeqTable st, const Workspace ws, const float scale_log2e, int* status) {
+        const SeqTable st, const Workspace ws, const float scale_log2e,
+        const unsigned long long call_tag, float* __restrict__ rbar_out, int* status) {
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* base =
       reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
@@ -409,7 +526,15 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
   tc_fence_before();
   __syncthreads();
   if (warp == kWarpMma) tmem_dealloc(tmem, MB * 256);
-  if (tid == 0 && bars->abort && status) atomicExch(status, MIXKV_ERR_TIMEOUT);
+  if (bars->abort) {
+    if (tid == 0 && status) atomicExch(status, MIXKV_ERR_TIMEOUT);
+    return;
+  }
+  // Every partial result of this CTA is written.  Its segments now count as delivered; the CTA
+  // that delivers the last segment of a (layer, sequence, head) folds all of them, once, into
+  // what pass 2 reads: one log2 normaliser per window row (the 1/W of the window mean folded
+  // in), the mean unit key, the redundancy of Eq. 4.
+  finish_heads<MB>(st, ws, lo, hi, call_tag, rbar_out, sks, &bars->last);
 }
 
 // ======================================================================== pass 2
@@ -454,7 +579,7 @@ __device__ __forceinline__ void colsum_chunk(const uint32_t (&r)[N], const float
 __global__ void __launch_bounds__(kThreads, 1)
 k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
         const __grid_constant__ CUtensorMap tmQ, const SeqTable st, const Workspace ws,
-        float* __restrict__ s_div_out, float* __restrict__ rbar_out, const float scale_log2e,
+        float* __restrict__ s_div_out, const float scale_log2e,
         const int use_vnorm, const int pool_half, const int vstages, int* status) {
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* base =
@@ -466,8 +591,7 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
   unsigned char* sV = sK + kP2KStages * kTileBytes;   // vstages x 16 KB
   float* sbq = reinterpret_cast<float*>(sV + vstages * kVSubBytes);  // [2][256] negated normalisers
   float* sred = sbq + 512;                    // [64]: 2 x 16 epilogue, 16 value norms + 4 mean key
-  float2* part = reinterpret_cast<float2*>(sred + 64);   // [2][4][256] per-warp row statistics
-  P2Bars* bars = reinterpret_cast<P2Bars*>(part + 8 * 256);
+  P2Bars* bars = reinterpret_cast<P2Bars*>(sred + 64);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int lo = cta_first_tile(blockIdx.x, split2(st));
@@ -594,15 +718,14 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
     // ------------------------------------------------------------------ epilogue
     // The two warpgroups take alternate tiles (warpgroup g owns accumulator stage g), one key
     // per thread and all G*W columns of it, so a tile needs no exchange between warpgroups and
-    // the groups never wait for each other: each folds the segment's row statistics into its
-    // own normaliser table and leaves its own partial score statistics.
+    // the groups never wait for each other: each keeps its own copy of the normaliser table
+    // and leaves its own partial score statistics.
     const int quarter = warp & 3, wg = (warp - kEpiWarp0) >> 2;
     const int gt = (tid - kEpiWarp0 * 32) & 127;   // thread inside the warpgroup
     const int gw = gt >> 5;                        // warp inside the warpgroup
     const int key = quarter * 32 + lane;
     const int nch = NQ / 16;
     float* mybq = sbq + wg * 256;
-    float2* mypart = part + wg * 4 * 256;
     const int barid = 1 + wg;                      // named barriers 1, 2: one per warpgroup
     const f32x2 sc2 = pack2(scale_log2e, scale_log2e);
     float dmin = INFINITY, dmax = -INFINITY, dsum = 0.f, exw = 0.f;
@@ -611,48 +734,9 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
     for (TileIter ti(st.tile2_start, st.batch, H, st.nt2, lo, hi); ti.valid(); ti.next()) {
       const int L = st.cu[ti.b + 1] - st.cu[ti.b], P = L - W;
       if (seg_start) {
-        // fold pass 1's per-segment softmax statistics of this (layer, b, h) into one log2
-        // normaliser per window row (the 1/W of the window mean folded in); the four warps
-        // take segments side by side
-        named_bar_sync(barid, 128);   // the previous segment's readers of mybq / mypart are done
-        {
-          const int per_head = (st.tile1_start[ti.b + 1] - st.tile1_start[ti.b]) / H;
-          const SegList sl(ti.layer * st.nt1 + st.tile1_start[ti.b] + ti.h * per_head, per_head,
-                           split1(st));
-          const int nunits = NQ <= 128 ? 2 : 1;
-          float M[8], Z[8];
-#pragma unroll
-          for (int r = 0; r < 8; ++r) M[r] = -1e30f, Z[r] = 0.f;
-#pragma unroll 2
-          for (int e = gw; e < sl.nseg; e += 4) {
-            const int start = sl.start(e);
-            for (int u = 0; u < nunits; ++u) {
-              const float2* src = ws.rowstat + ((size_t)start * 2 + u) * NQ;
-#pragma unroll
-              for (int r = 0; r < 8; ++r) {
-                const int q = lane + 32 * r;
-                if (q < NQ) {
-                  const float2 mz = src[q];
-                  const float mn = fmaxf(M[r], mz.x);
-                  Z[r] = Z[r] * ex2(M[r] - mn) + mz.y * ex2(mz.x - mn);
-                  M[r] = mn;
-                }
-              }
-            }
-          }
-#pragma unroll
-          for (int r = 0; r < 8; ++r) mypart[gw * 256 + lane + 32 * r] = make_float2(M[r], Z[r]);
-          named_bar_sync(barid, 128);
-          for (int q = gt; q < NQ; q += 128) {
-            float Mx = -1e30f;
-#pragma unroll
-            for (int w = 0; w < 4; ++w) Mx = fmaxf(Mx, mypart[w * 256 + q].x);
-            float Zs = 0.f;
-#pragma unroll
-            for (int w = 0; w < 4; ++w) Zs += mypart[w * 256 + q].y * exp2f(mypart[w * 256 + q].x - Mx);
-            mybq[q] = -(Mx + (log2f(Zs) + log2f((float)W)));
-          }
-        }
+        // pass 1 left one negated log2 normaliser per window row of this (layer, b, h)
+        named_bar_sync(barid, 128);   // the previous segment's readers of mybq are done
+        for (int q = gt; q < NQ; q += 128) mybq[q] = ws.bq[(size_t)ti.unit() * NQ + q];
         dmin = INFINITY, dmax = -INFINITY, dsum = 0.f, exw = 0.f;
         seg_first = ti.id;
         named_bar_sync(barid, 128);
@@ -736,9 +820,8 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
     }
   } else if (warp >= kAuxWarp0) {
     // ------------------------------------------------------------------ mean key, value norms
-    // At the start of a segment: fold pass 1's unit-key sums of this (b, h) into the mean unit
-    // key, write its bf16 hi / lo / lo2 split into the three extra B rows and (once per head)
-    // publish the redundancy of Eq. 4.  Per tile: warps 12, 13 read the first 64 rows of the V
+    // At the start of a segment: write the bf16 hi / lo / lo2 split of the head's mean unit key
+    // (pass 1) into the three extra B rows.  Per tile: warps 12, 13 read the first 64 rows of the V
     // tile, warps 14, 15 the last 64; one row per thread from the swizzled half tile.
     const int vt = tid - kAuxWarp0 * 32;         // 0..127
     const int sub = vt >> 6, vr = vt & 63;
@@ -747,25 +830,7 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
     bool seg_start = true;
     for (TileIter ti(st.tile2_start, st.batch, H, st.nt2, lo, hi); ti.valid(); ti.next()) {
       if (seg_start) {
-        const int L = st.cu[ti.b + 1] - st.cu[ti.b];
-        const int per_head = (st.tile1_start[ti.b + 1] - st.tile1_start[ti.b]) / H;
-        const SegList sl(ti.layer * st.nt1 + st.tile1_start[ti.b] + ti.h * per_head, per_head,
-                           split1(st));
-        float s = 0.f;
-        for (int e0 = 0; e0 < sl.nseg; e0 += 16) {   // sixteen loads in flight per thread
-          float v[16];
-#pragma unroll
-          for (int e = 0; e < 16; ++e)
-            v[e] = e0 + e < sl.nseg ? ws.ksum[(size_t)sl.start(e0 + e) * kHeadDim + vt] : 0.f;
-#pragma unroll
-          for (int e = 0; e < 16; ++e) s += v[e];
-        }
-        const bool owner = ti.t == 0;   // the CTA that holds the head's first tile publishes rbar
-        if (owner) {
-          const float n2 = warp_sum(s * s);
-          if (lane == 0) sred[48 + (warp - kAuxWarp0)] = n2;
-        }
-        const float kb = s / (float)L;
+        const float kb = ws.kbar[(size_t)ti.unit() * kHeadDim + vt];   // mean unit key (pass 1)
         __nv_bfloat16 parts[3];
         parts[0] = __float2bfloat16_rn(kb);
         const float r1 = kb - __bfloat162float(parts[0]);
@@ -788,16 +853,6 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) mbar_arrive(&bars->kbready);
-        if (owner) {
-          named_bar_sync(4, 128);
-          if (vt == 0) {
-            const double nn = ((double)sred[48] + (double)sred[49]) + ((double)sred[50] + (double)sred[51]);
-            const double T = (double)L;
-            const float r = (float)((nn - T) / (T * (T - 1.0)));   // Eq. 4
-            ws.rbar[ti.unit()] = r;
-            if (rbar_out) rbar_out[ti.unit()] = r;
-          }
-        }
         ++segn;
         vmin = INFINITY, vmax = -INFINITY, vsum = 0.f;
         seg_first = ti.id;
@@ -922,7 +977,7 @@ size_t pass1_smem(int MB) {
 }
 size_t pass2_smem(int NQ, int vstages) {
   return 1024 + (size_t)2 * (NQ + kExtraRows) * 128 + kP2KStages * kTileBytes +
-         (size_t)vstages * kVSubBytes + 512 * 4 + 64 * 4 + 8 * 256 * 8 + sizeof(P2Bars) + 64;
+         (size_t)vstages * kVSubBytes + 512 * 4 + 64 * 4 + sizeof(P2Bars) + 64;
 }
 
 // cudaFuncSetAttribute once per (kernel, device).
@@ -954,7 +1009,8 @@ int device_sm_count() {
   return cached[dev];
 }
 
-cudaError_t launch_pass1(const LaunchCtx& c, const void* K, const void* Q, int* status) {
+cudaError_t launch_pass1(const LaunchCtx& c, const void* K, const void* Q, float* rbar_out,
+                         int* status) {
   CUtensorMap tmK, tmQ;
   if (!map_kv(c, K, kTile, &tmK) || !map_q(c, Q, &tmQ)) return cudaErrorInvalidValue;
   static bool done1[64] = {false}, done2[64] = {false};
@@ -963,17 +1019,17 @@ cudaError_t launch_pass1(const LaunchCtx& c, const void* K, const void* Q, int* 
     cudaError_t e = ensure_smem(k_pass1<1>, smem, done1);
     if (e != cudaSuccess) return e;
     return launch_pdl(k_pass1<1>, dim3(c.st.g1), dim3(p1_threads(1)), smem, c.stream, 1, tmK, tmQ, c.st,
-                      c.ws, c.scale_log2e, status);
+                      c.ws, c.scale_log2e, c.call_tag, rbar_out, status);
   }
   const size_t smem = pass1_smem(2);
   cudaError_t e = ensure_smem(k_pass1<2>, smem, done2);
   if (e != cudaSuccess) return e;
   return launch_pdl(k_pass1<2>, dim3(c.st.g1), dim3(p1_threads(2)), smem, c.stream, 1, tmK, tmQ, c.st,
-                    c.ws, c.scale_log2e, status);
+                    c.ws, c.scale_log2e, c.call_tag, rbar_out, status);
 }
 
 cudaError_t launch_pass2(const LaunchCtx& c, const void* K, const void* V, const void* Q,
-                         float* s_div_out, float* rbar_out, int* status) {
+                         float* s_div_out, int* status) {
   CUtensorMap tmK, tmV, tmQ;
   const void* Vsrc = c.p.use_vnorm ? V : K;   // the V map is never used without VNorm
   if (!map_kv(c, K, kTile, &tmK) || !map_kv(c, Vsrc, 64, &tmV) || !map_q(c, Q, &tmQ))
@@ -985,7 +1041,7 @@ cudaError_t launch_pass2(const LaunchCtx& c, const void* K, const void* V, const
   while (vstages > 2 && pass2_smem(c.st.NQ, vstages) > kSmemLimit) --vstages;
   const size_t smem = pass2_smem(c.st.NQ, vstages);
   return launch_pdl(k_pass2, dim3(c.st.g2), dim3(kThreads), smem, c.stream, 1, tmK, tmV, tmQ, c.st,
-                    c.ws, s_div_out, rbar_out, c.scale_log2e, c.p.use_vnorm, c.p.pool_kernel >> 1,
+                    c.ws, s_div_out, c.scale_log2e, c.p.use_vnorm, c.p.pool_kernel >> 1,
                     vstages, status);
 }
 

@@ -28,21 +28,36 @@ __device__ void head_scalars(const SeqTable& st, const Workspace& ws, const int 
   const int P = st.cu[b + 1] - st.cu[b] - st.W;
   float dmin = INFINITY, dmax = -INFINITY, dsum = 0.f, exw = 0.f;
   float vmin = INFINITY, vmax = -INFINITY, vsum = 0.f;
+  float rbar = 0.f;
+  if (lane == 0) rbar = rbar_in ? rbar_in[unit] : ws.rbar[unit];
   {
     const int per_head = (st.tile2_start[b + 1] - st.tile2_start[b]) / st.H;
     const SegList sl(layer * st.nt2 + st.tile2_start[b] + h * per_head, per_head, split2(st));
-    for (int e = lane; e < sl.nseg; e += 32) {   // lanes take segments side by side
-      const int start = sl.start(e);
-      const float4 d4 = ws.dstat[(size_t)start * 2], e4 = ws.dstat[(size_t)start * 2 + 1];
-      dmin = fminf(dmin, fminf(d4.x, e4.x));
-      dmax = fmaxf(dmax, fmaxf(d4.y, e4.y));
-      dsum += d4.z + e4.z;
-      exw += d4.w + e4.w;
-      if (use_vnorm) {
-        const float4 v4 = ws.vstat[start];
-        vmin = fminf(vmin, v4.x);
-        vmax = fmaxf(vmax, v4.y);
-        vsum += v4.z;
+    // lanes take segments side by side, two per lane and round; all loads of a round are
+    // issued before the first is used
+    for (int e0 = lane; e0 < sl.nseg; e0 += 64) {
+      float4 d4[2], e4[2], v4[2];
+#pragma unroll
+      for (int k = 0; k < 2; ++k) {
+        const int e = e0 + 32 * k;
+        d4[k] = e4[k] = make_float4(INFINITY, -INFINITY, 0.f, 0.f);
+        v4[k] = d4[k];
+        if (e < sl.nseg) {
+          const int start = sl.start(e);
+          d4[k] = ws.dstat[(size_t)start * 2];
+          e4[k] = ws.dstat[(size_t)start * 2 + 1];
+          if (use_vnorm) v4[k] = ws.vstat[start];
+        }
+      }
+#pragma unroll
+      for (int k = 0; k < 2; ++k) {
+        dmin = fminf(dmin, fminf(d4[k].x, e4[k].x));
+        dmax = fmaxf(dmax, fmaxf(d4[k].y, e4[k].y));
+        dsum += d4[k].z + e4[k].z;
+        exw += d4[k].w + e4[k].w;
+        vmin = fminf(vmin, v4[k].x);
+        vmax = fmaxf(vmax, v4[k].y);
+        vsum += v4[k].z;
       }
     }
   }
@@ -81,7 +96,7 @@ __device__ void head_scalars(const SeqTable& st, const Workspace& ws, const int 
     sc[1] = cin;
     sc[2] = dmin;
     sc[3] = dinv * a_div;
-    sc[4] = rbar_in ? rbar_in[unit] : ws.rbar[unit];
+    sc[4] = rbar;
   }
 }
 
@@ -345,7 +360,7 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
   extern __shared__ __align__(16) unsigned char tail_smem[];
   __shared__ int hist[2][256];
   __shared__ int s_scan[32][2];
-  __shared__ int s_tot[2];
+  __shared__ __align__(8) int s_tot[2];
   __shared__ int s_sel[2];      // digit, remaining
   __shared__ int s_off;
   __shared__ float sc[8];
@@ -416,16 +431,25 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
     for (int j0 = 0; j0 < n; j0 += 8 * T) {
       const int nb = min(8 * T, n - j0);   // positions of this block
       __syncthreads();                     // the previous block's readers of sraw are done
-      for (int t = tid; t < nb + 2 * half; t += T) {
-        const int i = c0 + j0 - half + t;
-        sraw[t] = (i >= 0 && i < P) ? ws.s_ex_raw[poff + i] : pad;
+      // every load of the block is issued before the first use; the block and its pooling halo
+      // (62 positions at most) are nine rounds of T raw scores
+      float raw[9], vn[8], dv[8];
+      const int nstage = nb + 2 * half;
+#pragma unroll
+      for (int e = 0; e < 9; ++e) {
+        const int t = e * T + tid, i = c0 + j0 - half + t;
+        raw[e] = (t < nstage && i >= 0 && i < P) ? ws.s_ex_raw[poff + i] : pad;
       }
-      float vn[8], dv[8];   // every load of the block is issued before the first use
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
         const int jb = e * T + tid;
         vn[e] = (a.mp.use_vnorm && jb < nb) ? ws.vnorm[poff + c0 + j0 + jb] : 0.f;
         dv[e] = jb < nb ? a.s_div[poff + c0 + j0 + jb] : 0.f;
+      }
+#pragma unroll
+      for (int e = 0; e < 9; ++e) {
+        const int t = e * T + tid;
+        if (t < nstage) sraw[t] = raw[e];
       }
       __syncthreads();
       // the eight pooling windows advance together (same order of additions as pool_window),
@@ -474,30 +498,59 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
     // ---- threshold: the want-th largest key of the head, four 8-bit digit passes
     unsigned prefix = 0, mask = 0;
     int remaining = want;
+    // up to eight keys per thread stay in registers for the four passes; their votes are
+    // independent, so the eight chains of a pass overlap
+    const bool inreg = cached && R <= 8;
+    unsigned rk[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const int j = e * T + tid;
+      rk[e] = (inreg && j < n) ? skeys[kslot(j)] : 0u;
+    }
+    // one warp-wide count of a digit: most warps see one digit only (always in the first
+    // passes): one vote, one add
+    auto count_digit = [&](const unsigned digit, const int buf) {
+      const unsigned first = __shfl_sync(0xffffffffu, digit, 0);
+      if (__all_sync(0xffffffffu, digit == first)) {
+        if (lane == 0 && digit != 0xffffffffu) atomicAdd(&hist[buf][digit], 32);
+      } else {
+        const unsigned peers = __match_any_sync(0xffffffffu, digit);
+        if (digit != 0xffffffffu && (int)(__ffs(peers) - 1) == lane)
+          atomicAdd(&hist[buf][digit], __popc(peers));
+      }
+    };
     for (int pass = 0; pass < 4; ++pass) {
       const int shift = 24 - 8 * pass, buf = pass & 1;
-      for (int e = 0; e < R; ++e) {   // same trip count in every lane: full-warp votes
-        const int j = e * T + tid;
-        unsigned digit = 0xffffffffu;
-        if (j < n) {
-          const unsigned key = key_at(j);
-          if ((key & mask) == prefix) digit = (key >> shift) & 255u;
-        }
-        // most warps see one digit only (always in the first passes): one vote, one add
-        const unsigned first = __shfl_sync(0xffffffffu, digit, 0);
-        if (__all_sync(0xffffffffu, digit == first)) {
-          if (lane == 0 && digit != 0xffffffffu) atomicAdd(&hist[buf][digit], 32);
-        } else {
-          const unsigned peers = __match_any_sync(0xffffffffu, digit);
-          if (digit != 0xffffffffu && (int)(__ffs(peers) - 1) == lane)
-            atomicAdd(&hist[buf][digit], __popc(peers));
+      if (inreg) {
+        unsigned dg[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e)
+          dg[e] = (e * T + tid < n && (rk[e] & mask) == prefix) ? (rk[e] >> shift) & 255u
+                                                                : 0xffffffffu;
+#pragma unroll
+        for (int e = 0; e < 8; ++e)
+          if (e < R) count_digit(dg[e], buf);   // R is the same in every thread
+      } else {
+        for (int e = 0; e < R; ++e) {   // same trip count in every lane: full-warp votes
+          const int j = e * T + tid;
+          unsigned digit = 0xffffffffu;
+          if (j < n) {
+            const unsigned key = key_at(j);
+            if ((key & mask) == prefix) digit = (key >> shift) & 255u;
+          }
+          count_digit(digit, buf);
         }
       }
       cluster.sync();
       // every CTA adds up the cluster's histograms and finds the digit itself
       int tot = 0, incl = 0;
       if (tid < 256) {
-        for (int r = 0; r < cs; ++r) tot += *cluster.map_shared_rank(&hist[buf][tid], r);
+        int part[kTailCluster];
+#pragma unroll
+        for (int r = 0; r < kTailCluster; ++r)
+          part[r] = r < cs ? *cluster.map_shared_rank(&hist[buf][tid], r) : 0;
+#pragma unroll
+        for (int r = 0; r < kTailCluster; ++r) tot += part[r];
         hist[buf ^ 1][tid] = 0;   // every CTA is past its reads of the other buffer
         // suffix sums over the 256 bins: bins above this one
         incl = tot;
@@ -557,10 +610,14 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
       s_tot[1] = eq_before + eq;
     }
     cluster.sync();
-    for (int r = 0; r < crank; ++r) {
-      const int* t = cluster.map_shared_rank(&s_tot[0], r);
-      gt_before += t[0];
-      eq_before += t[1];
+    {
+      int2 before[kTailCluster];
+#pragma unroll
+      for (int r = 0; r < kTailCluster; ++r)
+        before[r] = r < crank ? *reinterpret_cast<const int2*>(cluster.map_shared_rank(&s_tot[0], r))
+                              : make_int2(0, 0);
+#pragma unroll
+      for (int r = 0; r < kTailCluster; ++r) gt_before += before[r].x, eq_before += before[r].y;
     }
     for (int j = r0; j < r1; ++j) {
       const int i = c0 + j;

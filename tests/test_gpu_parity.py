@@ -200,3 +200,47 @@ def test_many_units_long_prefix_and_widest_query_tile():
                               seed=32, centroids=16)
     wl = synth.replace(wl, layers=40)
     run_layers_parity(wl, range(40), check=(0, 17, 39))
+
+
+def test_workspace_needs_no_clearing():
+    # Pass 1 counts delivered segments in the caller's workspace under a per-call tag: whatever
+    # the workspace holds (all ones, all zeros, random bytes, the counters of an earlier call
+    # on another shape) the results are bit-identical.
+    wl = synth.small_workload(H=3, G=4, W=16, seq_lens=(3000, 1500), pool_kernel=5, budget=96,
+                              seed=41, centroids=8)
+    x = synth.make_layer(wl, 0, "calibrated")
+    _, pg = params_pair(wl)
+    K, V, Q = to_dev(x["K"]), to_dev(x["V"]), to_dev(x["Q"])
+    cu = [int(c) for c in wl.cu_seqlens]
+    nbytes = binding.workspace_size(pg, wl.batch, wl.total_tokens, max(wl.seq_lens))
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    gen = torch.Generator(device="cuda").manual_seed(5)
+    results = []
+    for fill in ("ones", "zeros", "random", "reuse", "other-shape-first"):
+        if fill == "ones":
+            ws.fill_(255)
+        elif fill == "zeros":
+            ws.zero_()
+        elif fill == "random":
+            ws.copy_(torch.randint(0, 256, (nbytes,), dtype=torch.uint8, device="cuda",
+                                   generator=gen))
+        elif fill == "other-shape-first":
+            wl2 = synth.small_workload(H=3, G=4, W=16, seq_lens=(700,), pool_kernel=5, budget=96,
+                                       seed=42, centroids=8)
+            x2 = synth.make_layer(wl2, 0, "literal")
+            o2 = binding.compress_layer(to_dev(x2["K"]), to_dev(x2["V"]), to_dev(x2["Q"]), pg,
+                                        workspace=ws)
+            assert int(o2["status"].item()) == 0
+        out = binding.compress_layer(K, V, Q, pg, cu_seqlens=cu, workspace=ws)
+        torch.cuda.synchronize()
+        assert int(out["status"].item()) == 0
+        results.append(out)
+    first = results[0]
+    n_rows = int(first["out_row_offsets"][-1].item())
+    for out in results[1:]:
+        for key in ("s_comp", "idx_offsets", "counts", "out_row_offsets"):
+            assert torch.equal(first[key], out[key]), key
+        n_idx = int(first["idx_offsets"][-1].item())
+        assert torch.equal(first["idx"][:n_idx], out["idx"][:n_idx])
+        assert torch.equal(first["K_out"][:n_rows].view(torch.int16), out["K_out"][:n_rows].view(torch.int16))
+        assert torch.equal(first["V_out"][:n_rows].view(torch.int16), out["V_out"][:n_rows].view(torch.int16))
