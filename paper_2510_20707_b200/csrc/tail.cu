@@ -211,57 +211,110 @@ __device__ __forceinline__ unsigned order_key(float f) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-// Finds the key of the `want`-th largest element (1-based) among n_rows rows of `len` floats
-// (row r at base + r*stride) and how many elements equal to it are still needed.  Four
-// 8-bit digit passes, most significant first; all threads of the CTA take part.
-// hist: 256 ints of shared memory.  Returns through tau / need_eq (same in every thread).
-__device__ void radix_threshold(const float* base, size_t stride, int n_rows, int len, int want,
-                                int* hist, unsigned* tau, int* need_eq) {
-  __shared__ unsigned s_prefix;
+// Adds the 32 digits of a warp (0xffffffff = none) to a shared-memory histogram.  The digit of
+// the lowest lane, then the digit of the lowest lane left, are counted with one vote and one add
+// each (the first passes of a selection see one or two digits almost everywhere); what is left
+// after that is spread over the bins and is added lane by lane.
+__device__ __forceinline__ void count_digits(int* hist, const unsigned digit, const int lane) {
+  unsigned left = 0xffffffffu;
+#pragma unroll
+  for (int round = 0; round < 2; ++round) {
+    const int src = __ffs(left) - 1;                       // lowest lane not counted yet
+    const unsigned d = __shfl_sync(0xffffffffu, digit, src);
+    const unsigned same = __ballot_sync(0xffffffffu, digit == d) & left;
+    if (lane == src && d != 0xffffffffu) atomicAdd(&hist[d], __popc(same));
+    left &= ~same;
+    if (left == 0) return;                                 // uniform across the warp
+  }
+  if (((left >> lane) & 1u) && digit != 0xffffffffu) atomicAdd(&hist[digit], 1);
+}
+
+// Threshold of the `want` largest of `total` keys: the want-th largest key and how many keys
+// equal to it are still needed.  All threads of the CTA take part.  A first sweep finds the
+// smallest and the largest key: the bits they share are the same in every key and are skipped,
+// so the first digit pass already sees digits that differ (scores of one sequence share sign
+// and most of the exponent; counting those bits would send every warp to the same one or two
+// bins).  Then digit passes of up to 8 bits, most significant first.  key_at(e) gives key e
+// (any order).  hist: 256 ints of shared memory.  Returns through tau / need_eq (same in every
+// thread).
+template <typename KeyAt>
+__device__ __forceinline__ void radix_threshold(const KeyAt& key_at, const int total, const int want,
+                                                int* hist, unsigned* tau, int* need_eq) {
+  __shared__ unsigned s_prefix, s_lo[32], s_hi[32];
   __shared__ int s_remaining;
-  unsigned prefix = 0, mask = 0;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = (blockDim.x + 31) >> 5;
+  unsigned lo = 0xffffffffu, hi = 0u;
+  for (int e = threadIdx.x; e < total; e += blockDim.x) {
+    const unsigned key = key_at(e);
+    lo = min(lo, key);
+    hi = max(hi, key);
+  }
+  lo = __reduce_min_sync(0xffffffffu, lo);
+  hi = __reduce_max_sync(0xffffffffu, hi);
+  if (lane == 0) s_lo[warp] = lo, s_hi[warp] = hi;
+  __syncthreads();
+  for (int w = 0; w < nwarps; ++w) lo = min(lo, s_lo[w]), hi = max(hi, s_hi[w]);
+  const unsigned diff = lo ^ hi;
+  int top = diff ? 32 - __clz(diff) : 0;   // the low `top` bits differ between keys
+  unsigned mask = top == 32 ? 0u : ~((1u << top) - 1u);
+  unsigned prefix = hi & mask;
   int remaining = want;
-  for (int shift = 24; shift >= 0; shift -= 8) {
+  while (top > 0) {
+    const int bits = min(8, top), shift = top - bits;
+    const unsigned dmask = (1u << bits) - 1u;
     for (int t = threadIdx.x; t < 256; t += blockDim.x) hist[t] = 0;
+    if (threadIdx.x == 0) s_prefix = prefix, s_remaining = remaining;
     __syncthreads();
-    for (int r = 0; r < n_rows; ++r) {
-      const float* row = base + (size_t)r * stride;
-      for (int i0 = 0; i0 < len; i0 += blockDim.x) {   // uniform trip count: full-warp votes
-        const int i = i0 + threadIdx.x;
-        unsigned digit = 0xffffffffu;
-        if (i < len) {
-          const unsigned key = order_key(row[i]);
-          if ((key & mask) == prefix) digit = (key >> shift) & 255u;
-        }
-        const unsigned peers = __match_any_sync(0xffffffffu, digit);
-        if (digit != 0xffffffffu && (int)(__ffs(peers) - 1) == (int)(threadIdx.x & 31))
-          atomicAdd(&hist[digit], __popc(peers));
+    for (int e0 = 0; e0 < total; e0 += blockDim.x) {   // uniform trip count: full-warp votes
+      const int e = e0 + threadIdx.x;
+      unsigned digit = 0xffffffffu;
+      if (e < total) {
+        const unsigned key = key_at(e);
+        if ((key & mask) == prefix) digit = (key >> shift) & dmask;
       }
+      count_digits(hist, digit, lane);
     }
     __syncthreads();
-    if (threadIdx.x == 0) {
-      int cum = 0, d = 255;
-      for (; d > 0; --d) {
-        if (cum + hist[d] >= remaining) break;
-        cum += hist[d];
+    if (threadIdx.x < 32) {
+      // lane l owns bins 8l .. 8l+7; `above` = keys in higher bins
+      int h8[8], mine = 0;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) h8[k] = hist[8 * lane + k], mine += h8[k];
+      // suffix sum over lanes: keys in the bins of higher lanes
+      int incl = mine;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_down_sync(0xffffffffu, incl, o);
+        if (lane + o < 32) incl += v;
       }
-      s_prefix = prefix | ((unsigned)d << shift);
-      s_remaining = remaining - cum;
+      int above = incl - mine;
+#pragma unroll
+      for (int k = 7; k >= 0; --k) {
+        if (above < remaining && remaining <= above + h8[k]) {
+          s_prefix = prefix | ((unsigned)(8 * lane + k) << shift);
+          s_remaining = remaining - above;
+        }
+        above += h8[k];
+      }
     }
     __syncthreads();
     prefix = s_prefix;
     remaining = s_remaining;
-    mask |= 255u << shift;
+    mask |= dmask << shift;
+    top = shift;
     __syncthreads();
   }
   *tau = prefix;
   *need_eq = remaining;
 }
 
-// Head budgets of one sequence under the adaptive rule (see mixkv.h).
+// Head budgets of one sequence under the adaptive rule (see mixkv.h).  The H * P pooled scores
+// of the sequence are turned into order-preserving keys once and kept in shared memory when
+// they fit (cache_cap keys); otherwise every pass reads them from global memory.
 __global__ void __launch_bounds__(1024)
 k_budget(const SeqTable st, const float* __restrict__ scores, int* __restrict__ counts,
-         const int Bp, const int floor_slots) {
+         const int Bp, const int floor_slots, const int cache_cap) {
+  extern __shared__ unsigned bkeys[];
   __shared__ int hist[256];
   __shared__ int s_gt[64], s_eq[64];
   pdl_launch_dependents();
@@ -273,20 +326,45 @@ k_budget(const SeqTable st, const float* __restrict__ scores, int* __restrict__ 
   long long N = (long long)H * (Bp - floor_slots);
   if (N > total) N = total;
   const float* base = scores + ppos(st, layer, 0, b, 0);
+  const size_t stride = (size_t)st.Ptot;
   if (N <= 0) {
     for (int h = threadIdx.x; h < H; h += blockDim.x) counts[b * H + h] = min(floor_slots, P);
     return;
   }
+  const bool cached = total <= (long long)cache_cap;
+  if (cached) {
+    for (int h = 0; h < H; ++h) {
+      const float* row = base + (size_t)h * stride;
+      for (int i0 = 0; i0 < P; i0 += 8 * blockDim.x) {   // eight loads in flight per thread
+        float v[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const int i = i0 + k * blockDim.x + threadIdx.x;
+          v[k] = i < P ? row[i] : 0.f;
+        }
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const int i = i0 + k * blockDim.x + threadIdx.x;
+          if (i < P) bkeys[h * P + i] = order_key(v[k]);
+        }
+      }
+    }
+    __syncthreads();
+  }
+  auto key_at = [&](const int e) -> unsigned {
+    if (cached) return bkeys[e];
+    const int h = e / P;
+    return order_key(base[(size_t)h * stride + (e - h * P)]);
+  };
   unsigned tau;
   int need_eq;
-  radix_threshold(base, (size_t)st.Ptot, H, P, (int)N, hist, &tau, &need_eq);
+  radix_threshold(key_at, (int)total, (int)N, hist, &tau, &need_eq);
   for (int h = threadIdx.x; h < H; h += blockDim.x) s_gt[h] = 0, s_eq[h] = 0;
   __syncthreads();
   for (int h = 0; h < H; ++h) {
     int gt = 0, eq = 0;
-    const float* row = base + (size_t)h * st.Ptot;
     for (int i = threadIdx.x; i < P; i += blockDim.x) {
-      const unsigned key = order_key(row[i]);
+      const unsigned key = key_at(h * P + i);
       gt += key > tau;
       eq += key == tau;
     }
@@ -507,17 +585,8 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
       const int j = e * T + tid;
       rk[e] = (inreg && j < n) ? skeys[kslot(j)] : 0u;
     }
-    // one warp-wide count of a digit: most warps see one digit only (always in the first
-    // passes): one vote, one add
     auto count_digit = [&](const unsigned digit, const int buf) {
-      const unsigned first = __shfl_sync(0xffffffffu, digit, 0);
-      if (__all_sync(0xffffffffu, digit == first)) {
-        if (lane == 0 && digit != 0xffffffffu) atomicAdd(&hist[buf][digit], 32);
-      } else {
-        const unsigned peers = __match_any_sync(0xffffffffu, digit);
-        if (digit != 0xffffffffu && (int)(__ffs(peers) - 1) == lane)
-          atomicAdd(&hist[buf][digit], __popc(peers));
-      }
+      count_digits(hist[buf], digit, lane);
     };
     for (int pass = 0; pass < 4; ++pass) {
       const int shift = 24 - 8 * pass, buf = pass & 1;
@@ -711,9 +780,24 @@ cudaError_t launch_mixpool(const LaunchCtx& c, const float* s_div, const float* 
 }
 
 cudaError_t launch_budget(const LaunchCtx& c, const float* scores, int* counts) {
-  return launch_pdl(k_budget, dim3(c.st.batch, c.st.layers), dim3(1024), 0, c.stream, 1, c.st,
-                    scores, counts,
-                    c.p.budget - c.p.window, floor_slots(c.p));
+  // keys of the longest sequence in shared memory when they fit
+  const size_t want = (size_t)c.st.H * (size_t)c.max_prefix * 4;
+  const size_t cap_bytes = 200 * 1024;
+  const size_t smem = want <= cap_bytes ? want : 0;
+  if (smem > 48 * 1024) {
+    static bool done[64] = {false};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64 || !done[dev]) {
+      e = cudaFuncSetAttribute(k_budget, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               (int)cap_bytes);
+      if (e != cudaSuccess) return e;
+      if (dev >= 0 && dev < 64) done[dev] = true;
+    }
+  }
+  return launch_pdl(k_budget, dim3(c.st.batch, c.st.layers), dim3(1024), smem, c.stream, 1, c.st,
+                    scores, counts, c.p.budget - c.p.window, floor_slots(c.p), (int)(smem / 4));
 }
 
 // Launch shape of k_tail: many (layer, sequence, head) units -> one 1024-thread CTA each; few ->
