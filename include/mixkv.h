@@ -216,6 +216,40 @@ int mixkv_compress_layers(const void* K, const void* V, const void* Qwin, int32_
                           int32_t* idx_offsets_opt, float* s_comp_opt, int32_t* status_dev,
                           void* stream, void* const* events_host, int32_t n_events);
 
+/* mixkv_compress_layers with the budgets chosen outside the library: the paper plugs its scores
+ * into compressors that differ only in how many rows a layer or a head may keep (Section 4.1 and
+ * the related-work appendix: PyramidKV gives lower layers more than higher ones, SparseMM / HeadKV
+ * give every head its own static share).  Scores, selection and gather are exactly those of
+ * mixkv_compress_layers; only the number of candidates taken per head comes from the caller.
+ *   head_budgets   device, [n_layers, batch * H] int32: rows to keep for that (layer, sequence,
+ *                  head), window included.  A value is used as min(max(v - W, 0), B - W, P_b)
+ *                  selected candidates plus the W window rows; p->budget (B) is the largest
+ *                  budget any head may get and sizes the outputs as in mixkv_compress_layers.
+ *   p->budget_mode must be MIXKV_BUDGET_FIXED (else MIXKV_ERR_INVALID_ARG).
+ * Outputs are ragged as with adaptive budgets: rows of (b, h) start at out_row_offsets[l][b*H+h]
+ * of layer l's slice; counts_opt receives the candidates actually selected. */
+int mixkv_compress_layers_budgeted(const void* K, const void* V, const void* Qwin,
+                                   int32_t n_layers, int64_t kv_layer_stride,
+                                   int64_t q_layer_stride, const int32_t* cu_seqlens_host,
+                                   int32_t batch, int32_t L, const mixkv_params* p,
+                                   void* workspace, size_t workspace_bytes,
+                                   const float* rbar_in_opt, const int32_t* head_budgets,
+                                   void* K_out, void* V_out, int32_t* out_row_offsets,
+                                   int32_t* idx_opt, int32_t* counts_opt, int32_t* idx_offsets_opt,
+                                   float* s_comp_opt, int32_t* status_dev, void* stream);
+
+/* Host-side layer schedule in the manner of PyramidKV (named in the paper's related work; the
+ * paper gives no formula, this is the build's reading): budgets fall linearly with depth and
+ * their sum stays n_layers * budget.  With B' = budget - window candidates per head and
+ * t = taper_permille / 1000 (0 <= taper_permille <= 999), layer l of n gets
+ * floor(B' * (1 + t * (1 - 2 l / (n - 1)))) candidates; the candidates lost to rounding go to
+ * the lowest layers, one each; window is added back.  budgets_host [n_layers] (host memory)
+ * receives the rows to keep per head of each layer: layer 0 gets the most.  Fill a
+ * [n_layers, batch * H] array with them for mixkv_compress_layers_budgeted and pass
+ * budgets_host[0] as p->budget.  No device work. */
+int mixkv_layer_budget_schedule(int32_t n_layers, int32_t budget, int32_t window,
+                                int32_t taper_permille, int32_t* budgets_host);
+
 /* Number of kernels one mixkv_compress_layer call enqueues for these parameters, and the
  * name of the i-th of them (NULL when i is out of range). */
 int mixkv_launches_per_layer(const mixkv_params* p);

@@ -254,3 +254,52 @@ def compress_layer(K, V, Q, params: Params, cu=None, rbar_in=None) -> Dict[str, 
     return {"s_comp": s_comp, "K_out": K_out[:rows].copy(), "V_out": V_out[:rows].copy(),
             "out_row_offsets": ro, "idx": idx[:offs[-1]].copy(),
             "counts": counts.reshape(batch, H), "idx_offsets": offs}
+
+
+# ------------------------------------------------------------------ budgets chosen outside
+# The paper plugs its scores into compressors that only differ in how many rows a layer or a
+# head keeps (Sec. 4.1; related work: PyramidKV layer schedules, SparseMM / HeadKV per-head
+# shares).  These two functions are plain Python on top of `topb`; the paper prints no formula
+# for either policy, so the schedule below is this build's reading (parity unpinned by the
+# paper; pinned by its invariants: total kept, monotone, taper 0 = uniform).
+def select_given(s: np.ndarray, head_budgets, params: Params, cu=None) -> Dict[str, np.ndarray]:
+    """Top-b on given scores [H, Ptot] with the rows to keep per (sequence, head) given
+    (window included): head (b, h) selects min(max(budget - W, 0), B - W, P_b) candidates."""
+    s = np.ascontiguousarray(s, dtype=np.float32)
+    H, Ptot = s.shape
+    W = params.window
+    if cu is None:
+        cu = [0, Ptot + W]
+    cu = _cu(cu)
+    batch = cu.shape[0] - 1
+    hb = np.asarray(head_budgets, dtype=np.int64).reshape(batch, H)
+    counts = np.zeros((batch, H), dtype=np.int32)
+    offs = np.zeros(batch * H + 1, dtype=np.int32)
+    parts = []
+    for b in range(batch):
+        P = int(cu[b + 1] - cu[b]) - W
+        p0 = int(cu[b]) - b * W
+        for h in range(H):
+            take = int(min(max(int(hb[b, h]) - W, 0), params.budget - W, P))
+            counts[b, h] = take
+            parts.append(topb(s[h, p0:p0 + P], take) if take > 0 else np.empty(0, np.int32))
+            offs[b * H + h + 1] = offs[b * H + h] + take
+    idx = np.concatenate(parts) if parts else np.empty(0, np.int32)
+    return {"idx": idx.astype(np.int32), "counts": counts, "idx_offsets": offs}
+
+
+def layer_budget_schedule(n_layers: int, budget: int, window: int, taper_permille: int):
+    """Rows to keep per head of each layer, falling linearly with depth, same total as a
+    uniform `budget`: with B' = budget - window and t = taper_permille / 1000, layer l gets
+    floor(B' (1 + t (1 - 2 l / (n - 1)))) candidates, the candidates lost to the rounding go
+    to the lowest layers one by one, and the window is added back."""
+    from fractions import Fraction
+    if n_layers == 1:
+        return [budget]
+    Bp = budget - window
+    t = Fraction(taper_permille, 1000)
+    cand = [int((Bp * (1 + t * (1 - Fraction(2 * l, n_layers - 1)))) // 1) for l in range(n_layers)]
+    short = n_layers * Bp - sum(cand)
+    for l in range(short):
+        cand[l] += 1
+    return [c + window for c in cand]

@@ -20,7 +20,8 @@ LIB_PATH = os.path.join(_PKG, "libmixkv.so")
 EXPORTS = ("mixkv_default_params", "mixkv_workspace_size", "mixkv_scores", "mixkv_select",
            "mixkv_compress_layer", "mixkv_compress_layer_traced", "mixkv_launches_per_layer",
            "mixkv_stage_name", "mixkv_status_string", "mixkv_scores_static",
-           "mixkv_workspace_size_layers", "mixkv_compress_layers")
+           "mixkv_workspace_size_layers", "mixkv_compress_layers",
+           "mixkv_compress_layers_budgeted", "mixkv_layer_budget_schedule")
 
 
 class MixKVError(RuntimeError):
@@ -98,6 +99,10 @@ def load_library() -> C.CDLL:
                                               C.POINTER(i32), i32, i32, C.POINTER(_CParams), vp,
                                               sz, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp,
                                               C.POINTER(vp), i32]
+        lib.mixkv_compress_layers_budgeted.argtypes = [
+            vp, vp, vp, i32, C.c_int64, C.c_int64, C.POINTER(i32), i32, i32, C.POINTER(_CParams),
+            vp, sz, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+        lib.mixkv_layer_budget_schedule.argtypes = [i32, i32, i32, i32, C.POINTER(i32)]
         lib.mixkv_stage_name.restype = C.c_char_p
         lib.mixkv_stage_name.argtypes = [C.POINTER(_CParams), i32]
         _lib = lib
@@ -294,11 +299,14 @@ def compress_layers(K: torch.Tensor, V: torch.Tensor, Q: torch.Tensor, params: P
                     rbar_in: Optional[torch.Tensor] = None,
                     workspace: Optional[torch.Tensor] = None, stream=None,
                     out: Optional[Dict[str, torch.Tensor]] = None,
-                    want_aux: bool = True, trace_events=None) -> Dict[str, torch.Tensor]:
+                    want_aux: bool = True, trace_events=None,
+                    head_budgets: Optional[torch.Tensor] = None) -> Dict[str, torch.Tensor]:
     """mixkv_compress_layers: K, V [n_layers, H, Ltot, 128], Q [n_layers, batch, H*G, W, 128]
     (bf16 device tensors; the layer dimension may be strided, the rest contiguous).  Returns
     K_out / V_out [n_layers, batch*H*B, 128], out_row_offsets [n_layers, batch*H+1] and, if
-    want_aux, idx [n_layers, cap] / counts / idx_offsets / s_comp."""
+    want_aux, idx [n_layers, cap] / counts / idx_offsets / s_comp.  With head_budgets (int32
+    device tensor [n_layers, batch*H], rows to keep per head, window included) the call goes to
+    mixkv_compress_layers_budgeted."""
     NL, H, Ltot, d = K.shape
     batch = 1 if cu_seqlens is None else len(cu_seqlens) - 1
     max_len = Ltot if cu_seqlens is None else max(int(cu_seqlens[b + 1]) - int(cu_seqlens[b])
@@ -328,6 +336,19 @@ def compress_layers(K: torch.Tensor, V: torch.Tensor, Q: torch.Tensor, params: P
     cu, _ = _cu_array(cu_seqlens)
     pc = params.c()
     ev, n_ev = (None, 0) if trace_events is None else (trace_events, len(trace_events))
+    if head_budgets is not None:
+        assert head_budgets.dtype == torch.int32 and head_budgets.is_contiguous()
+        assert tuple(head_budgets.shape) == (NL, batch * H) and trace_events is None
+        rc = load_library().mixkv_compress_layers_budgeted(
+            K.data_ptr(), V.data_ptr(), Q.data_ptr(), NL, K.stride(0), Q.stride(0), cu, batch,
+            Ltot, C.byref(pc), _ptr(workspace), workspace.numel(), _ptr(rbar_in),
+            _ptr(head_budgets), _ptr(out["K_out"]), _ptr(out["V_out"]),
+            _ptr(out["out_row_offsets"]), _ptr(out.get("idx")), _ptr(out.get("counts")),
+            _ptr(out.get("idx_offsets")), _ptr(out.get("s_comp")), _ptr(out["status"]),
+            _stream(stream))
+        if rc != 0:
+            raise MixKVError(rc, "mixkv_compress_layers_budgeted")
+        return out
     rc = load_library().mixkv_compress_layers(
         K.data_ptr(), V.data_ptr(), Q.data_ptr(), NL, K.stride(0), Q.stride(0), cu, batch, Ltot,
         C.byref(pc), _ptr(workspace), workspace.numel(), _ptr(rbar_in), _ptr(out["K_out"]),
@@ -337,3 +358,13 @@ def compress_layers(K: torch.Tensor, V: torch.Tensor, Q: torch.Tensor, params: P
     if rc != 0:
         raise MixKVError(rc, "mixkv_compress_layers")
     return out
+
+
+def layer_budget_schedule(n_layers: int, budget: int, window: int, taper_permille: int):
+    """mixkv_layer_budget_schedule: rows to keep per head of each layer (host list), falling
+    linearly with depth, total n_layers * budget."""
+    arr = (C.c_int32 * n_layers)()
+    rc = load_library().mixkv_layer_budget_schedule(n_layers, budget, window, taper_permille, arr)
+    if rc != 0:
+        raise MixKVError(rc, "mixkv_layer_budget_schedule")
+    return [int(v) for v in arr]

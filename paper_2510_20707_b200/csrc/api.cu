@@ -327,7 +327,8 @@ int compress_impl(const void* K, const void* V, const void* Qwin, int n_layers,
                   void* workspace, size_t workspace_bytes, const float* rbar_in_opt, void* K_out,
                   void* V_out, int32_t* out_row_offsets, int32_t* idx_opt, int32_t* counts_opt,
                   int32_t* idx_offsets_opt, float* s_comp_opt, int32_t* status_dev, void* stream,
-                  void* const* events_host, int32_t n_events) {
+                  void* const* events_host, int32_t n_events,
+                  const int32_t* head_budgets = nullptr) {
   LaunchCtx c;
   int rc = make_ctx(p, cu_seqlens_host, batch, L, workspace, workspace_bytes, stream, &c, n_layers,
                     kv_layer_stride, q_layer_stride);
@@ -350,6 +351,11 @@ int compress_impl(const void* K, const void* V, const void* Qwin, int n_layers,
   t.V = V;
   t.K_out = K_out;
   t.V_out = V_out;
+  if (head_budgets) {
+    // budgets given per (layer, sequence, head): no scores are needed to fix the counts
+    if (p->budget_mode != MIXKV_BUDGET_FIXED) return MIXKV_ERR_INVALID_ARG;
+    if (launch_given_budgets(c, head_budgets, counts) != cudaSuccess) return MIXKV_ERR_CUDA;
+  }
   rc = enqueue_passes(c, K, V, Qwin, c.ws.s_div, nullptr, status_dev);
   if (rc != MIXKV_OK) return rc;
   if (p->budget_mode == MIXKV_BUDGET_FIXED && tail_can_fuse(c)) {
@@ -357,7 +363,17 @@ int compress_impl(const void* K, const void* V, const void* Qwin, int n_layers,
     t.s_div = c.ws.s_div;
     t.rbar_in = rbar_in_opt;
     t.s_comp_out = s_comp;
-    t.counts_out = counts;
+    t.counts_dev = head_budgets ? counts : nullptr;
+    t.counts_out = head_budgets ? nullptr : counts;
+    c.mark();
+    if (launch_tail(c, t) != cudaSuccess) return MIXKV_ERR_CUDA;
+  } else if (head_budgets) {
+    c.mark();
+    if (launch_mixpool(c, c.ws.s_div, rbar_in_opt, nullptr, s_comp) != cudaSuccess)
+      return MIXKV_ERR_CUDA;
+    t.scores = s_comp;
+    t.counts_dev = counts;
+    t.counts_out = nullptr;
     c.mark();
     if (launch_tail(c, t) != cudaSuccess) return MIXKV_ERR_CUDA;
   } else {
@@ -398,6 +414,48 @@ int mixkv_compress_layers(const void* K, const void* V, const void* Qwin, int32_
                        batch, L, p, workspace, workspace_bytes, rbar_in_opt, K_out, V_out,
                        out_row_offsets, idx_opt, counts_opt, idx_offsets_opt, s_comp_opt,
                        status_dev, stream, events_host, n_events);
+}
+
+int mixkv_compress_layers_budgeted(const void* K, const void* V, const void* Qwin,
+                                   int32_t n_layers, int64_t kv_layer_stride,
+                                   int64_t q_layer_stride, const int32_t* cu_seqlens_host,
+                                   int32_t batch, int32_t L, const mixkv_params* p,
+                                   void* workspace, size_t workspace_bytes,
+                                   const float* rbar_in_opt, const int32_t* head_budgets,
+                                   void* K_out, void* V_out, int32_t* out_row_offsets,
+                                   int32_t* idx_opt, int32_t* counts_opt, int32_t* idx_offsets_opt,
+                                   float* s_comp_opt, int32_t* status_dev, void* stream) {
+  if (kv_layer_stride < 0 || q_layer_stride < 0 || !head_budgets) return MIXKV_ERR_INVALID_ARG;
+  return compress_impl(K, V, Qwin, n_layers, kv_layer_stride, q_layer_stride, cu_seqlens_host,
+                       batch, L, p, workspace, workspace_bytes, rbar_in_opt, K_out, V_out,
+                       out_row_offsets, idx_opt, counts_opt, idx_offsets_opt, s_comp_opt,
+                       status_dev, stream, nullptr, 0, head_budgets);
+}
+
+int mixkv_layer_budget_schedule(int32_t n_layers, int32_t budget, int32_t window,
+                                int32_t taper_permille, int32_t* budgets_host) {
+  if (n_layers < 1 || !budgets_host || window < 0 || budget <= window || taper_permille < 0 ||
+      taper_permille > 999)
+    return MIXKV_ERR_INVALID_ARG;
+  const long long Bp = budget - window, n = n_layers;
+  if (n == 1) {
+    budgets_host[0] = budget;
+    return MIXKV_OK;
+  }
+  // candidates of layer l: Bp * (1 + t * (1 - 2 l / (n - 1))), t = taper_permille / 1000, rounded
+  // down; the rows lost to rounding go to the lowest layers, one each, so the total stays n * Bp
+  const long long den = 1000 * (n - 1);
+  long long given = 0;
+  for (long long l = 0; l < n; ++l) {
+    const long long num = Bp * (den + (long long)taper_permille * ((n - 1) - 2 * l));
+    const long long c = num / den;
+    budgets_host[l] = (int32_t)c;
+    given += c;
+  }
+  long long rest = n * Bp - given;
+  for (long long l = 0; l < n && rest > 0; ++l, --rest) budgets_host[l] += 1;
+  for (long long l = 0; l < n; ++l) budgets_host[l] += window;
+  return MIXKV_OK;
 }
 
 int mixkv_compress_layer(const void* K, const void* V, const void* Qwin,

@@ -132,6 +132,8 @@ struct TailArgs {
   void* K_out;
   void* V_out;
 };
+// counts [layers, batch*H] <- candidates to select for budgets [layers, batch*H] given by the caller
+cudaError_t launch_given_budgets(const LaunchCtx& c, const int* budgets, int* counts);
 cudaError_t launch_tail(const LaunchCtx& c, const TailArgs& a);
 // Whether the longest sequence is short enough for the fused mix + select + gather kernel.
 bool tail_can_fuse(const LaunchCtx& c);

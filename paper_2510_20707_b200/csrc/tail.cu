@@ -779,6 +779,27 @@ cudaError_t launch_mixpool(const LaunchCtx& c, const float* s_div, const float* 
                     c.ws, s_div, rbar_in, s_ex_out, s_comp, mix_params(c.p));
 }
 
+// Budgets chosen by the caller (rows to keep per (layer, sequence, head), window included) ->
+// candidates to select: minus the window, at least 0, at most B - W and the candidates there are.
+__global__ void __launch_bounds__(256)
+k_given_budgets(const SeqTable st, const int* __restrict__ budgets, int* __restrict__ counts,
+                const int Bp) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int layer = blockIdx.x, BH = st.batch * st.H;
+  for (int t = threadIdx.x; t < BH; t += blockDim.x) {
+    const int b = t / st.H;
+    const int P = st.cu[b + 1] - st.cu[b] - st.W;
+    const int c = budgets[(size_t)layer * BH + t] - st.W;
+    counts[(size_t)layer * BH + t] = max(0, min(c, min(Bp, P)));
+  }
+}
+
+cudaError_t launch_given_budgets(const LaunchCtx& c, const int* budgets, int* counts) {
+  return launch_pdl(k_given_budgets, dim3(c.st.layers), dim3(256), 0, c.stream, 1, c.st, budgets,
+                    counts, c.p.budget - c.p.window);
+}
+
 cudaError_t launch_budget(const LaunchCtx& c, const float* scores, int* counts) {
   // keys of the longest sequence in shared memory when they fit
   const size_t want = (size_t)c.st.H * (size_t)c.max_prefix * 4;

@@ -135,10 +135,12 @@ def run_layer_parity(wl: synth.Workload, layer: int = 0, variant: str = "literal
 
 
 def run_layers_parity(wl: synth.Workload, layers, variant: str = "calibrated", pad_rows: int = 0,
-                      check=None, **kw):
+                      check=None, head_budgets=None, **kw):
     """mixkv_compress_layers over several layers at once against the oracle, layer by layer
     (only the positions listed in `check`, if given).  pad_rows > 0 leaves a gap between the
-    layers of K / V (a strided layer dimension)."""
+    layers of K / V (a strided layer dimension).  head_budgets (array [len(layers), batch*H],
+    rows to keep per head, window included) takes the budgeted entry point and the oracle's
+    select_given."""
     po, pg = params_pair(wl, **kw)
     cu = wl.cu_seqlens
     cu_arg = None if wl.batch == 1 else cu
@@ -156,14 +158,23 @@ def run_layers_parity(wl: synth.Workload, layers, variant: str = "calibrated", p
         return t
 
     K, V, Q = stack("K"), stack("V"), stack("Q")
-    out = binding.compress_layers(K, V, Q, pg, cu_seqlens=cu_list)
+    hb_dev = None
+    if head_budgets is not None:
+        head_budgets = np.asarray(head_budgets, dtype=np.int32).reshape(NL, wl.batch * H)
+        hb_dev = torch.from_numpy(head_budgets).cuda()
+    out = binding.compress_layers(K, V, Q, pg, cu_seqlens=cu_list, head_budgets=hb_dev)
     torch.cuda.synchronize()
     assert int(out["status"].item()) == 0
     for n, x in enumerate(xs):
         if check is not None and n not in check:
             continue
         ref_s = oracle.scores(x["K"], x["V"], x["Q"], po, cu=cu_arg)
-        ref = oracle.select(ref_s["s_comp"], po, cu=cu_arg)
+        if head_budgets is None:
+            ref = oracle.select(ref_s["s_comp"], po, cu=cu_arg)
+        else:
+            ref = oracle.select_given(ref_s["s_comp"], head_budgets[n], po, cu=cu)
+            assert np.array_equal(out["counts"][n].cpu().numpy().reshape(wl.batch, H),
+                                  ref["counts"])
         check_scores(f"s_comp[layer {n}]", out["s_comp"][n].cpu().numpy(), ref_s["s_comp"], cu, W)
         offs = out["idx_offsets"][n].cpu().numpy()
         idx = out["idx"][n].cpu().numpy()

@@ -244,3 +244,31 @@ def test_workspace_needs_no_clearing():
         assert torch.equal(first["idx"][:n_idx], out["idx"][:n_idx])
         assert torch.equal(first["K_out"][:n_rows].view(torch.int16), out["K_out"][:n_rows].view(torch.int16))
         assert torch.equal(first["V_out"][:n_rows].view(torch.int16), out["V_out"][:n_rows].view(torch.int16))
+
+
+def test_given_head_budgets_ragged():
+    # static per-head budgets (rows to keep, window included) chosen outside: below the window,
+    # above B, above the number of candidates of the short sequence, and everything between
+    wl = synth.small_workload(H=3, G=4, W=16, seq_lens=(900, 150, 2300), pool_kernel=5,
+                              budget=200, seed=51, centroids=8)
+    wl = synth.replace(wl, layers=3)
+    rng = np.random.default_rng(7)
+    hb = rng.integers(0, 260, size=(3, wl.batch * wl.kv_heads))
+    hb[0, 0], hb[0, 1], hb[1, 4], hb[2, 8] = 5, 16, 1000, 17
+    run_layers_parity(wl, range(3), head_budgets=hb)
+    # max pooling takes the unfused route (pooled-score sums, mix, then select + gather)
+    run_layers_parity(wl, range(3), head_budgets=hb, pool_mode=1)
+
+
+def test_layer_schedule_budgets():
+    # budgets falling linearly with depth (same total as a uniform budget of 96 rows per head)
+    n = 6
+    sched = binding.layer_budget_schedule(n, 96, 32, 600)
+    assert sched == oracle.layer_budget_schedule(n, 96, 32, 600) and sum(sched) == n * 96
+    wl = synth.small_workload(H=4, G=7, W=32, seq_lens=(4096,), pool_kernel=7, budget=sched[0],
+                              seed=52, centroids=16)
+    wl = synth.replace(wl, layers=n)
+    hb = np.repeat(np.asarray(sched)[:, None], wl.kv_heads, axis=1)
+    out = run_layers_parity(wl, range(n), head_budgets=hb, check=(0, 3, 5))
+    kept = out["out_row_offsets"][:, -1].cpu().numpy()
+    assert kept.tolist() == [wl.kv_heads * b for b in sched]
