@@ -60,6 +60,7 @@ enum { MIXKV_MIX_HEADWISE = 0, MIXKV_MIX_IMPORTANCE_ONLY = 1, MIXKV_MIX_DIVERSIT
        MIXKV_MIX_PLAIN_SUM = 3 };
 enum { MIXKV_POOL_AVG = 0, MIXKV_POOL_MAX = 1 };
 enum { MIXKV_BUDGET_FIXED = 0, MIXKV_BUDGET_ADAPTIVE = 1 };
+enum { MIXKV_INTRINSIC_NONE = 0, MIXKV_INTRINSIC_VNORM = 1, MIXKV_INTRINSIC_KNORM = 2 };
 
 typedef struct mixkv_params {
   int32_t kv_heads;     /* H */
@@ -68,7 +69,9 @@ typedef struct mixkv_params {
   int32_t window;       /* W: observation window, paper default 32 (Sec. 3.2) */
   int32_t pool_kernel;  /* odd k >= 1; 1-D pooling of the attention score, 1 = none */
   int32_t pool_mode;    /* MIXKV_POOL_AVG (zero padded, divides by k) or MIXKV_POOL_MAX */
-  int32_t use_vnorm;    /* 1: add the value-norm intrinsic importance of Eq. 2 */
+  int32_t use_vnorm;    /* intrinsic importance added in Eq. 2: MIXKV_INTRINSIC_VNORM (value norm,
+                           the paper's default), _KNORM (minus the key norm: the KNorm variant of
+                           Sec. 3.2 and of the ablation table), _NONE */
   int32_t mix_mode;     /* MIXKV_MIX_*: Eq. 5, or one of the ablation variants of Table 4 */
   int32_t budget_mode;  /* MIXKV_BUDGET_FIXED: B per head; _ADAPTIVE: B*H per sequence */
   int32_t budget;       /* B: rows kept per head INCLUDING the W window rows (Alg. 1) */
@@ -106,7 +109,7 @@ int mixkv_workspace_size_layers(const mixkv_params* p, int32_t n_layers, int32_t
  *   rbar_opt      out, optional, [batch, H]
  *   rbar_in_opt   in, optional, [batch, H]: redundancy to mix with instead of the computed
  *                 one (head weights calibrated offline, Sec. 4.3)
- *   V may be NULL when use_vnorm == 0. */
+ *   V may be NULL unless use_vnorm == MIXKV_INTRINSIC_VNORM. */
 int mixkv_scores(const void* K, const void* V, const void* Qwin,
                  const int32_t* cu_seqlens_host, int32_t batch, int32_t L,
                  const mixkv_params* p, void* workspace, size_t workspace_bytes,

@@ -49,7 +49,8 @@ typedef struct {
   int32_t window;        /* W, observation window (Sec. 3.2, default 32) */
   int32_t pool_kernel;   /* odd, 1 = no pooling */
   int32_t pool_mode;     /* 0 = average (zero padded), 1 = max */
-  int32_t use_vnorm;     /* 1 = add the VNorm intrinsic term (Eq. 2) */
+  int32_t use_vnorm;     /* intrinsic term of Eq. 2: 1 = VNorm (the default), 2 = KNorm (minus the
+                            key norm, Sec. 3.2), 0 = none */
   int32_t mix_mode;      /* 0 Eq. 5, 1 importance only, 2 diversity only, 3 plain sum */
   int32_t budget_mode;   /* 0 fixed B per head, 1 head-adaptive under a total of B*H */
   int32_t budget;        /* B: rows kept per head INCLUDING the W window rows */
@@ -314,7 +315,11 @@ int mixkv_oracle_scores(const uint16_t* K, const uint16_t* V, const uint16_t* Q,
       mixkv_oracle_window_attention(Kh, Qg, G, W, L, d, scale, ex_raw, NULL);
       mixkv_oracle_pool(ex_raw, P, p->pool_kernel, p->pool_mode, ex); /* prefix only */
       mixkv_oracle_key_geometry(Kh, L, d, dv, &r, NULL);               /* all L keys */
-      if (p->use_vnorm) mixkv_oracle_row_norms(Vh, P, d, vn);
+      if (p->use_vnorm == 1) mixkv_oracle_row_norms(Vh, P, d, vn);       /* VNorm (default) */
+      if (p->use_vnorm == 2) {                                           /* KNorm: minus the key norm */
+        mixkv_oracle_row_norms(Kh, P, d, vn);
+        for (int i = 0; i < P; ++i) vn[i] = -vn[i];
+      }
       const double r_mix = rbar_in ? (double)rbar_in[(size_t)b * H + h] : r;
       mixkv_oracle_mix(ex, p->use_vnorm ? vn : NULL, dv, P, r_mix, p->use_vnorm, p->mix_mode,
                        p->eps, comp, NULL, NULL, NULL);

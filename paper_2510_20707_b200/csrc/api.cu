@@ -43,6 +43,8 @@ int check_params(const mixkv_params* p) {
   if (p->pool_kernel < 1 || (p->pool_kernel & 1) == 0) return MIXKV_ERR_INVALID_ARG;
   if (p->pool_mode != MIXKV_POOL_AVG && p->pool_mode != MIXKV_POOL_MAX) return MIXKV_ERR_INVALID_ARG;
   if (p->mix_mode < 0 || p->mix_mode > 3) return MIXKV_ERR_INVALID_ARG;
+  if (p->use_vnorm < MIXKV_INTRINSIC_NONE || p->use_vnorm > MIXKV_INTRINSIC_KNORM)
+    return MIXKV_ERR_INVALID_ARG;
   if (p->budget_mode != MIXKV_BUDGET_FIXED && p->budget_mode != MIXKV_BUDGET_ADAPTIVE)
     return MIXKV_ERR_INVALID_ARG;
   if (p->budget <= p->window) return MIXKV_ERR_INVALID_ARG;
@@ -298,7 +300,8 @@ int mixkv_scores(const void* K, const void* V, const void* Qwin, const int32_t* 
   LaunchCtx c;
   int rc = make_ctx(p, cu_seqlens_host, batch, L, workspace, workspace_bytes, stream, &c);
   if (rc != MIXKV_OK) return rc;
-  if (!K || !Qwin || !s_comp || (p->use_vnorm && !V)) return MIXKV_ERR_INVALID_ARG;
+  if (!K || !Qwin || !s_comp || (p->use_vnorm == MIXKV_INTRINSIC_VNORM && !V))
+    return MIXKV_ERR_INVALID_ARG;
   if (!aligned16(K) || !aligned16(Qwin) || (V && !aligned16(V))) return MIXKV_ERR_INVALID_ARG;
   return enqueue_scores(c, K, V, Qwin, s_comp, s_ex_opt, s_div_opt, rbar_opt, rbar_in_opt,
                         status_dev);

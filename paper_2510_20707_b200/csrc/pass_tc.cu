@@ -660,7 +660,7 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
     }
   } else if (warp == kWarpTmaV) {
     // ------------------------------------------------------------------ V producer
-    if (lane == 0 && use_vnorm) {
+    if (lane == 0 && use_vnorm == MIXKV_INTRINSIC_VNORM) {
       int vit = 0;
       bool ok = true;
       for (TileIter ti(st.tile2_start, st.batch, H, st.nt2, lo, hi); ti.valid() && ok; ti.next()) {
@@ -858,7 +858,20 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
         seg_first = ti.id;
       }
       seg_start = ti.seg_last();
-      if (use_vnorm) {
+      if (use_vnorm == MIXKV_INTRINSIC_KNORM) {
+        // key-norm ablation: the intrinsic term is minus the key norm, which pass 1 left as its
+        // reciprocal; no V tile is loaded
+        const int P = st.cu[ti.b + 1] - st.cu[ti.b] - W;
+        const int i = ti.t * kTile + vt;
+        if (i < P) {
+          const float ki = ws.kinv[kpos(st, ti.layer, ti.h, ti.b, i)];
+          const float n = ki > 0.f ? -1.0f / ki : 0.f;
+          ws.vnorm[ppos(st, ti.layer, ti.h, ti.b, i)] = n;
+          vmin = fminf(vmin, n);
+          vmax = fmaxf(vmax, n);
+          vsum += n;
+        }
+      } else if (use_vnorm) {
         const int P = st.cu[ti.b + 1] - st.cu[ti.b] - W;
         const int vit = 2 * it + sub;
         const int vs = vit % vstages, vph = (vit / vstages) & 1;
@@ -1031,7 +1044,7 @@ cudaError_t launch_pass1(const LaunchCtx& c, const void* K, const void* Q, float
 cudaError_t launch_pass2(const LaunchCtx& c, const void* K, const void* V, const void* Q,
                          float* s_div_out, int* status) {
   CUtensorMap tmK, tmV, tmQ;
-  const void* Vsrc = c.p.use_vnorm ? V : K;   // the V map is never used without VNorm
+  const void* Vsrc = c.p.use_vnorm == MIXKV_INTRINSIC_VNORM ? V : K;   // the V map is never used without VNorm
   if (!map_kv(c, K, kTile, &tmK) || !map_kv(c, Vsrc, 64, &tmV) || !map_q(c, Q, &tmQ))
     return cudaErrorInvalidValue;
   static bool done[64] = {false};

@@ -39,7 +39,8 @@ def test_ragged_batch_fixed_and_adaptive():
 
 
 @pytest.mark.parametrize("kw", [
-    dict(pool_mode=1), dict(use_vnorm=0), dict(mix_mode=1), dict(mix_mode=2), dict(mix_mode=3),
+    dict(pool_mode=1), dict(use_vnorm=0), dict(use_vnorm=2), dict(use_vnorm=2, mix_mode=1),
+    dict(mix_mode=1), dict(mix_mode=2), dict(mix_mode=3),
     dict(use_vnorm=0, mix_mode=1), dict(eps=1e-3), dict(softmax_scale=0.05),
 ])
 def test_modes(kw):
@@ -107,6 +108,15 @@ def test_identical_keys_head():
 @pytest.mark.parametrize("name,layer", [("C2", 0), ("C2", 27), ("C5", 0)])
 def test_full_size_layers(name, layer):
     run_layer_parity(synth.CONFIGS[name], layer, "calibrated")
+
+
+def test_knorm_variant_full_size_and_batched():
+    # key-norm intrinsic term (Sec. 3.2 ablation): V is not read for the scores
+    run_layer_parity(synth.CONFIGS["C5"], 3, variant="calibrated", use_vnorm=2)
+    wl = synth.small_workload(H=2, G=4, W=32, seq_lens=(1500, 700), pool_kernel=7, budget=96,
+                              seed=61, centroids=8)
+    wl = synth.replace(wl, layers=4)
+    run_layers_parity(wl, range(4), use_vnorm=2)
 
 
 def test_c4_ragged_adaptive_layer():

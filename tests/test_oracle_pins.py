@@ -188,6 +188,34 @@ def test_normalisation_invariants_and_mix_limits():
     assert np.array_equal(oracle.mix(s_ex, None, s_div, 0.0, use_vnorm=0)["s_imp"], s_ex)
 
 
+def test_knorm_variant_rewards_small_key_norms():
+    # KNorm (Sec. 3.2): the intrinsic term is minus the key norm, normalised like VNorm.  With
+    # importance only, the layer score must equal mix(s_ex, -|K_i|, ...) of the same parts, the
+    # key of smallest norm gets the largest intrinsic term, and rescaling V changes nothing.
+    H, G, W, L, d = 2, 2, 4, 40, 8
+    K = RNG.standard_normal((H, L, d)) * (0.5 + RNG.random((H, L, 1)) * 3)
+    V = RNG.standard_normal((H, L, d))
+    Q = RNG.standard_normal((1, H * G, W, d))
+    Kb, Vb, Qb = bf16(K), bf16(V), bf16(Q)
+    pk = oracle.Params(kv_heads=H, gqa_ratio=G, head_dim=d, window=W, pool_kernel=1, budget=12,
+                       use_vnorm=2, mix_mode=1)
+    pn = oracle.Params(kv_heads=H, gqa_ratio=G, head_dim=d, window=W, pool_kernel=1, budget=12,
+                       use_vnorm=0, mix_mode=1)
+    sk = oracle.scores(Kb, Vb, Qb, pk)
+    s0 = oracle.scores(Kb, Vb, Qb, pn)
+    P = L - W
+    for h in range(H):
+        knorm = np.sqrt((f64(Kb[h, :P]) ** 2).sum(axis=1))
+        ref = oracle.mix(s0["s_comp"][h].astype(np.float64), -knorm, np.zeros(P), 0.0,
+                         mix_mode=1)["s_comp"]
+        assert np.allclose(sk["s_comp"][h], ref, rtol=2e-6, atol=0)
+        bonus = sk["s_comp"][h].astype(np.float64) - s0["s_comp"][h]
+        assert bonus.argmax() == knorm.argmin() and bonus.argmin() == knorm.argmax()
+        assert bonus.min() >= 0.0
+    again = oracle.scores(Kb, bf16(V * 7.0), Qb, pk)
+    assert np.array_equal(again["s_comp"], sk["s_comp"])
+
+
 def test_selection_invariant_to_rescaling_attention_scores():
     P = 500
     s_ex = RNG.random(P) ** 4
