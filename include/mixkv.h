@@ -253,6 +253,23 @@ int mixkv_compress_layers_budgeted(const void* K, const void* V, const void* Qwi
 int mixkv_layer_budget_schedule(int32_t n_layers, int32_t budget, int32_t window,
                                 int32_t taper_permille, int32_t* budgets_host);
 
+/* Redundancy analysis: the pairwise cosine similarity of the keys (or values) of a head, which
+ * the paper plots as heat maps and summarises per head (Sec. 1, Sec. 3.1, the redundancy
+ * figures), at block resolution.
+ *   X          device, [heads, L, head_dim] bf16, 16-byte aligned (head_dim must be 128)
+ *   block      rows per map cell (>= 1); T = ceil(L / block) cells per side (T <= 65535)
+ *   cells      device, [heads, T, T] fp32: mean of cos(x_i, x_j) over i in block I, j in block J,
+ *              pairs i == j left out (a diagonal cell averages n (n - 1) pairs, 0 if n == 1)
+ *   mean_opt   device, [heads] fp32 or NULL: mean over all ordered pairs i != j of the head,
+ *              the redundancy of Eq. 4
+ *   workspace  device, mixkv_similarity_workspace_size bytes, 16-byte aligned, caller-owned
+ * A zero row has cosine 0 with every row.  Enqueues three small kernels on `stream`; reads X
+ * once.  Errors as for the other entry points. */
+int mixkv_similarity_workspace_size(int32_t heads, int32_t L, int32_t block, size_t* bytes);
+int mixkv_similarity_map(const void* X, int32_t heads, int32_t L, int32_t head_dim, int32_t block,
+                         void* workspace, size_t workspace_bytes, float* cells, float* mean_opt,
+                         void* stream);
+
 /* Number of kernels one mixkv_compress_layer call enqueues for these parameters, and the
  * name of the i-th of them (NULL when i is out of range). */
 int mixkv_launches_per_layer(const mixkv_params* p);

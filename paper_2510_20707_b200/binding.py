@@ -21,7 +21,8 @@ EXPORTS = ("mixkv_default_params", "mixkv_workspace_size", "mixkv_scores", "mixk
            "mixkv_compress_layer", "mixkv_compress_layer_traced", "mixkv_launches_per_layer",
            "mixkv_stage_name", "mixkv_status_string", "mixkv_scores_static",
            "mixkv_workspace_size_layers", "mixkv_compress_layers",
-           "mixkv_compress_layers_budgeted", "mixkv_layer_budget_schedule")
+           "mixkv_compress_layers_budgeted", "mixkv_layer_budget_schedule",
+           "mixkv_similarity_workspace_size", "mixkv_similarity_map")
 
 
 class MixKVError(RuntimeError):
@@ -103,6 +104,8 @@ def load_library() -> C.CDLL:
             vp, vp, vp, i32, C.c_int64, C.c_int64, C.POINTER(i32), i32, i32, C.POINTER(_CParams),
             vp, sz, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.mixkv_layer_budget_schedule.argtypes = [i32, i32, i32, i32, C.POINTER(i32)]
+        lib.mixkv_similarity_workspace_size.argtypes = [i32, i32, i32, C.POINTER(sz)]
+        lib.mixkv_similarity_map.argtypes = [vp, i32, i32, i32, i32, vp, sz, vp, vp, vp]
         lib.mixkv_stage_name.restype = C.c_char_p
         lib.mixkv_stage_name.argtypes = [C.POINTER(_CParams), i32]
         _lib = lib
@@ -368,3 +371,24 @@ def layer_budget_schedule(n_layers: int, budget: int, window: int, taper_permill
     if rc != 0:
         raise MixKVError(rc, "mixkv_layer_budget_schedule")
     return [int(v) for v in arr]
+
+
+def similarity_map(X: torch.Tensor, block: int, want_mean: bool = True, stream=None):
+    """mixkv_similarity_map: X [heads, L, 128] bf16 device tensor -> (cells [heads, T, T] fp32,
+    mean [heads] fp32 or None): block-mean cosine similarity of the rows of every head."""
+    heads, L, d = X.shape
+    assert X.is_contiguous() and X.dtype == torch.bfloat16
+    need = C.c_size_t(0)
+    rc = load_library().mixkv_similarity_workspace_size(heads, L, block, C.byref(need))
+    if rc != 0:
+        raise MixKVError(rc, "mixkv_similarity_workspace_size")
+    ws = torch.empty(need.value, dtype=torch.uint8, device=X.device)
+    T = (L + block - 1) // block
+    cells = torch.empty((heads, T, T), dtype=torch.float32, device=X.device)
+    mean = torch.empty(heads, dtype=torch.float32, device=X.device) if want_mean else None
+    rc = load_library().mixkv_similarity_map(X.data_ptr(), heads, L, d, block, ws.data_ptr(),
+                                             ws.numel(), cells.data_ptr(), _ptr(mean),
+                                             _stream(stream))
+    if rc != 0:
+        raise MixKVError(rc, "mixkv_similarity_map")
+    return cells, mean
