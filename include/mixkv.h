@@ -270,6 +270,24 @@ int mixkv_similarity_map(const void* X, int32_t heads, int32_t L, int32_t head_d
                          void* workspace, size_t workspace_bytes, float* cells, float* mean_opt,
                          void* stream);
 
+/* The step after compression: one new query token per sequence attends over the compact cache
+ * that mixkv_compress_layers wrote (paper Sec. 3.1: decoding continues on the compressed K, V),
+ * all layers in one launch.  softmax(q . K^T * scale) V per query head over the rows kept for
+ * its KV head, fp32 accumulation.
+ *   K_cache, V_cache   device, [n_layers, rows_cap, d] bf16: K_out / V_out of the compression
+ *   out_row_offsets    device, [n_layers, batch * H + 1]: rows of (b, h) inside a layer's slice
+ *   rows_cap           rows between the slices of consecutive layers (batch * H * B)
+ *   q                  device, [n_layers, batch, H * G, d] bf16: the token's query per layer
+ *   max_rows           upper bound on the rows of one (layer, b, h), e.g. B; sizes shared memory
+ *                      (G * (128 + max_rows) floats <= 160 KB); rows beyond it are not read
+ *   out                device, [n_layers, batch, H * G, d] fp32; a head without rows gets zeros
+ * softmax_scale 0 means 1 / sqrt(d).  d must be 128, G <= 16 (else MIXKV_ERR_UNSUPPORTED). */
+int mixkv_decode_attention(const void* K_cache, const void* V_cache,
+                           const int32_t* out_row_offsets, int64_t rows_cap, const void* q,
+                           int32_t n_layers, int32_t batch, int32_t kv_heads, int32_t gqa_ratio,
+                           int32_t head_dim, float softmax_scale, int32_t max_rows, float* out,
+                           void* stream);
+
 /* Number of kernels one mixkv_compress_layer call enqueues for these parameters, and the
  * name of the i-th of them (NULL when i is out of range). */
 int mixkv_launches_per_layer(const mixkv_params* p);

@@ -22,7 +22,7 @@ EXPORTS = ("mixkv_default_params", "mixkv_workspace_size", "mixkv_scores", "mixk
            "mixkv_stage_name", "mixkv_status_string", "mixkv_scores_static",
            "mixkv_workspace_size_layers", "mixkv_compress_layers",
            "mixkv_compress_layers_budgeted", "mixkv_layer_budget_schedule",
-           "mixkv_similarity_workspace_size", "mixkv_similarity_map")
+           "mixkv_similarity_workspace_size", "mixkv_similarity_map", "mixkv_decode_attention")
 
 
 class MixKVError(RuntimeError):
@@ -106,6 +106,8 @@ def load_library() -> C.CDLL:
         lib.mixkv_layer_budget_schedule.argtypes = [i32, i32, i32, i32, C.POINTER(i32)]
         lib.mixkv_similarity_workspace_size.argtypes = [i32, i32, i32, C.POINTER(sz)]
         lib.mixkv_similarity_map.argtypes = [vp, i32, i32, i32, i32, vp, sz, vp, vp, vp]
+        lib.mixkv_decode_attention.argtypes = [vp, vp, vp, C.c_int64, vp, i32, i32, i32, i32, i32,
+                                               C.c_float, i32, vp, vp]
         lib.mixkv_stage_name.restype = C.c_char_p
         lib.mixkv_stage_name.argtypes = [C.POINTER(_CParams), i32]
         _lib = lib
@@ -392,3 +394,22 @@ def similarity_map(X: torch.Tensor, block: int, want_mean: bool = True, stream=N
     if rc != 0:
         raise MixKVError(rc, "mixkv_similarity_map")
     return cells, mean
+
+
+def decode_attention(K_cache: torch.Tensor, V_cache: torch.Tensor, out_row_offsets: torch.Tensor,
+                     q: torch.Tensor, kv_heads: int, gqa_ratio: int, max_rows: int,
+                     softmax_scale: float = 0.0, stream=None) -> torch.Tensor:
+    """mixkv_decode_attention: K_cache / V_cache [n_layers, rows_cap, 128] bf16 (the compact
+    cache), out_row_offsets [n_layers, batch*H+1] int32, q [n_layers, batch, H*G, 128] bf16 ->
+    [n_layers, batch, H*G, 128] fp32."""
+    NL, rows_cap, d = K_cache.shape
+    batch = q.shape[1]
+    assert K_cache.is_contiguous() and V_cache.is_contiguous() and q.is_contiguous()
+    assert out_row_offsets.dtype == torch.int32 and out_row_offsets.is_contiguous()
+    out = torch.empty(q.shape, dtype=torch.float32, device=q.device)
+    rc = load_library().mixkv_decode_attention(
+        K_cache.data_ptr(), V_cache.data_ptr(), out_row_offsets.data_ptr(), rows_cap, q.data_ptr(),
+        NL, batch, kv_heads, gqa_ratio, d, softmax_scale, max_rows, out.data_ptr(), _stream(stream))
+    if rc != 0:
+        raise MixKVError(rc, "mixkv_decode_attention")
+    return out
