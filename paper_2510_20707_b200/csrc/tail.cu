@@ -234,14 +234,17 @@ __device__ __forceinline__ void count_digits(int* hist, const unsigned digit, co
 // smallest and the largest key: the bits they share are the same in every key and are skipped,
 // so the first digit pass already sees digits that differ (scores of one sequence share sign
 // and most of the exponent; counting those bits would send every warp to the same one or two
-// bins).  Then digit passes of up to 8 bits, most significant first.  key_at(e) gives key e
-// (any order).  hist: 256 ints of shared memory.  Returns through tau / need_eq (same in every
-// thread).
+// bins).  Then digit passes of up to 8 bits, most significant first.  The first pass leaves one
+// bin to search; when its keys fit `list` (list_cap entries of shared memory) the second pass
+// copies them there while it counts, and the later passes read the list instead of all keys.
+// key_at(e) gives key e (any order).  hist: 256 ints of shared memory.  Returns through tau /
+// need_eq (same in every thread).
 template <typename KeyAt>
 __device__ __forceinline__ void radix_threshold(const KeyAt& key_at, const int total, const int want,
-                                                int* hist, unsigned* tau, int* need_eq) {
+                                                int* hist, unsigned* list, const int list_cap,
+                                                unsigned* tau, int* need_eq) {
   __shared__ unsigned s_prefix, s_lo[32], s_hi[32];
-  __shared__ int s_remaining;
+  __shared__ int s_remaining, s_cand, s_fill;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = (blockDim.x + 31) >> 5;
   unsigned lo = 0xffffffffu, hi = 0u;
   for (int e = threadIdx.x; e < total; e += blockDim.x) {
@@ -259,20 +262,44 @@ __device__ __forceinline__ void radix_threshold(const KeyAt& key_at, const int t
   unsigned mask = top == 32 ? 0u : ~((1u << top) - 1u);
   unsigned prefix = hi & mask;
   int remaining = want;
-  while (top > 0) {
+  int n_list = -1;        // >= 0: the candidates are in `list`
+  bool build = false;     // this pass copies the candidates to `list`
+  for (int pass = 0; top > 0; ++pass) {
     const int bits = min(8, top), shift = top - bits;
     const unsigned dmask = (1u << bits) - 1u;
     for (int t = threadIdx.x; t < 256; t += blockDim.x) hist[t] = 0;
-    if (threadIdx.x == 0) s_prefix = prefix, s_remaining = remaining;
+    if (threadIdx.x == 0) s_prefix = prefix, s_remaining = remaining, s_cand = 0, s_fill = 0;
     __syncthreads();
-    for (int e0 = 0; e0 < total; e0 += blockDim.x) {   // uniform trip count: full-warp votes
-      const int e = e0 + threadIdx.x;
-      unsigned digit = 0xffffffffu;
-      if (e < total) {
-        const unsigned key = key_at(e);
-        if ((key & mask) == prefix) digit = (key >> shift) & dmask;
+    if (n_list >= 0) {
+      for (int e0 = 0; e0 < n_list; e0 += blockDim.x) {   // uniform trip count: full-warp votes
+        const int e = e0 + threadIdx.x;
+        unsigned digit = 0xffffffffu;
+        if (e < n_list) {
+          const unsigned key = list[e];
+          if ((key & mask) == prefix) digit = (key >> shift) & dmask;
+        }
+        count_digits(hist, digit, lane);
       }
-      count_digits(hist, digit, lane);
+    } else {
+      for (int e0 = 0; e0 < total; e0 += blockDim.x) {   // uniform trip count: full-warp votes
+        const int e = e0 + threadIdx.x;
+        unsigned digit = 0xffffffffu, key = 0u;
+        if (e < total) {
+          key = key_at(e);
+          if ((key & mask) == prefix) digit = (key >> shift) & dmask;
+        }
+        count_digits(hist, digit, lane);
+        if (build) {   // one shared-memory add per warp reserves the slots of its candidates
+          const unsigned m = __ballot_sync(0xffffffffu, digit != 0xffffffffu);
+          if (m) {
+            const int leader = __ffs(m) - 1;
+            int base = 0;
+            if (lane == leader) base = atomicAdd(&s_fill, __popc(m));
+            base = __shfl_sync(0xffffffffu, base, leader);
+            if (digit != 0xffffffffu) list[base + __popc(m & ((1u << lane) - 1u))] = key;
+          }
+        }
+      }
     }
     __syncthreads();
     if (threadIdx.x < 32) {
@@ -293,6 +320,7 @@ __device__ __forceinline__ void radix_threshold(const KeyAt& key_at, const int t
         if (above < remaining && remaining <= above + h8[k]) {
           s_prefix = prefix | ((unsigned)(8 * lane + k) << shift);
           s_remaining = remaining - above;
+          s_cand = h8[k];
         }
         above += h8[k];
       }
@@ -302,6 +330,12 @@ __device__ __forceinline__ void radix_threshold(const KeyAt& key_at, const int t
     remaining = s_remaining;
     mask |= dmask << shift;
     top = shift;
+    if (build) {
+      n_list = s_fill;   // the list holds the keys under the prefix before this pass; the next
+      build = false;     // passes narrow the prefix inside it
+    } else if (n_list < 0 && pass == 0 && s_cand <= list_cap) {
+      build = true;
+    }
     __syncthreads();
   }
   *tau = prefix;
@@ -313,8 +347,8 @@ __device__ __forceinline__ void radix_threshold(const KeyAt& key_at, const int t
 // they fit (cache_cap keys); otherwise every pass reads them from global memory.
 __global__ void __launch_bounds__(1024)
 k_budget(const SeqTable st, const float* __restrict__ scores, int* __restrict__ counts,
-         const int Bp, const int floor_slots, const int cache_cap) {
-  extern __shared__ unsigned bkeys[];
+         const int Bp, const int floor_slots, const int cache_cap, const int list_cap) {
+  extern __shared__ unsigned bkeys[];   // [cache_cap] keys, then [list_cap] candidates
   __shared__ int hist[256];
   __shared__ int s_gt[64], s_eq[64];
   pdl_launch_dependents();
@@ -358,7 +392,7 @@ k_budget(const SeqTable st, const float* __restrict__ scores, int* __restrict__ 
   };
   unsigned tau;
   int need_eq;
-  radix_threshold(key_at, (int)total, (int)N, hist, &tau, &need_eq);
+  radix_threshold(key_at, (int)total, (int)N, hist, bkeys + cache_cap, list_cap, &tau, &need_eq);
   for (int h = threadIdx.x; h < H; h += blockDim.x) s_gt[h] = 0, s_eq[h] = 0;
   __syncthreads();
   for (int h = 0; h < H; ++h) {
@@ -804,7 +838,12 @@ cudaError_t launch_budget(const LaunchCtx& c, const float* scores, int* counts) 
   // keys of the longest sequence in shared memory when they fit
   const size_t want = (size_t)c.st.H * (size_t)c.max_prefix * 4;
   const size_t cap_bytes = 200 * 1024;
-  const size_t smem = want <= cap_bytes ? want : 0;
+  const size_t key_bytes = want <= cap_bytes - 16 * 1024 ? want : 0;
+  // the rest, up to 16 K entries, holds the candidates left after the first digit pass
+  size_t list_bytes = cap_bytes - key_bytes;
+  if (list_bytes > 64 * 1024) list_bytes = 64 * 1024;
+  if (list_bytes > want) list_bytes = want;
+  const size_t smem = key_bytes + list_bytes;
   if (smem > 48 * 1024) {
     static bool done[64] = {false};
     int dev = 0;
@@ -818,7 +857,8 @@ cudaError_t launch_budget(const LaunchCtx& c, const float* scores, int* counts) 
     }
   }
   return launch_pdl(k_budget, dim3(c.st.batch, c.st.layers), dim3(1024), smem, c.stream, 1, c.st,
-                    scores, counts, c.p.budget - c.p.window, floor_slots(c.p), (int)(smem / 4));
+                    scores, counts, c.p.budget - c.p.window, floor_slots(c.p), (int)(key_bytes / 4),
+                    (int)(list_bytes / 4));
 }
 
 // Launch shape of k_tail: many (layer, sequence, head) units -> one 1024-thread CTA each; few ->
