@@ -293,6 +293,14 @@ int mixkv_decode_attention(const void* K_cache, const void* V_cache,
 int mixkv_launches_per_layer(const mixkv_params* p);
 const char* mixkv_stage_name(const mixkv_params* p, int32_t i);
 
+/* Diagnostic (no counterpart in the paper): enqueues a one-CTA kernel that waits, through the
+ * same bounded-wait helper as the pass kernels, on a barrier nothing arrives on.  After the
+ * wait limit (2 s) the kernel writes MIXKV_ERR_TIMEOUT to *status_dev and, if waited_ns_dev is
+ * not NULL, the time it waited; it never traps and the context stays usable.  For tests of the
+ * error path. */
+int mixkv_selftest_bounded_wait(int32_t* status_dev, unsigned long long* waited_ns_dev,
+                                void* stream);
+
 /* Static, human-readable name of a status code. */
 const char* mixkv_status_string(int status);
 

@@ -22,7 +22,8 @@ EXPORTS = ("mixkv_default_params", "mixkv_workspace_size", "mixkv_scores", "mixk
            "mixkv_stage_name", "mixkv_status_string", "mixkv_scores_static",
            "mixkv_workspace_size_layers", "mixkv_compress_layers",
            "mixkv_compress_layers_budgeted", "mixkv_layer_budget_schedule",
-           "mixkv_similarity_workspace_size", "mixkv_similarity_map", "mixkv_decode_attention")
+           "mixkv_similarity_workspace_size", "mixkv_similarity_map", "mixkv_decode_attention",
+           "mixkv_selftest_bounded_wait")
 
 
 class MixKVError(RuntimeError):
@@ -108,6 +109,7 @@ def load_library() -> C.CDLL:
         lib.mixkv_similarity_map.argtypes = [vp, i32, i32, i32, i32, vp, sz, vp, vp, vp]
         lib.mixkv_decode_attention.argtypes = [vp, vp, vp, C.c_int64, vp, i32, i32, i32, i32, i32,
                                                C.c_float, i32, vp, vp]
+        lib.mixkv_selftest_bounded_wait.argtypes = [vp, vp, vp]
         lib.mixkv_stage_name.restype = C.c_char_p
         lib.mixkv_stage_name.argtypes = [C.POINTER(_CParams), i32]
         _lib = lib
@@ -413,3 +415,15 @@ def decode_attention(K_cache: torch.Tensor, V_cache: torch.Tensor, out_row_offse
     if rc != 0:
         raise MixKVError(rc, "mixkv_decode_attention")
     return out
+
+
+def selftest_bounded_wait(stream=None):
+    """mixkv_selftest_bounded_wait: returns (status, seconds waited) after the kernel has ended."""
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    waited = torch.zeros(1, dtype=torch.int64, device="cuda")
+    rc = load_library().mixkv_selftest_bounded_wait(status.data_ptr(), waited.data_ptr(),
+                                                    _stream(stream))
+    if rc != 0:
+        raise MixKVError(rc, "mixkv_selftest_bounded_wait")
+    torch.cuda.synchronize()
+    return int(status.item()), int(waited.item()) * 1e-9

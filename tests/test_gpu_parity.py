@@ -282,3 +282,13 @@ def test_layer_schedule_budgets():
     out = run_layers_parity(wl, range(n), head_budgets=hb, check=(0, 3, 5))
     kept = out["out_row_offsets"][:, -1].cpu().numpy()
     assert kept.tolist() == [wl.kv_heads * b for b in sched]
+
+
+def test_bounded_wait_reports_timeout_and_context_survives():
+    # a wait that nothing satisfies ends by itself after the limit, the status word says so,
+    # and the next call on the same context works
+    status, seconds = binding.selftest_bounded_wait()
+    assert status == -5 and binding.status_string(status) == "device-side bounded wait expired"
+    assert 1.5 < seconds < 4.0
+    wl = synth.small_workload(H=2, G=2, W=16, seq_lens=(600,), pool_kernel=5, budget=64, seed=81)
+    run_layer_parity(wl, variant="literal")
