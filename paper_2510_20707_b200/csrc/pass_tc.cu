@@ -440,15 +440,15 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
     const int chalf = c >> 3, cc = c & 7;
     constexpr int aux_threads = kP1AuxWarps * 32;
     const int kt = tid - kAuxWarp0 * 32;
-    float acc[8];
+    f32x2 acc2[4];   // dims 8c .. 8c+7 as four packed pairs
 #pragma unroll
-    for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+    for (int e = 0; e < 4; ++e) acc2[e] = pack2(0.f, 0.f);
     int it = 0, seg_first = lo;
     bool seg_start = true;
     for (TileIter ti(st.tile1_start, st.batch, H, st.nt1, lo, hi); ti.valid(); ti.next()) {
       if (seg_start) {
 #pragma unroll
-        for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+        for (int e = 0; e < 4; ++e) acc2[e] = pack2(0.f, 0.f);
         seg_first = ti.id;
       }
       seg_start = ti.seg_last();
@@ -465,13 +465,15 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
         for (int rr = 0; rr < 8; ++rr) {
           u[rr] = *reinterpret_cast<const uint4*>(tile + sw128_offset(row0 + rr, cc));
           const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&u[rr]);
-          float s0 = 0.f, s1 = 0.f;
+          f32x2 sq = pack2(0.f, 0.f);
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             const float2 f = __bfloat1622float2(p2[e]);
-            s0 = fmaf(f.x, f.x, s0);
-            s1 = fmaf(f.y, f.y, s1);
+            const f32x2 f2 = pack2(f.x, f.y);
+            sq = fma2(f2, f2, sq);
           }
+          float s0, s1;
+          unpack2(sq, s0, s1);
           p[rr] = s0 + s1;
         }
         if (bp == kPairs - 1) {   // the tile now lives in registers: hand the stage back
@@ -496,16 +498,19 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
         for (int rr = 0; rr < 8; ++rr) {
           const float w = __shfl_sync(0xffffffffu, inv, (lane & 16) | (rr << 1));
           const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&u[rr]);
+          const f32x2 w2 = pack2(w, w);
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             const float2 f = __bfloat1622float2(p2[e]);
-            acc[2 * e] = fmaf(f.x, w, acc[2 * e]);
-            acc[2 * e + 1] = fmaf(f.y, w, acc[2 * e + 1]);
+            acc2[e] = fma2(pack2(f.x, f.y), w2, acc2[e]);
           }
         }
       }
       if (group_sync_stop(2, aux_threads, kt == 0, abort, bars->vote, it)) break;
       if (seg_start) {
+        float acc[8];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) unpack2(acc2[e], acc[2 * e], acc[2 * e + 1]);
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
           const float v = acc[e] + __shfl_xor_sync(0xffffffffu, acc[e], 16);
@@ -877,7 +882,7 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
         const int vs = vit % vstages, vph = (vit / vstages) & 1;
         const bool ok = mbar_wait(&bars->vfull[vs], vph, abort);
         const unsigned char* tile = sV + vs * kVSubBytes;
-        float ss[4] = {0.f, 0.f, 0.f, 0.f};
+        f32x2 ss2[2] = {pack2(0.f, 0.f), pack2(0.f, 0.f)};
         if (ok) {
 #pragma unroll
           for (int half = 0; half < 2; ++half) {
@@ -889,8 +894,8 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
 #pragma unroll
               for (int e = 0; e < 4; ++e) {
                 const float2 f = __bfloat1622float2(p2[e]);
-                ss[e & 1] = fmaf(f.x, f.x, ss[e & 1]);
-                ss[2 + (e & 1)] = fmaf(f.y, f.y, ss[2 + (e & 1)]);
+                const f32x2 f2 = pack2(f.x, f.y);
+                ss2[e & 1] = fma2(f2, f2, ss2[e & 1]);
               }
             }
           }
@@ -899,6 +904,9 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
         if (lane == 0) mbar_arrive(&bars->vempty[vs]);
         const int i = ti.t * kTile + sub * 64 + vr;
         if (ok && i < P) {
+          float ss[4];
+          unpack2(ss2[0], ss[0], ss[2]);
+          unpack2(ss2[1], ss[1], ss[3]);
           const float n = sqrtf((ss[0] + ss[1]) + (ss[2] + ss[3]));
           ws.vnorm[ppos(st, ti.layer, ti.h, ti.b, i)] = n;
           vmin = fminf(vmin, n);
