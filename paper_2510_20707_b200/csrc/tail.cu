@@ -229,23 +229,29 @@ __device__ __forceinline__ void count_digits(int* hist, const unsigned digit, co
   if (((left >> lane) & 1u) && digit != 0xffffffffu) atomicAdd(&hist[digit], 1);
 }
 
-// Threshold of the `want` largest of `total` keys: the want-th largest key and how many keys
-// equal to it are still needed.  All threads of the CTA take part.  A first sweep finds the
-// smallest and the largest key: the bits they share are the same in every key and are skipped,
-// so the first digit pass already sees digits that differ (scores of one sequence share sign
-// and most of the exponent; counting those bits would send every warp to the same one or two
-// bins).  Then digit passes of up to 8 bits, most significant first.  The first pass leaves one
-// bin to search; when its keys fit `list` (list_cap entries of shared memory) the second pass
-// copies them there while it counts, and the later passes read the list instead of all keys.
-// key_at(e) gives key e (any order).  hist: 256 ints of shared memory.  Returns through tau /
-// need_eq (same in every thread).
+// Threshold of the `want` largest keys of a set spread over the CTAs of a cluster (one CTA: a
+// cluster of one): the want-th largest key and how many keys equal to it are still needed.  All
+// threads of all CTAs take part; key_at(e), e < total, gives the keys of this CTA (any order).
+// A first sweep finds the smallest and the largest key: the bits they share are the same in
+// every key and are skipped, so the first digit pass already sees digits that differ (scores of
+// one sequence share sign and most of the exponent; counting those bits would send every warp
+// to the same one or two bins).  Then digit passes of up to 8 bits, most significant first:
+// every CTA counts its keys, the histograms are added up through distributed shared memory
+// after a cluster barrier and every CTA finds the digit itself.  The first pass leaves one bin
+// to search; when its keys fit `list` (list_cap entries of shared memory) the second pass
+// copies this CTA's share of them there while it counts, and the later passes read the list
+// instead of all keys.  hist: 2 x 256 ints of shared memory, zeroed here.  Returns through
+// tau / need_eq (same in every thread of the cluster).
 template <typename KeyAt>
 __device__ __forceinline__ void radix_threshold(const KeyAt& key_at, const int total, const int want,
-                                                int* hist, unsigned* list, const int list_cap,
-                                                unsigned* tau, int* need_eq) {
-  __shared__ unsigned s_prefix, s_lo[32], s_hi[32];
-  __shared__ int s_remaining, s_cand, s_fill;
+                                                cg::cluster_group& cluster, int (*hist)[256],
+                                                unsigned* list, const int list_cap, unsigned* tau,
+                                                int* need_eq) {
+  __shared__ unsigned s_prefix, s_lo[32], s_hi[32], s_range[2];
+  __shared__ int s_remaining, s_cand, s_fill, htot[256];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = (blockDim.x + 31) >> 5;
+  const int cs = (int)cluster.num_blocks();
+  for (int t = threadIdx.x; t < 512; t += blockDim.x) hist[t >> 8][t & 255] = 0;
   unsigned lo = 0xffffffffu, hi = 0u;
   for (int e = threadIdx.x; e < total; e += blockDim.x) {
     const unsigned key = key_at(e);
@@ -256,18 +262,27 @@ __device__ __forceinline__ void radix_threshold(const KeyAt& key_at, const int t
   hi = __reduce_max_sync(0xffffffffu, hi);
   if (lane == 0) s_lo[warp] = lo, s_hi[warp] = hi;
   __syncthreads();
-  for (int w = 0; w < nwarps; ++w) lo = min(lo, s_lo[w]), hi = max(hi, s_hi[w]);
+  if (threadIdx.x == 0) {
+    for (int w = 0; w < nwarps; ++w) lo = min(lo, s_lo[w]), hi = max(hi, s_hi[w]);
+    s_range[0] = lo, s_range[1] = hi;
+  }
+  cluster.sync();
+  lo = 0xffffffffu, hi = 0u;
+  for (int r = 0; r < cs; ++r) {
+    const unsigned* rr = cluster.map_shared_rank(&s_range[0], r);
+    lo = min(lo, rr[0]);
+    hi = max(hi, rr[1]);
+  }
   const unsigned diff = lo ^ hi;
-  int top = diff ? 32 - __clz(diff) : 0;   // the low `top` bits differ between keys
+  int top = (hi >= lo && diff) ? 32 - __clz(diff) : 0;   // the low `top` bits differ between keys
   unsigned mask = top == 32 ? 0u : ~((1u << top) - 1u);
   unsigned prefix = hi & mask;
   int remaining = want;
-  int n_list = -1;        // >= 0: the candidates are in `list`
+  int n_list = -1;        // >= 0: this CTA's candidates are in `list`
   bool build = false;     // this pass copies the candidates to `list`
   for (int pass = 0; top > 0; ++pass) {
-    const int bits = min(8, top), shift = top - bits;
+    const int bits = min(8, top), shift = top - bits, buf = pass & 1;
     const unsigned dmask = (1u << bits) - 1u;
-    for (int t = threadIdx.x; t < 256; t += blockDim.x) hist[t] = 0;
     if (threadIdx.x == 0) s_prefix = prefix, s_remaining = remaining, s_cand = 0, s_fill = 0;
     __syncthreads();
     if (n_list >= 0) {
@@ -278,7 +293,7 @@ __device__ __forceinline__ void radix_threshold(const KeyAt& key_at, const int t
           const unsigned key = list[e];
           if ((key & mask) == prefix) digit = (key >> shift) & dmask;
         }
-        count_digits(hist, digit, lane);
+        count_digits(hist[buf], digit, lane);
       }
     } else {
       for (int e0 = 0; e0 < total; e0 += blockDim.x) {   // uniform trip count: full-warp votes
@@ -288,7 +303,7 @@ __device__ __forceinline__ void radix_threshold(const KeyAt& key_at, const int t
           key = key_at(e);
           if ((key & mask) == prefix) digit = (key >> shift) & dmask;
         }
-        count_digits(hist, digit, lane);
+        count_digits(hist[buf], digit, lane);
         if (build) {   // one shared-memory add per warp reserves the slots of its candidates
           const unsigned m = __ballot_sync(0xffffffffu, digit != 0xffffffffu);
           if (m) {
@@ -301,12 +316,19 @@ __device__ __forceinline__ void radix_threshold(const KeyAt& key_at, const int t
         }
       }
     }
+    cluster.sync();
+    if (threadIdx.x < 256) {
+      int tot = 0;
+      for (int r = 0; r < cs; ++r) tot += *cluster.map_shared_rank(&hist[buf][threadIdx.x], r);
+      htot[threadIdx.x] = tot;
+      hist[buf ^ 1][threadIdx.x] = 0;   // every CTA is past its reads of the other buffer
+    }
     __syncthreads();
     if (threadIdx.x < 32) {
       // lane l owns bins 8l .. 8l+7; `above` = keys in higher bins
       int h8[8], mine = 0;
 #pragma unroll
-      for (int k = 0; k < 8; ++k) h8[k] = hist[8 * lane + k], mine += h8[k];
+      for (int k = 0; k < 8; ++k) h8[k] = htot[8 * lane + k], mine += h8[k];
       // suffix sum over lanes: keys in the bins of higher lanes
       int incl = mine;
 #pragma unroll
@@ -331,8 +353,8 @@ __device__ __forceinline__ void radix_threshold(const KeyAt& key_at, const int t
     mask |= dmask << shift;
     top = shift;
     if (build) {
-      n_list = s_fill;   // the list holds the keys under the prefix before this pass; the next
-      build = false;     // passes narrow the prefix inside it
+      n_list = s_fill;   // the list holds this CTA's keys under the prefix before this pass; the
+      build = false;     // next passes narrow the prefix inside it
     } else if (n_list < 0 && pass == 0 && s_cand <= list_cap) {
       build = true;
     }
@@ -342,18 +364,24 @@ __device__ __forceinline__ void radix_threshold(const KeyAt& key_at, const int t
   *need_eq = remaining;
 }
 
-// Head budgets of one sequence under the adaptive rule (see mixkv.h).  The H * P pooled scores
-// of the sequence are turned into order-preserving keys once and kept in shared memory when
-// they fit (cache_cap keys); otherwise every pass reads them from global memory.
+constexpr int kBudgetCluster = 8;
+
+// Head budgets of one sequence under the adaptive rule (see mixkv.h).  One CTA per (sequence,
+// layer) when the call has many of them, else a cluster of kBudgetCluster CTAs, each with a
+// slice of the positions of every head.  A CTA turns its H * n pooled scores into
+// order-preserving keys once and keeps them in shared memory when they fit (cache_cap keys);
+// otherwise every pass reads them from global memory.
 __global__ void __launch_bounds__(1024)
 k_budget(const SeqTable st, const float* __restrict__ scores, int* __restrict__ counts,
          const int Bp, const int floor_slots, const int cache_cap, const int list_cap) {
   extern __shared__ unsigned bkeys[];   // [cache_cap] keys, then [list_cap] candidates
-  __shared__ int hist[256];
-  __shared__ int s_gt[64], s_eq[64];
+  __shared__ int hist[2][256];
+  __shared__ int s_gt[64], s_eq[64], t_gt[64], t_eq[64];
+  cg::cluster_group cluster = cg::this_cluster();
+  const int cs = (int)cluster.num_blocks(), crank = (int)cluster.block_rank();
   pdl_launch_dependents();
   pdl_wait();
-  const int b = blockIdx.x, layer = blockIdx.y, H = st.H;
+  const int b = blockIdx.x / cs, layer = blockIdx.y, H = st.H;
   counts += (size_t)layer * st.batch * H;
   const int P = st.cu[b + 1] - st.cu[b] - st.W;
   const long long total = (long long)H * P;
@@ -361,25 +389,30 @@ k_budget(const SeqTable st, const float* __restrict__ scores, int* __restrict__ 
   if (N > total) N = total;
   const float* base = scores + ppos(st, layer, 0, b, 0);
   const size_t stride = (size_t)st.Ptot;
-  if (N <= 0) {
-    for (int h = threadIdx.x; h < H; h += blockDim.x) counts[b * H + h] = min(floor_slots, P);
+  if (N <= 0) {   // the same in every CTA of the cluster
+    if (crank == 0)
+      for (int h = threadIdx.x; h < H; h += blockDim.x) counts[b * H + h] = min(floor_slots, P);
     return;
   }
-  const bool cached = total <= (long long)cache_cap;
+  // this CTA's slice of every head: positions [p0, p0 + n)
+  const int chunk = (P + cs - 1) / cs;
+  const int p0 = min(crank * chunk, P), n = min(chunk, P - p0);
+  const int local = H * n;
+  const bool cached = local <= cache_cap;
   if (cached) {
     for (int h = 0; h < H; ++h) {
-      const float* row = base + (size_t)h * stride;
-      for (int i0 = 0; i0 < P; i0 += 8 * blockDim.x) {   // eight loads in flight per thread
+      const float* row = base + (size_t)h * stride + p0;
+      for (int i0 = 0; i0 < n; i0 += 8 * blockDim.x) {   // eight loads in flight per thread
         float v[8];
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
           const int i = i0 + k * blockDim.x + threadIdx.x;
-          v[k] = i < P ? row[i] : 0.f;
+          v[k] = i < n ? row[i] : 0.f;
         }
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
           const int i = i0 + k * blockDim.x + threadIdx.x;
-          if (i < P) bkeys[h * P + i] = order_key(v[k]);
+          if (i < n) bkeys[h * n + i] = order_key(v[k]);
         }
       }
     }
@@ -387,18 +420,18 @@ k_budget(const SeqTable st, const float* __restrict__ scores, int* __restrict__ 
   }
   auto key_at = [&](const int e) -> unsigned {
     if (cached) return bkeys[e];
-    const int h = e / P;
-    return order_key(base[(size_t)h * stride + (e - h * P)]);
+    const int h = e / n;
+    return order_key(base[(size_t)h * stride + p0 + (e - h * n)]);
   };
   unsigned tau;
   int need_eq;
-  radix_threshold(key_at, (int)total, (int)N, hist, bkeys + cache_cap, list_cap, &tau, &need_eq);
+  radix_threshold(key_at, local, (int)N, cluster, hist, bkeys + cache_cap, list_cap, &tau, &need_eq);
   for (int h = threadIdx.x; h < H; h += blockDim.x) s_gt[h] = 0, s_eq[h] = 0;
   __syncthreads();
   for (int h = 0; h < H; ++h) {
     int gt = 0, eq = 0;
-    for (int i = threadIdx.x; i < P; i += blockDim.x) {
-      const unsigned key = key_at(h * P + i);
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+      const unsigned key = key_at(h * n + i);
       gt += key > tau;
       eq += key == tau;
     }
@@ -411,15 +444,27 @@ k_budget(const SeqTable st, const float* __restrict__ scores, int* __restrict__ 
       atomicAdd(&s_eq[h], eq);
     }
   }
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    int rem = need_eq;  // equal-to-threshold elements go to the lower (head, position) first
-    for (int h = 0; h < H; ++h) {
-      const int take = min(s_eq[h], rem);
-      rem -= take;
-      counts[b * H + h] = min(floor_slots + s_gt[h] + take, P);
+  cluster.sync();   // every CTA's per-head counts are complete
+  if (crank == 0) {
+    for (int h = threadIdx.x; h < H; h += blockDim.x) {
+      int g = 0, q = 0;
+      for (int r = 0; r < cs; ++r) {
+        g += *cluster.map_shared_rank(&s_gt[h], r);
+        q += *cluster.map_shared_rank(&s_eq[h], r);
+      }
+      t_gt[h] = g, t_eq[h] = q;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      int rem = need_eq;  // equal-to-threshold elements go to the lower (head, position) first
+      for (int h = 0; h < H; ++h) {
+        const int take = min(t_eq[h], rem);
+        rem -= take;
+        counts[b * H + h] = min(floor_slots + t_gt[h] + take, P);
+      }
     }
   }
+  cluster.sync();   // the peers' shared memory stays alive until rank 0 has read it
 }
 
 // ------------------------------------------------------------------------------ tail
@@ -835,8 +880,11 @@ cudaError_t launch_given_budgets(const LaunchCtx& c, const int* budgets, int* co
 }
 
 cudaError_t launch_budget(const LaunchCtx& c, const float* scores, int* counts) {
-  // keys of the longest sequence in shared memory when they fit
-  const size_t want = (size_t)c.st.H * (size_t)c.max_prefix * 4;
+  // few (sequence, layer) pairs: a cluster of CTAs each; many: one CTA each
+  const int cs = c.st.batch * c.st.layers < device_sm_count() / kBudgetCluster ? kBudgetCluster : 1;
+  const size_t chunk = ((size_t)c.max_prefix + cs - 1) / cs;
+  // the keys of a CTA's slice of the longest sequence in shared memory when they fit
+  const size_t want = (size_t)c.st.H * chunk * 4;
   const size_t cap_bytes = 200 * 1024;
   const size_t key_bytes = want <= cap_bytes - 16 * 1024 ? want : 0;
   // the rest, up to 16 K entries, holds the candidates left after the first digit pass
@@ -856,9 +904,9 @@ cudaError_t launch_budget(const LaunchCtx& c, const float* scores, int* counts) 
       if (dev >= 0 && dev < 64) done[dev] = true;
     }
   }
-  return launch_pdl(k_budget, dim3(c.st.batch, c.st.layers), dim3(1024), smem, c.stream, 1, c.st,
-                    scores, counts, c.p.budget - c.p.window, floor_slots(c.p), (int)(key_bytes / 4),
-                    (int)(list_bytes / 4));
+  return launch_pdl(k_budget, dim3(c.st.batch * cs, c.st.layers), dim3(1024), smem, c.stream, cs,
+                    c.st, scores, counts, c.p.budget - c.p.window, floor_slots(c.p),
+                    (int)(key_bytes / 4), (int)(list_bytes / 4));
 }
 
 // Launch shape of k_tail: many (layer, sequence, head) units -> one 1024-thread CTA each; few ->
