@@ -187,18 +187,37 @@ k_mixpool(const SeqTable st, const Workspace ws, const float* __restrict__ s_div
   if (threadIdx.x < 32)
     head_scalars(st, ws, layer, b, h, mp.pool_k, mp.pool_mode, mp.use_vnorm, mp.eps, rbar_in,
                  threadIdx.x, sc);
-  for (int t = threadIdx.x; t < (p1 - p0) + 2 * half; t += 256) {
-    const int i = p0 - half + t;
-    tile[t] = (i >= 0 && i < P) ? ws.s_ex_raw[poff + i] : pad;
+  // a chunk is eight rounds of 256 positions (+ the pooling halo in a ninth); every load of the
+  // chunk is issued before the first use
+  constexpr int kRounds = kPChunk / 256;
+  const int nstage = (p1 - p0) + 2 * half;
+  float raw[kRounds + 1], vn[kRounds], dv[kRounds];
+#pragma unroll
+  for (int e = 0; e <= kRounds; ++e) {
+    const int t = e * 256 + threadIdx.x, i = p0 - half + t;
+    raw[e] = (t < nstage && i >= 0 && i < P) ? ws.s_ex_raw[poff + i] : pad;
+  }
+#pragma unroll
+  for (int e = 0; e < kRounds; ++e) {
+    const int i = p0 + e * 256 + threadIdx.x;
+    vn[e] = (mp.use_vnorm && i < p1) ? ws.vnorm[poff + i] : 0.f;
+    dv[e] = i < p1 ? s_div[poff + i] : 0.f;
+  }
+#pragma unroll
+  for (int e = 0; e <= kRounds; ++e) {
+    const int t = e * 256 + threadIdx.x;
+    if (t < nstage) tile[t] = raw[e];
   }
   __syncthreads();
   const float invk = 1.0f / (float)mp.pool_k;
-  for (int t = threadIdx.x; t < p1 - p0; t += 256) {
-    const int i = p0 + t;
-    const float ex = pool_window(tile + t, mp.pool_k, mp.pool_mode, invk);
-    if (s_ex_out) s_ex_out[poff + i] = ex;
-    const float vn = mp.use_vnorm ? ws.vnorm[poff + i] : 0.f;
-    s_comp[poff + i] = mix_one(ex, vn, s_div[poff + i], sc, mp.use_vnorm, mp.mix_mode);
+#pragma unroll
+  for (int e = 0; e < kRounds; ++e) {
+    const int t = e * 256 + threadIdx.x, i = p0 + t;
+    if (i < p1) {
+      const float ex = pool_window(tile + t, mp.pool_k, mp.pool_mode, invk);
+      if (s_ex_out) s_ex_out[poff + i] = ex;
+      s_comp[poff + i] = mix_one(ex, vn[e], dv[e], sc, mp.use_vnorm, mp.mix_mode);
+    }
   }
 }
 
