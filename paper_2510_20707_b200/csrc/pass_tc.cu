@@ -6,12 +6,12 @@
 //   pass 1  K from HBM.  Logits with the window queries on the M side (one query row per TMEM
 //           lane), so the running softmax (max, sum) of a row is thread-local; alongside, key
 //           norms and the sum of unit keys from the shared-memory tile.
-//   pass 2  K again (served by L2), V from HBM.  At the start of a (sequence, head) segment the
-//           CTA folds pass 1's per-CTA partials: the softmax statistics become one log2
-//           normaliser per window row, the unit-key sums become the mean unit key (bf16 hi /
-//           lo / lo2 rows) and the redundancy of Eq. 4.  Logits with the keys on the M side (one key
-//           per TMEM lane), normalised with the finished row statistics, so the column sum over
-//           window rows and query heads is thread-local -> s_ex_raw.  The mean unit key rides
+//           The CTA that delivers the last segment of a (layer, sequence, head) folds all of
+//           its segments: the softmax statistics become one log2 normaliser per window row,
+//           the unit-key sums become the mean unit key and the redundancy of Eq. 4.
+//   pass 2  K again, V from HBM.  Logits with the keys on the M side (one key per TMEM lane),
+//           normalised with the finished row statistics, so the column sum over window rows
+//           and query heads is thread-local -> s_ex_raw.  The mean unit key rides
 //           along as three extra bf16 "query" rows -> K_i . kbar -> s_div.  Value norms are
 //           computed from V tiles staged next to the K tiles.
 //
@@ -27,21 +27,29 @@ namespace {
 constexpr int kTileBytes = kTile * 256;    // 128 keys x 128 bf16
 constexpr int kHalfBytes = kTile * 128;    // one 64-column half of a K tile
 
-// warp roles (16 warps per CTA)
-constexpr int kThreads = 16 * 32;
+// Warp roles.  Warpgroup 0 (warps 0..3) holds the single-thread roles: TMA producer, MMA
+// issuer, (pass 2) V producer; warps 4..19 are the epilogue: two groups of eight warps, group g
+// owns accumulator stage g of tensor memory and therefore every other tile, so the exponentials
+// of two tiles are in flight on every scheduler at any time (the exp2 unit is what bounds both
+// passes, and eight warps cannot keep it busy: their chains are too short to cover its latency);
+// the warps from 20 on compute key statistics (pass 1) or value norms (pass 2).  A warp's TMEM
+// lane quarter is warp % 4.  Register budgets per role are set with setmaxnreg: the kernels are
+// launched with 72 / 80 registers per thread and the single-thread roles hand most of theirs to
+// the epilogue warps.
 constexpr int kWarpTma = 0, kWarpMma = 1;
-constexpr int kEpiWarp0 = 4, kEpiWarps = 8;      // warps 4..11: warp % 4 = TMEM lane quarter
+constexpr int kP1WarpMma = 3;                    // pass 1: see k_pass1
+constexpr int kEpiWarp0 = 4;
+constexpr int kEpiWarps = 16;                    // warps 4..19
 constexpr int kEpiThreads = kEpiWarps * 32;
-constexpr int kAuxWarp0 = 12;                    // warps 12..15: key statistics / value norms
+constexpr int kAuxWarp0 = kEpiWarp0 + kEpiWarps; // warps 20..: key statistics / value norms
+constexpr int kThreads2 = (kAuxWarp0 + 4) * 32;  // pass 2: 24 warps
 
-// Named barrier among n threads that also agrees on whether to stop: the leader samples the
-// CTA abort flag before the barrier and everybody reads that sample after it, so a group
-// never splits around a later barrier.
-__device__ __forceinline__ bool group_sync_stop(int id, int n, bool leader, volatile int* abort,
-                                                volatile int* slots, int it) {
-  if (leader) slots[it & 1] = *abort;
-  named_bar_sync(id, n);
-  return slots[it & 1] != 0;
+// Registers per thread of the calling warpgroup from here on: N, where the kernel was launched
+// with BASE (every warp of the warpgroup executes this).
+template <int N, int BASE>
+__device__ __forceinline__ void set_regs() {
+  if constexpr (N < BASE) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
+  if constexpr (N > BASE) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
 }
 
 // Counts a delivered segment of a (layer, sequence, head) whose partial results come from
@@ -110,15 +118,22 @@ __device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
 constexpr size_t kSmemLimit = 227 * 1024;   // dynamic shared memory a CTA may ask for
 
 // ======================================================================== pass 1
-// Key-statistics warps (from warp 12 on): 8 for one 128-row query block, where their latency
-// chains set the pace, 4 for two blocks, where the epilogue does.  One tile = 8 pairs of 8-row
-// batches, spread evenly over the warps.
-__host__ __device__ constexpr int p1_aux_warps(int MB) { return MB == 2 ? 4 : 8; }
+// Eight key-statistics warps (from warp 20 on): one tile = 8 pairs of 8-row batches, one pair per
+// warp.  28 warps per CTA.
+__host__ __device__ constexpr int p1_aux_warps(int MB) { return 8; }
 __host__ __device__ constexpr int p1_threads(int MB) { return (kAuxWarp0 + p1_aux_warps(MB)) * 32; }
 constexpr int kP1MaxStages = 6;
 // K tile ring: as deep as shared memory allows next to the query tile (the deeper the ring, the
 // more bytes in flight towards HBM)
 __host__ __device__ constexpr int p1_stages(int MB) { return 5; }
+// registers per thread: at launch, then per role (7 warpgroups: 40 + 4 * 72 + 2 * 88 = 7 * 72;
+// the key-statistics warps hold a batch of eight key rows in registers between their two sweeps)
+#ifndef P1_LEAD
+#define P1_LEAD 40
+#define P1_EPI 72
+#define P1_AUX 88
+#endif
+constexpr int kP1RegsLaunch = 72, kP1RegsLead = P1_LEAD, kP1RegsEpi = P1_EPI, kP1RegsAux = P1_AUX;
 
 struct P1Bars {
   uint64_t full[kP1MaxStages];
@@ -129,7 +144,6 @@ struct P1Bars {
   uint64_t qfree;
   uint32_t tmem_base;
   int abort;
-  int vote[2];
   int last;   // this CTA delivered the last segment of the head at hand
 };
 
@@ -144,16 +158,16 @@ __device__ __forceinline__ float fold_row_stats(const float2* rowstat, const Seg
   const int total = sl.nseg * NU;
   float Mx = -1e30f, Zs = 0.f;
 #pragma unroll 1
-  for (int i0 = 0; i0 < total; i0 += 20) {   // twenty loads in flight
-    float2 v[20];
+  for (int i0 = 0; i0 < total; i0 += 12) {   // twelve loads in flight
+    float2 v[12];
 #pragma unroll
-    for (int k = 0; k < 20; ++k) {
+    for (int k = 0; k < 12; ++k) {
       const int i = i0 + k;
       v[k] = make_float2(-1e30f, 0.f);
-      if (i < total) v[k] = __ldcg(rowstat + ((size_t)sl.start(i / NU) * 2 + (i % NU)) * NQ + q);
+      if (i < total) v[k] = __ldcg(rowstat + ((size_t)sl.start(i / NU) * NU + (i % NU)) * NQ + q);
     }
 #pragma unroll
-    for (int k = 0; k < 20; ++k) {
+    for (int k = 0; k < 12; ++k) {
       const float mn = fmaxf(Mx, v[k].x);
       Zs = Zs * ex2(Mx - mn) + v[k].y * ex2(v[k].x - mn);
       Mx = mn;
@@ -165,25 +179,28 @@ __device__ __forceinline__ float fold_row_stats(const float2* rowstat, const Seg
 __device__ __forceinline__ float fold_key_sums(const float* ksum, const SegList& sl, const int kt) {
   float sum = 0.f;
 #pragma unroll 1
-  for (int e0 = 0; e0 < sl.nseg; e0 += 20) {   // twenty loads in flight
-    float v[20];
+  for (int e0 = 0; e0 < sl.nseg; e0 += 12) {   // twelve loads in flight
+    float v[12];
 #pragma unroll
-    for (int e = 0; e < 20; ++e)
+    for (int e = 0; e < 12; ++e)
       v[e] = e0 + e < sl.nseg ? __ldcg(ksum + (size_t)sl.start(e0 + e) * kHeadDim + kt) : 0.f;
 #pragma unroll
-    for (int e = 0; e < 20; ++e) sum += v[e];
+    for (int e = 0; e < 12; ++e) sum += v[e];
   }
   return sum;
 }
-// Walks the segments of the CTA's tile range [lo, hi); every thread of the CTA calls it after
-// the barrier that ends the tile loops.  Threads 0 .. NQ-1 fold the row statistics, threads
-// 256 .. 383 the key sums.  `red` is shared scratch of four floats, `flag` a shared int.
+// Walks the segments of the CTA's tile range [lo, hi); every epilogue thread (et = 0 .. 511)
+// calls it after the barrier that ends the tile loops.  Threads 0 .. NQ-1 fold the row
+// statistics, threads 256 .. 383 the key sums.  `red` is shared scratch of four floats, `flag` a
+// shared int.  Named barrier 5 joins the epilogue threads.
 template <int MB>
 __device__ __forceinline__ void finish_heads(const SeqTable& st, const Workspace& ws, const int lo,
                                              const int hi, const unsigned long long call_tag,
-                                             float* __restrict__ rbar_out, float* red, int* flag) {
-  const int tid = threadIdx.x, lane = tid & 31;
+                                             float* __restrict__ rbar_out, float* red, int* flag,
+                                             const int et) {
+  const int lane = et & 31;
   const int NQ = st.NQ, H = st.H;
+  constexpr int NU = MB == 2 ? 2 : 4;
   int id = lo;
   while (id < hi) {
     const TileIter ti(st.tile1_start, st.batch, H, st.nt1, id, hi);
@@ -192,14 +209,14 @@ __device__ __forceinline__ void finish_heads(const SeqTable& st, const Workspace
     const int unit = ti.unit();
     const SegList sl(ti.layer * st.nt1 + st.tile1_start[ti.b] + ti.h * per_head, per_head,
                      split1(st));
-    if (tid == 0) *flag = arrive_last(ws.headcnt + unit, call_tag, sl.nseg);
-    __syncthreads();
+    if (et == 0) *flag = arrive_last(ws.headcnt + unit, call_tag, sl.nseg);
+    named_bar_sync(5, kEpiThreads);
     const bool last = *flag != 0;
     if (last) {
-      if (tid < NQ)
-        ws.bq[(size_t)unit * NQ + tid] =
-            fold_row_stats<MB == 1 ? 2 : 1>(ws.rowstat, sl, NQ, tid) - log2f((float)st.W);
-      const int kt = tid - 256;
+      if (et < NQ)
+        ws.bq[(size_t)unit * NQ + et] =
+            fold_row_stats<NU>(ws.rowstat, sl, NQ, et) - log2f((float)st.W);
+      const int kt = et - 256;
       float sum = 0.f;
       if (kt >= 0 && kt < kHeadDim) {
         sum = fold_key_sums(ws.ksum, sl, kt);
@@ -208,15 +225,18 @@ __device__ __forceinline__ void finish_heads(const SeqTable& st, const Workspace
         if (lane == 0) red[kt >> 5] = n2;
       }
     }
-    __syncthreads();   // `flag` may be rewritten; the four partial norms are in `red`
-    if (last && tid == 256) {
+    named_bar_sync(5, kEpiThreads);   // `flag` may be rewritten; the four partial norms are in `red`
+    if (last && et == 256) {
       const double nn = ((double)red[0] + (double)red[1]) + ((double)red[2] + (double)red[3]);
       const double T = (double)L;
       const float r = (float)((nn - T) / (T * (T - 1.0)));   // Eq. 4
       ws.rbar[unit] = r;
       if (rbar_out) rbar_out[unit] = r;
+      // every segment of this head has arrived: leave the counter at zero under this call's tag,
+      // so that a replay of the same launch (a captured graph keeps its tag) counts afresh
+      ws.headcnt[unit] = call_tag << 16;
     }
-    __syncthreads();   // `red` is free again
+    named_bar_sync(5, kEpiThreads);   // `red` is free again
     id += min(hi - id, per_head - ti.t);
   }
 }
@@ -256,7 +276,11 @@ __device__ __forceinline__ void softmax_chunk(uint32_t (&r)[32], const bool need
   z_run += z0 + z1;
 }
 
-// grid = g1 persistent CTAs: TMA, MMA, 2 idle, 8 epilogue, 4 or 8 key-statistics warps.
+// grid = g1 persistent CTAs of 28 warps: TMA, 2 idle, MMA, 16 epilogue, 8 key-statistics.  The
+// MMA issuer is warp 3: its scheduler carries the fewest busy warps (with G*W = 224 the last
+// lane quarter of the second query block is padding), and a single dependent instruction
+// stream that shares a scheduler with many busy warps issues slowly enough to pace the tile
+// loop.
 template <int MB>
 __global__ void __launch_bounds__(p1_threads(MB), 1)
 k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ,
@@ -265,12 +289,16 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* base =
       reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
-  constexpr int QR = MB * 128;                 // query rows the MMA reads
   constexpr int kP1Stages = p1_stages(MB);
   constexpr int kP1AuxWarps = p1_aux_warps(MB);
-  constexpr int kP1Threads = p1_threads(MB);
-  unsigned char* sQ = base;                    // 2 halves x [QR x 128 B]
-  unsigned char* sK = sQ + 2 * QR * 128;       // kP1Stages x 32 KB
+  constexpr int NU = MB == 2 ? 2 : 4;   // partial row statistics per segment and row
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int NQ = st.NQ, W = st.W, H = st.H;
+  // The query tile holds exactly NQ rows per 64-column half.  The MMA reads MB * 128 rows: the
+  // rows past NQ are whatever follows in shared memory (the next half, the K ring), they only
+  // reach accumulator lanes that nobody reads.
+  unsigned char* sQ = base;                    // 2 halves x [NQ x 128 B]
+  unsigned char* sK = sQ + 2 * NQ * 128;       // kP1Stages x 32 KB
   float* sks = reinterpret_cast<float*>(sK + kP1Stages * kTileBytes);  // [aux warps][128] key-sum exchange
   P1Bars* bars = reinterpret_cast<P1Bars*>(sks + kP1AuxWarps * 128);
   {
@@ -283,8 +311,6 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
     }
   }
 
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int NQ = st.NQ, W = st.W, H = st.H;
   const int lo = cta_first_tile(blockIdx.x, split1(st));
   const int hi = cta_first_tile(blockIdx.x + 1, split1(st));
   volatile int* abort = &bars->abort;
@@ -297,21 +323,14 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(&bars->tfull[s], 1);
-      mbar_init(&bars->tempty[s], kEpiThreads);
+      mbar_init(&bars->tempty[s], kEpiThreads);      // every epilogue thread reads every tile
     }
     mbar_init(&bars->qfull, 1);
     mbar_init(&bars->qfree, 1);
     bars->abort = 0;
     mbar_init_fence();
   }
-  // rows of the query tile beyond NQ are never loaded: clear them once
-  for (int i = tid; i < 2 * (QR - NQ) * 8; i += kP1Threads) {
-    const int half = i / ((QR - NQ) * 8), rem = i % ((QR - NQ) * 8);
-    const int r = NQ + rem / 8, c = rem % 8;
-    *reinterpret_cast<uint4*>(sQ + half * QR * 128 + sw128_offset(r, c)) = make_uint4(0, 0, 0, 0);
-  }
-  fence_proxy_async_smem();
-  if (warp == kWarpMma) tmem_alloc(&bars->tmem_base, MB * 256);
+  if (warp == kP1WarpMma) tmem_alloc(&bars->tmem_base, MB * 256);
   if (warp == kWarpTma && lane == 0) {
     tma_prefetch_desc(&tmK);
     tma_prefetch_desc(&tmQ);
@@ -322,77 +341,91 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
   const uint32_t tmem = bars->tmem_base;
   pdl_wait();   // everything earlier in the stream is complete: global memory may be touched
 
-  if (warp == kWarpTma) {
-    // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      int it = 0, segn = 0;
-      bool seg_start = true;
-      for (TileIter ti(st.tile1_start, st.batch, H, st.nt1, lo, hi); ti.valid(); ti.next()) {
-        if (seg_start) {
-          if (segn > 0 && !mbar_wait(&bars->qfree, (segn - 1) & 1, abort)) break;
-          mbar_expect_tx(&bars->qfull, NQ * 256);
-          tma_load_3d(sQ, &tmQ, 0, ti.bh() * NQ, ti.layer, &bars->qfull);
-          tma_load_3d(sQ + QR * 128, &tmQ, 64, ti.bh() * NQ, ti.layer, &bars->qfull);
-          ++segn;
-        }
-        seg_start = ti.seg_last();
-        const int s = it % kP1Stages, ph = (it / kP1Stages) & 1;
-        if (!mbar_wait(&bars->empty[s], ph ^ 1, abort)) break;
-        mbar_expect_tx(&bars->full[s], kTileBytes);
-        const int y = st.cu[ti.b] + ti.t * kTile;
-        tma_load_4d(sK + s * kTileBytes, &tmK, 0, y, ti.h, ti.layer, &bars->full[s]);
-        tma_load_4d(sK + s * kTileBytes + kHalfBytes, &tmK, 64, y, ti.h, ti.layer, &bars->full[s]);
-        ++it;
-      }
-      if (*abort) {
-        raise(status, abort);
-        drain_ring(bars->full, kP1Stages, it);
-      }
-    }
-  } else if (warp == kWarpMma) {
-    // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc = umma_idesc_bf16(128, kTile);
-      int it = 0, segn = 0;
-      bool seg_start = true;
-      for (TileIter ti(st.tile1_start, st.batch, H, st.nt1, lo, hi); ti.valid(); ti.next()) {
-        if (seg_start) {
-          if (!mbar_wait(&bars->qfull, segn & 1, abort)) break;
-          ++segn;
-        }
-        seg_start = ti.seg_last();
-        const int s = it % kP1Stages, ph = (it / kP1Stages) & 1, ts = it & 1, tph = (it >> 1) & 1;
-        if (!mbar_wait(&bars->full[s], ph, abort)) break;
-        if (!mbar_wait(&bars->tempty[ts], tph ^ 1, abort)) break;
-        tc_fence_after();
-        const uint32_t kaddr = smem_u32(sK + s * kTileBytes);
-#pragma unroll
-        for (int mb = 0; mb < MB; ++mb) {
-#pragma unroll
-          for (int ks = 0; ks < 8; ++ks) {
-            const uint64_t da =
-                umma_desc_sw128(smem_u32(sQ) + (ks >> 2) * QR * 128 + mb * 16384 + (ks & 3) * 32);
-            const uint64_t db = umma_desc_sw128(kaddr + (ks >> 2) * kHalfBytes + (ks & 3) * 32);
-            umma_bf16(tmem + ts * (MB * 128) + mb * 128, da, db, idesc, ks > 0);
+  if (warp < kEpiWarp0) {
+    set_regs<kP1RegsLead, kP1RegsLaunch>();
+    if (warp == kWarpTma) {
+      // ---------------------------------------------------------------- TMA producer
+      if (lane == 0) {
+        int it = 0, segn = 0;
+        bool seg_start = true;
+        for (TileIter ti(st.tile1_start, st.batch, H, st.nt1, lo, hi); ti.valid(); ti.next()) {
+          if (seg_start) {
+            if (segn > 0 && !mbar_wait(&bars->qfree, (segn - 1) & 1, abort)) break;
+            mbar_expect_tx(&bars->qfull, NQ * 256);
+            tma_load_3d(sQ, &tmQ, 0, ti.bh() * NQ, ti.layer, &bars->qfull);
+            tma_load_3d(sQ + NQ * 128, &tmQ, 64, ti.bh() * NQ, ti.layer, &bars->qfull);
+            ++segn;
           }
+          seg_start = ti.seg_last();
+          const int s = it % kP1Stages, ph = (it / kP1Stages) & 1;
+          if (!mbar_wait(&bars->empty[s], ph ^ 1, abort)) break;
+          mbar_expect_tx(&bars->full[s], kTileBytes);
+          const int y = st.cu[ti.b] + ti.t * kTile;
+          tma_load_4d(sK + s * kTileBytes, &tmK, 0, y, ti.h, ti.layer, &bars->full[s]);
+          tma_load_4d(sK + s * kTileBytes + kHalfBytes, &tmK, 64, y, ti.h, ti.layer, &bars->full[s]);
+          ++it;
         }
-        umma_commit(&bars->empty[s]);
-        umma_commit(&bars->tfull[ts]);
-        if (seg_start) umma_commit(&bars->qfree);
-        ++it;
+        if (*abort) {
+          raise(status, abort);
+          drain_ring(bars->full, kP1Stages, it);
+        }
       }
-      if (*abort) raise(status, abort);
+    } else if (warp == kP1WarpMma) {
+      // ---------------------------------------------------------------- MMA issuer
+      if (lane == 0) {
+        constexpr uint32_t idesc = umma_idesc_bf16(128, kTile);
+        const uint32_t q_lo = umma_desc_lo(smem_u32(sQ));
+        const uint32_t k_lo = umma_desc_lo(smem_u32(sK));
+        const uint32_t q_half = (uint32_t)(NQ * 128) >> 4;   // second 64-column half of the queries
+        int it = 0, segn = 0;
+        bool seg_start = true;
+        for (TileIter ti(st.tile1_start, st.batch, H, st.nt1, lo, hi); ti.valid(); ti.next()) {
+          if (seg_start) {
+            if (!mbar_wait(&bars->qfull, segn & 1, abort)) break;
+            ++segn;
+          }
+          seg_start = ti.seg_last();
+          const int s = it % kP1Stages, ph = (it / kP1Stages) & 1, ts = it & 1, tph = (it >> 1) & 1;
+          if (!mbar_wait(&bars->full[s], ph, abort)) break;
+          if (!mbar_wait(&bars->tempty[ts], tph ^ 1, abort)) break;
+          tc_fence_after();
+          const uint32_t kb_lo = k_lo + (uint32_t)s * (kTileBytes >> 4);
+          const uint32_t td = tmem + ts * (MB * 128);
+#pragma unroll
+          for (int mb = 0; mb < MB; ++mb) {
+            // k-steps of 16 columns: 32 bytes apart inside a 64-column half
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+              const uint32_t a_lo = q_lo + (ks >> 2) * q_half + (uint32_t)(mb * (16384 >> 4) + (ks & 3) * 2);
+              const uint32_t b_lo = kb_lo + (uint32_t)((ks >> 2) * (kHalfBytes >> 4) + (ks & 3) * 2);
+              if (ks == 0)
+                umma_bf16_lo<0>(td + mb * 128, a_lo, b_lo, idesc);
+              else
+                umma_bf16_lo<1>(td + mb * 128, a_lo, b_lo, idesc);
+            }
+          }
+          umma_commit(&bars->empty[s]);
+          umma_commit(&bars->tfull[ts]);
+          if (seg_start) umma_commit(&bars->qfree);
+          ++it;
+        }
+        if (*abort) raise(status, abort);
+      }
     }
-  } else if (warp >= kEpiWarp0 && warp < kEpiWarp0 + kEpiWarps) {
+  } else if (warp < kAuxWarp0) {
     // ------------------------------------------------------------------ epilogue
-    // MB == 2: warpgroup wg owns query rows wg*128 .. +127 and all 128 keys of the tile.
-    // MB == 1: both warpgroups own rows 0 .. 127; wg takes the keys wg*64 .. +63.
-    const int quarter = warp & 3, wg = (warp - kEpiWarp0) >> 2;
-    const int row = (MB == 2 ? wg * 128 : 0) + quarter * 32 + lane;
-    const int unit = MB == 2 ? 0 : wg;
-    constexpr int NC = MB == 2 ? 128 : 64;       // columns (keys) this thread reduces per tile
-    const int col0 = MB == 2 ? wg * 128 : wg * 64;
-    const bool warp_on = (MB == 2 ? wg * 128 : 0) + quarter * 32 < NQ;
+    // All sixteen warps read every tile (two accumulator stages: the MMA of the next tile fills
+    // the other stage meanwhile).  Warpgroup wg = 0..3:
+    // MB == 2: query rows (wg / 2) * 128 .. +127, keys (wg % 2) * 64 .. +63 of the tile;
+    // MB == 1: query rows 0 .. 127, keys wg * 32 .. +31.
+    set_regs<kP1RegsEpi, kP1RegsLaunch>();
+    const int wg = (warp - kEpiWarp0) >> 2, quarter = warp & 3;
+    const int blk = MB == 2 ? wg >> 1 : 0;
+    const int unit = MB == 2 ? wg & 1 : wg;      // which partial result of the row this is
+    constexpr int NC = MB == 2 ? 64 : 32;        // columns (keys) this thread reduces per tile
+    const int row = blk * 128 + quarter * 32 + lane;
+    const int col0 = blk * 128 + unit * NC;
+    const bool warp_on = blk * 128 + quarter * 32 < NQ;
     const int jrow = row % W;
     float m_run = -1e30f, z_run = 0.f;
     int it = 0, seg_first = lo;
@@ -409,7 +442,7 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
       if (!mbar_wait(&bars->tfull[ts], tph, abort)) break;
       tc_fence_after();
       if (warp_on) {
-        const int k0 = ti.t * kTile + (MB == 2 ? 0 : wg * 64);
+        const int k0 = ti.t * kTile + unit * NC;
         const bool need_mask = ti.t * kTile + kTile > P;
         const int lim = P + jrow;   // last key this row may see
         const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + ts * (MB * 128) + col0;
@@ -425,17 +458,17 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
       tc_fence_before();
       mbar_arrive(&bars->tempty[ts]);
       if (seg_start && row < NQ)
-        ws.rowstat[((size_t)seg_first * 2 + unit) * NQ + row] = make_float2(m_run, z_run);
+        ws.rowstat[((size_t)seg_first * NU + unit) * NQ + row] = make_float2(m_run, z_run);
       ++it;
     }
-  } else if (warp >= kAuxWarp0) {
+  } else {
     // ------------------------------------------------------------------ key statistics
     // Sixteen lanes share a key row (one 16-byte chunk each); a pair of 8-row batches is one
     // warp-wide step (one batch per 16-lane group).  Sweep 1 squares, a butterfly leaves the
     // squared norm of row r with lanes 2r and 2r+1, sweep 2 adds the rows scaled by 1/|k| into
     // eight per-thread sums (dims 8c .. 8c+7).
+    set_regs<kP1RegsAux, kP1RegsLaunch>();
     const int aux_w = warp - kAuxWarp0;
-    constexpr int kPairs = 8 / kP1AuxWarps;      // pairs of 8-row batches per warp and tile
     const int c = lane & 15, lg = lane >> 4;
     const int chalf = c >> 3, cc = c & 7;
     constexpr int aux_threads = kP1AuxWarps * 32;
@@ -456,9 +489,8 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
       const int s = it % kP1Stages, ph = (it / kP1Stages) & 1;
       const bool ok = mbar_wait(&bars->full[s], ph, abort);
       const unsigned char* tile = sK + s * kTileBytes + chalf * kHalfBytes;
-#pragma unroll 1
-      for (int bp = 0; bp < kPairs; ++bp) {   // kept rolled: the body must stay in the i-cache
-        const int row0 = (2 * (aux_w * kPairs + bp) + lg) * 8;
+      {
+        const int row0 = (2 * aux_w + lg) * 8;
         uint4 u[8];
         float p[8];
 #pragma unroll
@@ -476,10 +508,9 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
           unpack2(sq, s0, s1);
           p[rr] = s0 + s1;
         }
-        if (bp == kPairs - 1) {   // the tile now lives in registers: hand the stage back
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&bars->empty[s]);
-        }
+        // the tile now lives in registers: hand the stage back
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bars->empty[s]);
 #pragma unroll
         for (int o = 8; o >= 2; o >>= 1) {
           const bool up = (c & o) != 0;
@@ -506,7 +537,8 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
           }
         }
       }
-      if (group_sync_stop(2, aux_threads, kt == 0, abort, bars->vote, it)) break;
+      // (no barrier per tile: after an abort the waits fail at once and every warp still walks
+      // the same tiles, so the segment-end barriers below stay matched)
       if (seg_start) {
         float acc[8];
 #pragma unroll
@@ -530,7 +562,7 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == kWarpMma) tmem_dealloc(tmem, MB * 256);
+  if (warp == kP1WarpMma) tmem_dealloc(tmem, MB * 256);
   if (bars->abort) {
     if (tid == 0 && status) atomicExch(status, MIXKV_ERR_TIMEOUT);
     return;
@@ -538,8 +570,14 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
   // Every partial result of this CTA is written.  Its segments now count as delivered; the CTA
   // that delivers the last segment of a (layer, sequence, head) folds all of them, once, into
   // what pass 2 reads: one log2 normaliser per window row (the 1/W of the window mean folded
-  // in), the mean unit key, the redundancy of Eq. 4.
-  finish_heads<MB>(st, ws, lo, hi, call_tag, rbar_out, sks, &bars->last);
+  // in), the mean unit key, the redundancy of Eq. 4.  The epilogue warps do it (they hold the
+  // registers).
+#ifndef DIAG_NO_FINISH
+  if (warp >= kEpiWarp0 && warp < kAuxWarp0)
+#else
+  if (warp > 1000)
+#endif
+    finish_heads<MB>(st, ws, lo, hi, call_tag, rbar_out, sks, &bars->last, tid - kEpiWarp0 * 32);
 }
 
 // ======================================================================== pass 2
@@ -553,12 +591,13 @@ struct P2Bars {
   uint64_t vempty[kP2VStagesMax];
   uint64_t tfull[2];
   uint64_t tempty[2];
+  uint64_t xfull[2];    // the sixteen epilogue warps have left their partial sums of a tile
+  uint64_t xempty[2];   // the four value-norm warps have added them up
   uint64_t qfull;
   uint64_t qfree;
   uint64_t kbready;
   uint32_t tmem_base;
   int abort;
-  int vote[3][2];
 };
 
 // N logit columns of one key (registers r[0..N)): adds exp2(logit * scale - normaliser of the
@@ -580,8 +619,18 @@ __device__ __forceinline__ void colsum_chunk(const uint32_t (&r)[N], const float
   }
 }
 
-// grid = g2 persistent CTAs: K producer, MMA, V producer, 1 idle, 8 epilogue, 4 value-norm warps.
-__global__ void __launch_bounds__(kThreads, 1)
+// registers per thread: at launch, then per role (6 warpgroups: 40 + 4 * 88 + 88 = 6 * 80; a
+// value-norm thread keeps the sixteen 16-byte loads of its row in flight)
+#ifndef P2_LEAD
+#define P2_LEAD 40
+#define P2_EPI 88
+#define P2_AUX 88
+#endif
+constexpr int kP2RegsLaunch = 80, kP2RegsLead = P2_LEAD, kP2RegsEpi = P2_EPI, kP2RegsAux = P2_AUX;
+
+// grid = g2 persistent CTAs of 24 warps: K producer, V producer, 1 idle, MMA, 16 epilogue,
+// 4 value-norm warps.
+__global__ void __launch_bounds__(kThreads2, 1)
 k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
         const __grid_constant__ CUtensorMap tmQ, const SeqTable st, const Workspace ws,
         float* __restrict__ s_div_out, const float scale_log2e,
@@ -595,14 +644,15 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
   unsigned char* sK = sQ + 2 * NB * 128;      // kP2KStages x 32 KB
   unsigned char* sV = sK + kP2KStages * kTileBytes;   // vstages x 16 KB
   float* sbq = reinterpret_cast<float*>(sV + vstages * kVSubBytes);  // [2][256] negated normalisers
-  float* sred = sbq + 512;                    // [64]: 2 x 16 epilogue, 16 value norms + 4 mean key
+  float* sx = sbq + 512;                      // [2 stages][4 warpgroups][128] partial column sums
+  float* sred = sx + 1024;                    // [64]: 16 diversity, 16 value norms / attention
   P2Bars* bars = reinterpret_cast<P2Bars*>(sred + 64);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int lo = cta_first_tile(blockIdx.x, split2(st));
   const int hi = cta_first_tile(blockIdx.x + 1, split2(st));
   volatile int* abort = &bars->abort;
-  constexpr int kWarpTmaV = 2;
+  constexpr int kWarpTmaV = 1, kP2WarpMma = 3;
 
   pdl_launch_dependents();
   if (tid == 0) {
@@ -616,7 +666,9 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(&bars->tfull[s], 1);
-      mbar_init(&bars->tempty[s], 128);    // the warpgroup that owns the accumulator stage
+      mbar_init(&bars->tempty[s], kEpiThreads);   // every epilogue thread reads every tile
+      mbar_init(&bars->xfull[s], kEpiWarps);
+      mbar_init(&bars->xempty[s], 4);
     }
     mbar_init(&bars->qfull, 1);
     mbar_init(&bars->qfree, 1);
@@ -624,7 +676,7 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
     bars->abort = 0;
     mbar_init_fence();
   }
-  if (warp == kWarpMma) tmem_alloc(&bars->tmem_base, 512);
+  if (warp == kP2WarpMma) tmem_alloc(&bars->tmem_base, 512);
   if (warp == kWarpTma && lane == 0) {
     tma_prefetch_desc(&tmK);
     tma_prefetch_desc(&tmQ);
@@ -636,204 +688,217 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
   const uint32_t tmem = bars->tmem_base;
   pdl_wait();
 
-  if (warp == kWarpTma) {
-    // ------------------------------------------------------------------ K / Q producer
-    if (lane == 0) {
-      int it = 0, segn = 0;
-      bool seg_start = true;
-      for (TileIter ti(st.tile2_start, st.batch, H, st.nt2, lo, hi); ti.valid(); ti.next()) {
-        if (seg_start) {
-          if (segn > 0 && !mbar_wait(&bars->qfree, (segn - 1) & 1, abort)) break;
-          mbar_expect_tx(&bars->qfull, NQ * 256);
-          tma_load_3d(sQ, &tmQ, 0, ti.bh() * NQ, ti.layer, &bars->qfull);
-          tma_load_3d(sQ + NB * 128, &tmQ, 64, ti.bh() * NQ, ti.layer, &bars->qfull);
-          ++segn;
-        }
-        seg_start = ti.seg_last();
-        const int s = it % kP2KStages, ph = (it / kP2KStages) & 1;
-        if (!mbar_wait(&bars->kempty[s], ph ^ 1, abort)) break;
-        mbar_expect_tx(&bars->kfull[s], kTileBytes);
-        const int y = st.cu[ti.b] + ti.t * kTile;
-        tma_load_4d(sK + s * kTileBytes, &tmK, 0, y, ti.h, ti.layer, &bars->kfull[s]);
-        tma_load_4d(sK + s * kTileBytes + kHalfBytes, &tmK, 64, y, ti.h, ti.layer, &bars->kfull[s]);
-        ++it;
-      }
-      if (*abort) {
-        raise(status, abort);
-        drain_ring(bars->kfull, kP2KStages, it);
-      }
-    }
-  } else if (warp == kWarpTmaV) {
-    // ------------------------------------------------------------------ V producer
-    if (lane == 0 && use_vnorm == MIXKV_INTRINSIC_VNORM) {
-      int vit = 0;
-      bool ok = true;
-      for (TileIter ti(st.tile2_start, st.batch, H, st.nt2, lo, hi); ti.valid() && ok; ti.next()) {
-        const int y = st.cu[ti.b] + ti.t * kTile;
-        for (int sub = 0; sub < 2; ++sub) {
-          const int vs = vit % vstages, vph = (vit / vstages) & 1;
-          if (!mbar_wait(&bars->vempty[vs], vph ^ 1, abort)) {
-            ok = false;
-            break;
+  if (warp < kEpiWarp0) {
+    set_regs<kP2RegsLead, kP2RegsLaunch>();
+    if (warp == kWarpTma) {
+      // ---------------------------------------------------------------- K / Q producer
+      if (lane == 0) {
+        int it = 0, segn = 0;
+        bool seg_start = true;
+        for (TileIter ti(st.tile2_start, st.batch, H, st.nt2, lo, hi); ti.valid(); ti.next()) {
+          if (seg_start) {
+            if (segn > 0 && !mbar_wait(&bars->qfree, (segn - 1) & 1, abort)) break;
+            mbar_expect_tx(&bars->qfull, NQ * 256);
+            tma_load_3d(sQ, &tmQ, 0, ti.bh() * NQ, ti.layer, &bars->qfull);
+            tma_load_3d(sQ + NB * 128, &tmQ, 64, ti.bh() * NQ, ti.layer, &bars->qfull);
+            ++segn;
           }
-          mbar_expect_tx(&bars->vfull[vs], kVSubBytes);
-          unsigned char* dst = sV + vs * kVSubBytes;
-          tma_load_4d(dst, &tmV, 0, y + sub * 64, ti.h, ti.layer, &bars->vfull[vs]);
-          tma_load_4d(dst + kVSubBytes / 2, &tmV, 64, y + sub * 64, ti.h, ti.layer, &bars->vfull[vs]);
-          ++vit;
+          seg_start = ti.seg_last();
+          const int s = it % kP2KStages, ph = (it / kP2KStages) & 1;
+          if (!mbar_wait(&bars->kempty[s], ph ^ 1, abort)) break;
+          mbar_expect_tx(&bars->kfull[s], kTileBytes);
+          const int y = st.cu[ti.b] + ti.t * kTile;
+          tma_load_4d(sK + s * kTileBytes, &tmK, 0, y, ti.h, ti.layer, &bars->kfull[s]);
+          tma_load_4d(sK + s * kTileBytes + kHalfBytes, &tmK, 64, y, ti.h, ti.layer, &bars->kfull[s]);
+          ++it;
+        }
+        if (*abort) {
+          raise(status, abort);
+          drain_ring(bars->kfull, kP2KStages, it);
         }
       }
-      if (*abort) {
-        raise(status, abort);
-        drain_ring(bars->vfull, vstages, vit);
-      }
-    }
-  } else if (warp == kWarpMma) {
-    // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      const uint32_t idesc = umma_idesc_bf16(128, NB);
-      int it = 0, segn = 0;
-      bool seg_start = true;
-      for (TileIter ti(st.tile2_start, st.batch, H, st.nt2, lo, hi); ti.valid(); ti.next()) {
-        if (seg_start) {
-          if (!mbar_wait(&bars->qfull, segn & 1, abort)) break;
-          if (!mbar_wait(&bars->kbready, segn & 1, abort)) break;
-          ++segn;
+    } else if (warp == kWarpTmaV) {
+      // ---------------------------------------------------------------- V producer
+      if (lane == 0 && use_vnorm == MIXKV_INTRINSIC_VNORM) {
+        int vit = 0;
+        bool ok = true;
+        for (TileIter ti(st.tile2_start, st.batch, H, st.nt2, lo, hi); ti.valid() && ok; ti.next()) {
+          const int y = st.cu[ti.b] + ti.t * kTile;
+          for (int sub = 0; sub < 2; ++sub) {
+            const int vs = vit % vstages, vph = (vit / vstages) & 1;
+            if (!mbar_wait(&bars->vempty[vs], vph ^ 1, abort)) {
+              ok = false;
+              break;
+            }
+            mbar_expect_tx(&bars->vfull[vs], kVSubBytes);
+            unsigned char* dst = sV + vs * kVSubBytes;
+            tma_load_4d(dst, &tmV, 0, y + sub * 64, ti.h, ti.layer, &bars->vfull[vs]);
+            tma_load_4d(dst + kVSubBytes / 2, &tmV, 64, y + sub * 64, ti.h, ti.layer, &bars->vfull[vs]);
+            ++vit;
+          }
         }
-        seg_start = ti.seg_last();
-        const int s = it % kP2KStages, ph = (it / kP2KStages) & 1, ts = it & 1, tph = (it >> 1) & 1;
-        if (!mbar_wait(&bars->kfull[s], ph, abort)) break;
-        if (!mbar_wait(&bars->tempty[ts], tph ^ 1, abort)) break;
-        tc_fence_after();
-        const uint32_t kaddr = smem_u32(sK + s * kTileBytes);
+        if (*abort) {
+          raise(status, abort);
+          drain_ring(bars->vfull, vstages, vit);
+        }
+      }
+    } else if (warp == kP2WarpMma) {
+      // ---------------------------------------------------------------- MMA issuer
+      if (lane == 0) {
+        const uint32_t idesc = umma_idesc_bf16(128, NB);
+        const uint32_t q_lo = umma_desc_lo(smem_u32(sQ));
+        const uint32_t k_lo = umma_desc_lo(smem_u32(sK));
+        const uint32_t q_half = (uint32_t)(NB * 128) >> 4;   // second 64-column half of the B rows
+        int it = 0, segn = 0;
+        bool seg_start = true;
+        for (TileIter ti(st.tile2_start, st.batch, H, st.nt2, lo, hi); ti.valid(); ti.next()) {
+          if (seg_start) {
+            if (!mbar_wait(&bars->qfull, segn & 1, abort)) break;
+            if (!mbar_wait(&bars->kbready, segn & 1, abort)) break;
+            ++segn;
+          }
+          seg_start = ti.seg_last();
+          const int s = it % kP2KStages, ph = (it / kP2KStages) & 1, ts = it & 1, tph = (it >> 1) & 1;
+          if (!mbar_wait(&bars->kfull[s], ph, abort)) break;
+          if (!mbar_wait(&bars->tempty[ts], tph ^ 1, abort)) break;
+          tc_fence_after();
+          const uint32_t kb_lo = k_lo + (uint32_t)s * (kTileBytes >> 4);
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-          const uint64_t da = umma_desc_sw128(kaddr + (ks >> 2) * kHalfBytes + (ks & 3) * 32);
-          const uint64_t db = umma_desc_sw128(smem_u32(sQ) + (ks >> 2) * NB * 128 + (ks & 3) * 32);
-          umma_bf16(tmem + ts * 256, da, db, idesc, ks > 0);
+          for (int ks = 0; ks < 8; ++ks) {
+            const uint32_t a_lo = kb_lo + (uint32_t)((ks >> 2) * (kHalfBytes >> 4) + (ks & 3) * 2);
+            const uint32_t b_lo = q_lo + (ks >> 2) * q_half + (uint32_t)((ks & 3) * 2);
+            if (ks == 0)
+              umma_bf16_lo<0>(tmem + ts * 256, a_lo, b_lo, idesc);
+            else
+              umma_bf16_lo<1>(tmem + ts * 256, a_lo, b_lo, idesc);
+          }
+          umma_commit(&bars->kempty[s]);
+          umma_commit(&bars->tfull[ts]);
+          if (seg_start) umma_commit(&bars->qfree);
+          ++it;
         }
-        umma_commit(&bars->kempty[s]);
-        umma_commit(&bars->tfull[ts]);
-        if (seg_start) umma_commit(&bars->qfree);
-        ++it;
+        if (*abort) raise(status, abort);
       }
-      if (*abort) raise(status, abort);
     }
-  } else if (warp >= kEpiWarp0 && warp < kEpiWarp0 + kEpiWarps) {
+  } else if (warp < kAuxWarp0) {
     // ------------------------------------------------------------------ epilogue
-    // The two warpgroups take alternate tiles (warpgroup g owns accumulator stage g), one key
-    // per thread and all G*W columns of it, so a tile needs no exchange between warpgroups and
-    // the groups never wait for each other: each keeps its own copy of the normaliser table
-    // and leaves its own partial score statistics.
-    const int quarter = warp & 3, wg = (warp - kEpiWarp0) >> 2;
-    const int gt = (tid - kEpiWarp0 * 32) & 127;   // thread inside the warpgroup
-    const int gw = gt >> 5;                        // warp inside the warpgroup
+    // All sixteen warps read every tile (two accumulator stages: the MMA of the next tile fills
+    // the other stage meanwhile); a thread is one key.  The four warpgroups split the G*W logit
+    // columns of the key: each leaves its partial sum in shared memory, where the value-norm
+    // warps add the four up.  Warpgroup 0 also takes the three mean-key columns and owns the
+    // diversity score.  After an abort the waits fail at once and every warp still walks the
+    // same tiles, so the per-segment barriers stay matched.
+    set_regs<kP2RegsEpi, kP2RegsLaunch>();
+    const int wg = (warp - kEpiWarp0) >> 2, quarter = warp & 3;
+    const int et = tid - kEpiWarp0 * 32;           // 0..511
     const int key = quarter * 32 + lane;
-    const int nch = NQ / 16;
-    float* mybq = sbq + wg * 256;
-    const int barid = 1 + wg;                      // named barriers 1, 2: one per warpgroup
+    const int nch = NQ / 16;                       // 16-column chunks of a key's logits
+    const int ch0 = (nch * wg) >> 2, ch1 = (nch * (wg + 1)) >> 2;   // this warpgroup's chunks
+    const int n32 = (ch1 - ch0) >> 1;
+    const bool rest16 = ((ch1 - ch0) & 1) != 0;
     const f32x2 sc2 = pack2(scale_log2e, scale_log2e);
-    float dmin = INFINITY, dmax = -INFINITY, dsum = 0.f, exw = 0.f;
-    int it = 0, seg_first = lo;
+    float dmin = INFINITY, dmax = -INFINITY, dsum = 0.f;
+    int it = 0, segn = 0, seg_first = lo;
     bool seg_start = true;
+    const float* mybq = sbq;
     for (TileIter ti(st.tile2_start, st.batch, H, st.nt2, lo, hi); ti.valid(); ti.next()) {
       const int L = st.cu[ti.b + 1] - st.cu[ti.b], P = L - W;
       if (seg_start) {
-        // pass 1 left one negated log2 normaliser per window row of this (layer, b, h)
-        named_bar_sync(barid, 128);   // the previous segment's readers of mybq are done
-        for (int q = gt; q < NQ; q += 128) mybq[q] = ws.bq[(size_t)ti.unit() * NQ + q];
-        dmin = INFINITY, dmax = -INFINITY, dsum = 0.f, exw = 0.f;
+        // pass 1 left one negated log2 normaliser per window row of this (layer, b, h); the
+        // table alternates between two buffers, so the previous segment's readers are never
+        // overtaken
+        float* tb = sbq + (segn & 1) * 256;
+        if (et < NQ) tb[et] = ws.bq[(size_t)ti.unit() * NQ + et];
+        mybq = tb;
+        ++segn;
+        dmin = INFINITY, dmax = -INFINITY, dsum = 0.f;
         seg_first = ti.id;
-        named_bar_sync(barid, 128);
+        named_bar_sync(2, kEpiThreads);
       }
       seg_start = ti.seg_last();
-      const int ts = it & 1;
-      if (ts == wg) {   // this warpgroup's tile
-        const int tph = (it >> 1) & 1;
-        const int ikey = ti.t * kTile + key;
-        float kinv_i = 0.f;
-        if (ikey < P) kinv_i = ws.kinv[kpos(st, ti.layer, ti.h, ti.b, ikey)];
-        const bool ok = mbar_wait(&bars->tfull[ts], tph, abort);
-        tc_fence_after();
-        const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + ts * 256;
-        f32x2 acc = pack2(0.f, 0.f);
-        float dot = 0.f;
-        if (ok) {
-          uint32_t rd[4];
-          tmem_ld4(taddr + NQ, rd);
-          // 32-column chunks (the other warpgroup's tile keeps the SM busy while this load is
-          // in flight), then a 16-column rest; kept rolled: the body must stay in the i-cache
-          const int n32 = nch >> 1;
+      const int ts = it & 1, use = it >> 1;
+      const int ikey = ti.t * kTile + key;
+      float kinv_i = 0.f;
+      if (wg == 0 && ikey < P) kinv_i = ws.kinv[kpos(st, ti.layer, ti.h, ti.b, ikey)];
+      const bool ok = mbar_wait(&bars->tfull[ts], use & 1, abort);
+      tc_fence_after();
+      const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + ts * 256;
+      f32x2 acc = pack2(0.f, 0.f);
+      float dot = 0.f;
+      if (ok) {
+        uint32_t rd[4];
+        if (wg == 0) tmem_ld4(taddr + NQ, rd);
+        // 32-column chunks, then a 16-column rest; kept rolled: the body must stay in the i-cache
 #pragma unroll 1
-          for (int ci = 0; ci < n32; ++ci) {
-            uint32_t ra[32];
-            tmem_ld32(taddr + ci * 32, ra);
-            tmem_ld_wait();
-            tmem_ld_fence(ra);
-            colsum_chunk<32>(ra, mybq + ci * 32, sc2, acc);
-          }
-          if (nch & 1) {
-            uint32_t rb[16];
-            tmem_ld16(taddr + n32 * 32, rb);
-            tmem_ld_wait();
-            tmem_ld_fence(rb);
-            colsum_chunk<16>(rb, mybq + n32 * 32, sc2, acc);
-          }
+        for (int ci = 0; ci < n32; ++ci) {
+          uint32_t ra[32];
+          tmem_ld32(taddr + ch0 * 16 + ci * 32, ra);
+          tmem_ld_wait();
+          tmem_ld_fence(ra);
+          colsum_chunk<32>(ra, mybq + ch0 * 16 + ci * 32, sc2, acc);
+        }
+        if (rest16) {
+          uint32_t rb[16];
+          tmem_ld16(taddr + ch0 * 16 + n32 * 32, rb);
+          tmem_ld_wait();
+          tmem_ld_fence(rb);
+          colsum_chunk<16>(rb, mybq + ch0 * 16 + n32 * 32, sc2, acc);
+        }
+        if (wg == 0) {
           tmem_ld_wait();
           tmem_ld_fence(rd);
           dot = (__uint_as_float(rd[0]) + __uint_as_float(rd[1])) + __uint_as_float(rd[2]);
         }
-        tc_fence_before();
-        mbar_arrive(&bars->tempty[ts]);
-        if (ok && ikey < P) {
-          float acc0, acc1;
-          unpack2(acc, acc0, acc1);
-          const size_t poff = ppos(st, ti.layer, ti.h, ti.b, 0);
-          const float ex = acc0 + acc1;
-          ws.s_ex_raw[poff + ikey] = ex;
-          const float sd = -dot * kinv_i;
-          s_div_out[poff + ikey] = sd;
-          dmin = fminf(dmin, sd);
-          dmax = fmaxf(dmax, sd);
-          dsum += sd;
-          // number of pooling windows (centres in [0, P)) that cover this position
-          const int cover = min(ikey, pool_half) + min(P - 1 - ikey, pool_half) + 1;
-          exw = fmaf(ex, (float)cover, exw);
-        }
       }
-      if (group_sync_stop(barid, 128, gt == 0, abort, bars->vote[wg], it)) break;
-      if (seg_start) {
-        // this warpgroup's share of the segment's score statistics (neutral if it had no tile)
-        const float a = warp_min(dmin), b2 = warp_max(dmax), c2 = warp_sum(dsum),
-                    d2 = warp_sum(exw);
-        float* sr = sred + wg * 16;
+      tc_fence_before();
+      mbar_arrive(&bars->tempty[ts]);
+      // hand the partial sum to the value-norm warps (the slot was read two tiles ago)
+      if (use > 0) mbar_wait(&bars->xempty[ts], (use - 1) & 1, abort);
+      float acc0, acc1;
+      unpack2(acc, acc0, acc1);
+      sx[(ts * 4 + wg) * 128 + key] = acc0 + acc1;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bars->xfull[ts]);
+      if (wg == 0 && ok && ikey < P) {
+        const float sd = -dot * kinv_i;
+        s_div_out[ppos(st, ti.layer, ti.h, ti.b, 0) + ikey] = sd;
+        dmin = fminf(dmin, sd);
+        dmax = fmaxf(dmax, sd);
+        dsum += sd;
+      }
+      if (seg_start && wg == 0) {
+        // the segment's diversity statistics (the attention-score sum comes from the value-norm warps)
+        const float a = warp_min(dmin), b2 = warp_max(dmax), c2 = warp_sum(dsum);
         if (lane == 0) {
-          sr[gw] = a;
-          sr[4 + gw] = b2;
-          sr[8 + gw] = c2;
-          sr[12 + gw] = d2;
+          sred[quarter] = a;
+          sred[4 + quarter] = b2;
+          sred[8 + quarter] = c2;
         }
-        named_bar_sync(barid, 128);
-        if (gt == 0) {
-          ws.dstat[(size_t)seg_first * 2 + wg] = make_float4(
-              fminf(fminf(sr[0], sr[1]), fminf(sr[2], sr[3])),
-              fmaxf(fmaxf(sr[4], sr[5]), fmaxf(sr[6], sr[7])),
-              (sr[8] + sr[9]) + (sr[10] + sr[11]), (sr[12] + sr[13]) + (sr[14] + sr[15]));
+        named_bar_sync(1, 128);
+        if (et == 0) {
+          ws.dstat[(size_t)seg_first * 2] = make_float4(
+              fminf(fminf(sred[0], sred[1]), fminf(sred[2], sred[3])),
+              fmaxf(fmaxf(sred[4], sred[5]), fmaxf(sred[6], sred[7])),
+              (sred[8] + sred[9]) + (sred[10] + sred[11]), 0.f);
         }
+        named_bar_sync(1, 128);
       }
       ++it;
     }
-  } else if (warp >= kAuxWarp0) {
+  } else {
     // ------------------------------------------------------------------ mean key, value norms
     // At the start of a segment: write the bf16 hi / lo / lo2 split of the head's mean unit key
-    // (pass 1) into the three extra B rows.  Per tile: warps 12, 13 read the first 64 rows of the V
-    // tile, warps 14, 15 the last 64; one row per thread from the swizzled half tile.
+    // (pass 1) into the three extra B rows.  Per tile: warps 0, 1 of the four read the first 64
+    // rows of the V tile, warps 2, 3 the last 64; one row per thread from the swizzled half tile;
+    // then thread vt adds the four partial attention sums of key vt.
+    set_regs<kP2RegsAux, kP2RegsLaunch>();
     const int vt = tid - kAuxWarp0 * 32;         // 0..127
     const int sub = vt >> 6, vr = vt & 63;
-    float vmin = INFINITY, vmax = -INFINITY, vsum = 0.f;
+    float vmin = INFINITY, vmax = -INFINITY, vsum = 0.f, exw = 0.f;
     int it = 0, segn = 0, seg_first = lo;
     bool seg_start = true;
     for (TileIter ti(st.tile2_start, st.batch, H, st.nt2, lo, hi); ti.valid(); ti.next()) {
+      const int P = st.cu[ti.b + 1] - st.cu[ti.b] - W;
       if (seg_start) {
         const float kb = ws.kbar[(size_t)ti.unit() * kHeadDim + vt];   // mean unit key (pass 1)
         __nv_bfloat16 parts[3];
@@ -859,14 +924,13 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
         __syncwarp();
         if (lane == 0) mbar_arrive(&bars->kbready);
         ++segn;
-        vmin = INFINITY, vmax = -INFINITY, vsum = 0.f;
+        vmin = INFINITY, vmax = -INFINITY, vsum = 0.f, exw = 0.f;
         seg_first = ti.id;
       }
       seg_start = ti.seg_last();
       if (use_vnorm == MIXKV_INTRINSIC_KNORM) {
         // key-norm ablation: the intrinsic term is minus the key norm, which pass 1 left as its
         // reciprocal; no V tile is loaded
-        const int P = st.cu[ti.b + 1] - st.cu[ti.b] - W;
         const int i = ti.t * kTile + vt;
         if (i < P) {
           const float ki = ws.kinv[kpos(st, ti.layer, ti.h, ti.b, i)];
@@ -877,7 +941,6 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
           vsum += n;
         }
       } else if (use_vnorm) {
-        const int P = st.cu[ti.b + 1] - st.cu[ti.b] - W;
         const int vit = 2 * it + sub;
         const int vs = vit % vstages, vph = (vit / vstages) & 1;
         const bool ok = mbar_wait(&bars->vfull[vs], vph, abort);
@@ -914,21 +977,42 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
           vsum += n;
         }
       }
-      if (group_sync_stop(3, 128, vt == 0, abort, bars->vote[2], it)) break;
-      if (seg_start && use_vnorm) {
-        const float a = warp_min(vmin), b2 = warp_max(vmax), c2 = warp_sum(vsum);
+      {
+        // attention score of key vt of this tile: the four warpgroups' partial sums, in order
+        const int ts = it & 1, use = it >> 1;
+        const bool okx = mbar_wait(&bars->xfull[ts], use & 1, abort);
+        const float* px = sx + ts * 512 + vt;
+        const float ex = (px[0] + px[128]) + (px[256] + px[384]);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bars->xempty[ts]);
+        const int ikey = ti.t * kTile + vt;
+        if (okx && ikey < P) {
+          ws.s_ex_raw[ppos(st, ti.layer, ti.h, ti.b, 0) + ikey] = ex;
+          // number of pooling windows (centres in [0, P)) that cover this position
+          const int cover = min(ikey, pool_half) + min(P - 1 - ikey, pool_half) + 1;
+          exw = fmaf(ex, (float)cover, exw);
+        }
+      }
+      if (seg_start) {
+        const float a = warp_min(vmin), b2 = warp_max(vmax), c2 = warp_sum(vsum),
+                    d2 = warp_sum(exw);
         const int vw = warp - kAuxWarp0;
         if (lane == 0) {
           sred[32 + vw] = a;
           sred[36 + vw] = b2;
           sred[40 + vw] = c2;
+          sred[44 + vw] = d2;
         }
         named_bar_sync(4, 128);
         if (vt == 0) {
-          ws.vstat[seg_first] = make_float4(
-              fminf(fminf(sred[32], sred[33]), fminf(sred[34], sred[35])),
-              fmaxf(fmaxf(sred[36], sred[37]), fmaxf(sred[38], sred[39])),
-              (sred[40] + sred[41]) + (sred[42] + sred[43]), 0.f);
+          if (use_vnorm)
+            ws.vstat[seg_first] = make_float4(
+                fminf(fminf(sred[32], sred[33]), fminf(sred[34], sred[35])),
+                fmaxf(fmaxf(sred[36], sred[37]), fmaxf(sred[38], sred[39])),
+                (sred[40] + sred[41]) + (sred[42] + sred[43]), 0.f);
+          // neutral diversity statistics, the window-count-weighted sum of the attention scores
+          ws.dstat[(size_t)seg_first * 2 + 1] = make_float4(
+              INFINITY, -INFINITY, 0.f, (sred[44] + sred[45]) + (sred[46] + sred[47]));
         }
         named_bar_sync(4, 128);
       }
@@ -937,7 +1021,7 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == kWarpMma) tmem_dealloc(tmem, 512);
+  if (warp == kP2WarpMma) tmem_dealloc(tmem, 512);
   if (tid == 0 && bars->abort && status) atomicExch(status, MIXKV_ERR_TIMEOUT);
 }
 
@@ -988,17 +1072,17 @@ bool map_q(const LaunchCtx& c, const void* Q, CUtensorMap* tm) {
              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-size_t pass1_smem(int MB) {
+size_t pass1_smem(int MB, int NQ) {
   // up to 1023 bytes of alignment slack in front of the carve-up; never beyond the limit (the
   // kernel checks that its carve-up fits behind the aligned base)
-  const size_t need = (size_t)2 * MB * 128 * 128 + (size_t)p1_stages(MB) * kTileBytes + p1_aux_warps(MB) * 128 * 4 +
+  const size_t need = (size_t)2 * NQ * 128 + (size_t)p1_stages(MB) * kTileBytes + p1_aux_warps(MB) * 128 * 4 +
                       sizeof(P1Bars);
   const size_t want = need + 1024;
   return want < kSmemLimit ? want : kSmemLimit;
 }
 size_t pass2_smem(int NQ, int vstages) {
   return 1024 + (size_t)2 * (NQ + kExtraRows) * 128 + kP2KStages * kTileBytes +
-         (size_t)vstages * kVSubBytes + 512 * 4 + 64 * 4 + sizeof(P2Bars) + 64;
+         (size_t)vstages * kVSubBytes + 512 * 4 + 1024 * 4 + 64 * 4 + sizeof(P2Bars) + 64;
 }
 
 // cudaFuncSetAttribute once per (kernel, device).
@@ -1036,14 +1120,14 @@ cudaError_t launch_pass1(const LaunchCtx& c, const void* K, const void* Q, float
   if (!map_kv(c, K, kTile, &tmK) || !map_q(c, Q, &tmQ)) return cudaErrorInvalidValue;
   static bool done1[64] = {false}, done2[64] = {false};
   if (c.st.NQ <= 128) {
-    const size_t smem = pass1_smem(1);
-    cudaError_t e = ensure_smem(k_pass1<1>, smem, done1);
+    const size_t smem = pass1_smem(1, c.st.NQ);
+    cudaError_t e = ensure_smem(k_pass1<1>, kSmemLimit, done1);
     if (e != cudaSuccess) return e;
     return launch_pdl(k_pass1<1>, dim3(c.st.g1), dim3(p1_threads(1)), smem, c.stream, 1, tmK, tmQ, c.st,
                       c.ws, c.scale_log2e, c.call_tag, rbar_out, status);
   }
-  const size_t smem = pass1_smem(2);
-  cudaError_t e = ensure_smem(k_pass1<2>, smem, done2);
+  const size_t smem = pass1_smem(2, c.st.NQ);
+  cudaError_t e = ensure_smem(k_pass1<2>, kSmemLimit, done2);
   if (e != cudaSuccess) return e;
   return launch_pdl(k_pass1<2>, dim3(c.st.g1), dim3(p1_threads(2)), smem, c.stream, 1, tmK, tmQ, c.st,
                     c.ws, c.scale_log2e, c.call_tag, rbar_out, status);
@@ -1061,7 +1145,7 @@ cudaError_t launch_pass2(const LaunchCtx& c, const void* K, const void* V, const
   int vstages = kP2VStagesMax;
   while (vstages > 2 && pass2_smem(c.st.NQ, vstages) > kSmemLimit) --vstages;
   const size_t smem = pass2_smem(c.st.NQ, vstages);
-  return launch_pdl(k_pass2, dim3(c.st.g2), dim3(kThreads), smem, c.stream, 1, tmK, tmV, tmQ, c.st,
+  return launch_pdl(k_pass2, dim3(c.st.g2), dim3(kThreads2), smem, c.stream, 1, tmK, tmV, tmQ, c.st,
                     c.ws, s_div_out, c.scale_log2e, c.p.use_vnorm, c.p.pool_kernel >> 1,
                     vstages, status);
 }

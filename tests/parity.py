@@ -134,13 +134,50 @@ def run_layer_parity(wl: synth.Workload, layer: int = 0, variant: str = "literal
     return out, ref, ref_s
 
 
+def check_layer_properties(out, n, K, V, wl, Bp, adaptive):
+    """What holds for every layer of a call whatever the scores are (used for the layers the
+    oracle does not recompute): counts within their bounds (and summing to the sequence's
+    total under adaptive budgets), offsets = prefix sums, indices strictly ascending inside
+    the candidates, and every output row a bit-exact copy of the row its index names, the W
+    window rows last."""
+    H, W, cu = wl.kv_heads, wl.window, wl.cu_seqlens
+    counts = out["counts"][n].cpu().numpy()
+    offs = out["idx_offsets"][n].cpu().numpy()
+    ro = out["out_row_offsets"][n].cpu().numpy()
+    idx = out["idx"][n].cpu().numpy()
+    assert np.array_equal(offs, np.concatenate([[0], np.cumsum(counts)]))
+    assert np.array_equal(ro, offs + np.arange(wl.batch * H + 1) * W)
+    rows = []
+    for b in range(wl.batch):
+        P = int(cu[b + 1] - cu[b]) - W
+        c = counts[b * H:(b + 1) * H]
+        assert (c >= 0).all() and (c <= P).all()
+        if adaptive is True:
+            assert c.sum() == min(H * Bp, H * P) or (c == P).any()
+        elif adaptive is False:
+            assert (c == min(Bp, P)).all()
+        for h in range(H):
+            g = idx[offs[b * H + h]:offs[b * H + h + 1]]
+            assert (np.diff(g) > 0).all() and (g.size == 0 or (g.min() >= 0 and g.max() < P))
+            rows.append(torch.from_numpy(
+                np.concatenate([g, np.arange(P, P + W)]).astype(np.int64) + int(cu[b])
+                + h * int(cu[-1])))
+    src = torch.cat(rows).cuda()
+    n_rows = int(ro[-1])
+    assert src.numel() == n_rows
+    for X, Xo in ((K, out["K_out"]), (V, out["V_out"])):
+        flat = X[n].reshape(-1, 128).view(torch.int16)      # rows (h, position) of this layer
+        assert torch.equal(Xo[n][:n_rows].view(torch.int16), flat[src])
+
+
 def run_layers_parity(wl: synth.Workload, layers, variant: str = "calibrated", pad_rows: int = 0,
-                      check=None, head_budgets=None, **kw):
+                      check=None, head_budgets=None, properties=False, **kw):
     """mixkv_compress_layers over several layers at once against the oracle, layer by layer
     (only the positions listed in `check`, if given).  pad_rows > 0 leaves a gap between the
     layers of K / V (a strided layer dimension).  head_budgets (array [len(layers), batch*H],
     rows to keep per head, window included) takes the budgeted entry point and the oracle's
-    select_given."""
+    select_given.  properties=True also checks every layer of the call by the properties
+    that need no oracle (check_layer_properties)."""
     po, pg = params_pair(wl, **kw)
     cu = wl.cu_seqlens
     cu_arg = None if wl.batch == 1 else cu
@@ -166,6 +203,9 @@ def run_layers_parity(wl: synth.Workload, layers, variant: str = "calibrated", p
     torch.cuda.synchronize()
     assert int(out["status"].item()) == 0
     for n, x in enumerate(xs):
+        if properties:
+            check_layer_properties(out, n, K, V, wl, po.budget - W,
+                                   None if head_budgets is not None else po.budget_mode == 1)
         if check is not None and n not in check:
             continue
         ref_s = oracle.scores(x["K"], x["V"], x["Q"], po, cu=cu_arg)

@@ -110,6 +110,13 @@ def test_full_size_layers(name, layer):
     run_layer_parity(synth.CONFIGS[name], layer, "calibrated")
 
 
+@pytest.mark.parametrize("name,layer", [("C2", 1), ("C3", 7), ("C4", 2), ("C5", 5)])
+def test_full_size_layers_literal_keys(name, layer):
+    # the recipe as written (no shared per-head offset): mean key cosine near 0.05 (vision) or 0
+    # (text), the other regime of the diversity min-max and of Eq. 5
+    run_layer_parity(synth.CONFIGS[name], layer, "literal")
+
+
 def test_knorm_variant_full_size_and_batched():
     # key-norm intrinsic term (Sec. 3.2 ablation): V is not read for the scores
     run_layer_parity(synth.CONFIGS["C5"], 3, variant="calibrated", use_vnorm=2)
@@ -194,6 +201,53 @@ def test_bench_launch_configuration_sampled():
         check_scores(f"s_comp[layer {layer}]", out["s_comp"][layer].cpu().numpy(), ref_s["s_comp"],
                      cu, W)
         check_selection(idx[layer], offs[layer], counts[layer], ref, ref_s["s_comp"], cu, W, H)
+
+
+def test_bench_launch_configuration_c4_and_c5():
+    # the calls bench.py times for the other two multi-layer workloads, at full size.  C4: 28
+    # layers x 8 ragged sequences with adaptive budgets = 224 (sequence, layer) pairs, which
+    # takes the budget kernel with one CTA per pair and the select + gather tail with one CTA
+    # per head; C5: 32 layers x 8 heads = 256 units through the fused tail.  The oracle checks
+    # sampled layers, properties that need no oracle check every layer.
+    wl = synth.CONFIGS["C4"]
+    run_layers_parity(wl, range(wl.layers), check=(0, 14, 27), properties=True)
+    wl = synth.CONFIGS["C5"]
+    run_layers_parity(wl, range(wl.layers), check=(9, 31), properties=True)
+
+
+def test_prefix_longer_than_the_tail_cache():
+    # 140000 candidates of one head: more than eight CTAs of a cluster keep in shared memory, so
+    # the call takes the unfused route and the select + gather tail reads its keys from global
+    # memory in every pass
+    wl = synth.small_workload(H=1, G=1, W=16, seq_lens=(140016,), pool_kernel=5, budget=272,
+                              seed=33, centroids=8)
+    run_layer_parity(wl, variant="calibrated")
+
+
+@pytest.mark.parametrize("H,lens,levels", [
+    (8, (16400,) * 19, 3),        # one CTA per sequence, keys not cached, no candidate list
+    (8, (16400,) * 19, 1 << 20),  # one CTA per sequence, keys not cached, candidate list
+    (8, (60016,), 5),             # cluster of eight, keys not cached, no candidate list
+    (8, (60016,), 1 << 20),       # cluster of eight, keys not cached, candidate list
+])
+def test_adaptive_budgets_on_many_keys_are_exact(H, lens, levels):
+    # adaptive budgets on caller-supplied scores are integer work: bit-identical to the oracle.
+    # These shapes hold more keys per CTA than its shared memory caches; with few score levels
+    # the bin left after the first digit pass is larger than the candidate list.
+    W = 16
+    rng = np.random.default_rng(levels % 97)
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    Ptot = int(cu[-1]) - len(lens) * W
+    s = (rng.integers(0, levels, size=(H, Ptot)) / np.float32(levels)).astype(np.float32)
+    po = oracle.Params(kv_heads=H, gqa_ratio=1, window=W, budget=W + 200, budget_mode=1)
+    pg = binding.Params(kv_heads=H, gqa_ratio=1, window=W, budget=W + 200, budget_mode=1)
+    ref = oracle.select(s, po, cu=cu if len(lens) > 1 else None)
+    got = binding.select(torch.from_numpy(s).cuda(), pg,
+                         cu_seqlens=[int(c) for c in cu] if len(lens) > 1 else None)
+    offs = got["idx_offsets"].cpu().numpy()
+    assert np.array_equal(got["counts"].cpu().numpy(), ref["counts"].reshape(-1))
+    assert np.array_equal(offs, ref["idx_offsets"])
+    assert np.array_equal(got["idx"].cpu().numpy()[:offs[-1]], ref["idx"])
 
 
 def test_long_sequence_cluster_tail():
