@@ -49,6 +49,9 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-per-layer", action="store_true")
+    ap.add_argument("--min-seconds", type=float, default=1.0,
+                    help="repeat the block of --steps steps until this much has been timed")
+    ap.add_argument("--max-blocks", type=int, default=200)
     return ap.parse_args()
 
 
@@ -139,18 +142,21 @@ def run_reference(args):
         oracle.compress_layer(xs["K"], xs["V"], xs["Q"], pos, cu=cu)
         if s >= args.warmup:
             times.append(time.perf_counter() - t0)
-    per_layer = statistics.mean(times) * H / hs
-    step_s = per_layer * wl.layers          # a full step is all heads of all layers
+    sample_s = statistics.mean(times)       # what one timed step of this arm really ran
+    scale = (H / hs) * wl.layers            # a full step is all heads of all layers
+    step_s = sample_s * scale
     value = wl.total_tokens / step_s
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT,
             "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
-            "ms_per_step": step_s * 1e3, "higher_is_better": True, "scaling": "weak",
+            "ms_per_step": sample_s * 1e3, "sample_to_full_step_scale": scale,
+            "full_step_ms_scaled": step_s * 1e3, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": workload_config(wl, args.variant),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.threads(),
                              "kind": "oracle",
-                             "sample": f"{hs} of {H} KV heads of one layer per step, scaled to "
-                                       f"{H} heads x {wl.layers} layers"},
+                             "sample": f"each timed step is {hs} of {H} KV heads of layer 0 "
+                                       f"(ms_per_step is that sample's time); value scales it by "
+                                       f"{scale:g} to {H} heads x {wl.layers} layers"},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line), flush=True)
 
@@ -230,10 +236,10 @@ def cpu_baseline(wl, variant, budget_s=12.0):
                        pool_kernel=wl.pool_kernel, budget=wl.budget, budget_mode=wl.budget_mode,
                        ada_floor=wl.ada_floor)
     cu = None if wl.batch == 1 else wl.cu_seqlens
-    x = synth.make_layer(wl, 0, variant)
     oracle.lib()
     n, t_total = 0, 0.0
     while n < wl.layers and (t_total < budget_s or n < 1):
+        x = synth.make_layer(wl, n, variant)      # each layer's own tensors (drawn outside the timing)
         t0 = time.perf_counter()
         oracle.compress_layer(x["K"], x["V"], x["Q"], po, cu=cu)
         t_total += time.perf_counter() - t0
@@ -241,7 +247,8 @@ def cpu_baseline(wl, variant, budget_s=12.0):
     per_layer = t_total / n
     return {"value": wl.total_tokens / (per_layer * wl.layers), "unit": UNIT,
             "cores": oracle.threads(), "kind": "oracle",
-            "sample": f"{n} layer(s) of {wl.layers}, {t_total:.1f} s, scaled to all layers",
+            "sample": f"layers 0..{n - 1} of {wl.layers} (their own tensors), {t_total:.1f} s of "
+                      f"oracle time, scaled to all layers",
             "ms_per_layer": per_layer * 1e3}
 
 
@@ -345,9 +352,18 @@ def run_mixkv(args):
     if rank == 0:
         sampler.start()
         time.sleep(0.25)
-    ms_per_step = timed(step, 0, args.steps)
+    # A block is exactly --steps steps between two barriers.  Blocks are repeated until about
+    # --min-seconds of steps have been timed, so that the figure is the sustained one (clocks
+    # and power settle over hundreds of milliseconds); the line carries the median block, the
+    # best block and what the clocks did meanwhile.
+    blocks = [timed(step, 0, args.steps)]
+    n_blocks = int(min(args.max_blocks, max(1, np.ceil(args.min_seconds * 1e3 / (blocks[0] * args.steps)))))
+    n_blocks = int(max_over_ranks(float(n_blocks), world, dev))
+    for _ in range(n_blocks - 1):
+        blocks.append(timed(step, 0, args.steps))
     clocks = sampler.stop() if rank == 0 else None
     check_status()
+    ms_per_step = statistics.median(blocks)
     value = whole_job_value(wl.total_tokens, world, ms_per_step)
 
     # ---- per-kernel CUDA-event times: every kernel of a step bracketed by events on the
@@ -411,6 +427,12 @@ def run_mixkv(args):
                   f"(> 126 MB L2) between two uses of a buffer",
             "launch": "one mixkv_compress_layers call per step (all layers in one set of kernels)",
             "parallelism": "replicas only" if world > 1 else "single GPU"}),
+        "timing": {"blocks": len(blocks), "steps_per_block": args.steps,
+                   "ms_per_step_median_block": ms_per_step, "ms_per_step_best_block": min(blocks),
+                   "ms_per_step_first_block": blocks[0],
+                   "regime": ("sustained: sw_power_cap seen during the timed blocks"
+                              if clocks and "sw_power_cap" in clocks.get("reasons", [])
+                              else "no throttle reason seen during the timed blocks")},
         "per_layer_latency_us": layer_ms * 1e3,
         "token_layers_per_s": world * wl.total_tokens * NL / (ms_per_step * 1e-3),
         "stage_ms": stage_ms,
@@ -426,11 +448,16 @@ def run_mixkv(args):
                      "algorithmic_bytes_per_launch": NL * ab[dom],
                      "kernel_ms": dom_ms},
         "clocks": clocks,
-        "gpu_launches": n_stage * args.steps,
+        "gpu_launches": n_stage * args.steps * len(blocks),
     }
     if per_layer_ms is not None:
+        one_us = per_layer_ms / NL * 1e3
         line["one_layer_per_call"] = {
-            "ms_per_step": per_layer_ms, "per_layer_latency_us": per_layer_ms / NL * 1e3,
+            "ms_per_step": per_layer_ms, "per_layer_latency_us": one_us,
+            "roofline": {"bound": "hbm", "achieved": ab["layer"] / (one_us * 1e-6) / 1e9,
+                         "peak": peak, "unit": "GB/s",
+                         "frac": ab["layer"] / (one_us * 1e-6) / 1e9 / peak,
+                         "frac_of_8TBs_nominal": ab["layer"] / (one_us * 1e-6) / 8e12},
             "note": "same step as one mixkv_compress_layer call per layer, issued from Python"}
     if e2e is not None:
         line["e2e"] = e2e

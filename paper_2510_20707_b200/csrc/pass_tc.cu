@@ -42,7 +42,6 @@ constexpr int kEpiWarp0 = 4;
 constexpr int kEpiWarps = 16;                    // warps 4..19
 constexpr int kEpiThreads = kEpiWarps * 32;
 constexpr int kAuxWarp0 = kEpiWarp0 + kEpiWarps; // warps 20..: key statistics / value norms
-constexpr int kThreads2 = (kAuxWarp0 + 4) * 32;  // pass 2: 24 warps
 
 // Registers per thread of the calling warpgroup from here on: N, where the kernel was launched
 // with BASE (every warp of the warpgroup executes this).
@@ -113,6 +112,42 @@ __device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
   f32x2 d;
   asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
   return d;
+}
+
+// exp2 of both halves of t on the FMA pipe, for the share of the exponentials that the
+// special-function unit (16 results per clock and SM, the bound of both passes) cannot take:
+// t = j + f with j the nearest integer (the magic-number add leaves j in the low mantissa bits),
+// 2^f by a cubic (relative error below 7.5e-5 on [-0.5, 0.5]), j added to the exponent field.
+// t is clamped at -125 (a masked logit, -inf, gives 2^-125 instead of 0).
+__device__ __forceinline__ f32x2 ex2_poly2(f32x2 t2) {
+  float t0, t1;
+  unpack2(t2, t0, t1);
+  t2 = pack2(fmaxf(t0, -125.f), fmaxf(t1, -125.f));
+  const f32x2 y = add2(t2, pack2(12582912.f, 12582912.f));             // 1.5 * 2^23 + j
+  const f32x2 jf = add2(y, pack2(-12582912.f, -12582912.f));
+  const f32x2 f = fma2(jf, pack2(-1.f, -1.f), t2);
+  f32x2 p = fma2(pack2(0.0551716536f, 0.0551716536f), f, pack2(0.242611125f, 0.242611125f));
+  p = fma2(p, f, pack2(0.693260968f, 0.693260968f));
+  p = fma2(p, f, pack2(0.999928057f, 0.999928057f));
+  float p0, p1, y0, y1;
+  unpack2(p, p0, p1);
+  unpack2(y, y0, y1);
+  return pack2(__uint_as_float(__float_as_uint(p0) + (__float_as_uint(y0) << 23)),
+               __uint_as_float(__float_as_uint(p1) + (__float_as_uint(y1) << 23)));
+}
+// Of every 16 pairs of exponentials, kPolyPairs go through ex2_poly2, spread evenly.
+#ifndef MIXKV_POLY_PAIRS
+#define MIXKV_POLY_PAIRS 0
+#endif
+constexpr int kPolyPairs = MIXKV_POLY_PAIRS;
+__host__ __device__ constexpr bool poly_pair(int k) {
+  return ((k % 16) * kPolyPairs) % 16 < kPolyPairs && kPolyPairs > 0;
+}
+__device__ __forceinline__ f32x2 ex2_pair(f32x2 t2, const bool poly) {
+  if (poly) return ex2_poly2(t2);
+  float a0, a1;
+  unpack2(t2, a0, a1);
+  return pack2(ex2(a0), ex2(a1));
 }
 
 constexpr size_t kSmemLimit = 227 * 1024;   // dynamic shared memory a CTA may ask for
@@ -241,11 +276,46 @@ __device__ __forceinline__ void finish_heads(const SeqTable& st, const Workspace
   }
 }
 
-// One 32-column chunk of a logit row: running (max, sum) of the softmax in log2 units.
-__device__ __forceinline__ void softmax_chunk(uint32_t (&r)[32], const bool need_mask,
-                                              const int kbase, const int lim,
-                                              const float scale_log2e, float& m_run,
-                                              float& z_run) {
+// The running softmax statistics of a query row are a pair (m, z): z = sum over the keys seen
+// so far of exp2(logit * c - m), where m is a REFERENCE in log2 units, a logit of the row seen
+// earlier, not necessarily the largest one: z * 2^m is the same number whatever m is, fp32
+// carries 2^±126 around it, and searching the maximum of every chunk costs a quarter of the
+// epilogue's instructions on its critical path.
+//
+// Fast path, one 32-column chunk: the sum of exp2(logit * c - m) with the standing reference.
+__device__ __forceinline__ float chunk_expsum(const uint32_t (&r)[32], const float scale_log2e,
+                                              const float m_run) {
+  const f32x2 sc2 = pack2(scale_log2e, scale_log2e), nm2 = pack2(-m_run, -m_run);
+  f32x2 za = pack2(0.f, 0.f), zb = za;
+#pragma unroll
+  for (int j = 0; j < 32; j += 4) {
+    const f32x2 ta = fma2(pack2(__uint_as_float(r[j]), __uint_as_float(r[j + 1])), sc2, nm2);
+    const f32x2 tb = fma2(pack2(__uint_as_float(r[j + 2]), __uint_as_float(r[j + 3])), sc2, nm2);
+    za = add2(za, ex2_pair(ta, poly_pair(j / 2)));
+    zb = add2(zb, ex2_pair(tb, poly_pair(j / 2 + 1)));
+  }
+  float z0, z1;
+  unpack2(add2(za, zb), z0, z1);
+  return z0 + z1;
+}
+// A chunk sum at or above this means a logit about 2^99 above the reference (or no reference
+// yet): the chunk is redone on the slow path.  Below it nothing can overflow: 1024 chunks of a
+// head add up to less than 2^110.
+constexpr float kChunkSumLimit = 1e30f;
+
+// Slow path: the chunk again from tensor memory with the causal mask and a maximum search; the
+// reference moves up to the chunk's maximum if that is larger.  Taken for the first chunk of
+// a segment, for the tiles that need the mask, and when the fast path's sum says that the
+// reference is too low.  Every lane of the warp takes part (the load is warp-wide).  Returns
+// the new (m, z).
+__device__ __noinline__ float2 softmax_chunk_ref(const uint32_t taddr, const bool need_mask,
+                                                 const int kbase, const int lim,
+                                                 const float scale_log2e, float m_run,
+                                                 float z_run) {
+  uint32_t r[32];
+  tmem_ld32(taddr, r);
+  tmem_ld_wait();
+  tmem_ld_fence(r);
   if (need_mask) {
 #pragma unroll
     for (int j = 0; j < 32; ++j)
@@ -261,19 +331,8 @@ __device__ __forceinline__ void softmax_chunk(uint32_t (&r)[32], const bool need
     z_run *= ex2(m_run - mn);
     m_run = mn;
   }
-  const f32x2 sc2 = pack2(scale_log2e, scale_log2e), nm2 = pack2(-m_run, -m_run);
-  f32x2 za = pack2(0.f, 0.f), zb = za;
-#pragma unroll
-  for (int j = 0; j < 32; j += 4) {
-    float a0, a1, b0, b1;
-    unpack2(fma2(pack2(__uint_as_float(r[j]), __uint_as_float(r[j + 1])), sc2, nm2), a0, a1);
-    unpack2(fma2(pack2(__uint_as_float(r[j + 2]), __uint_as_float(r[j + 3])), sc2, nm2), b0, b1);
-    za = add2(za, pack2(ex2(a0), ex2(a1)));
-    zb = add2(zb, pack2(ex2(b0), ex2(b1)));
-  }
-  float z0, z1;
-  unpack2(add2(za, zb), z0, z1);
-  z_run += z0 + z1;
+  z_run += chunk_expsum(r, scale_log2e, m_run);
+  return make_float2(m_run, z_run);
 }
 
 // grid = g1 persistent CTAs of 28 warps: TMA, 2 idle, MMA, 16 epilogue, 8 key-statistics.  The
@@ -323,7 +382,7 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(&bars->tfull[s], 1);
-      mbar_init(&bars->tempty[s], kEpiThreads);      // every epilogue thread reads every tile
+      mbar_init(&bars->tempty[s], kEpiWarps);        // every epilogue warp reads every tile
     }
     mbar_init(&bars->qfull, 1);
     mbar_init(&bars->qfree, 1);
@@ -429,11 +488,12 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
     const int jrow = row % W;
     float m_run = -1e30f, z_run = 0.f;
     int it = 0, seg_first = lo;
-    bool seg_start = true;
+    bool seg_start = true, no_ref = true;
     for (TileIter ti(st.tile1_start, st.batch, H, st.nt1, lo, hi); ti.valid(); ti.next()) {
       if (seg_start) {
         m_run = -1e30f;
         z_run = 0.f;
+        no_ref = true;   // the segment's first chunk sets the reference
         seg_first = ti.id;
       }
       seg_start = ti.seg_last();
@@ -448,15 +508,30 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
         const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + ts * (MB * 128) + col0;
 #pragma unroll 1
         for (int c0 = 0; c0 < NC; c0 += 32) {   // kept rolled: the body must stay in the i-cache
-          uint32_t ra[32];
-          tmem_ld32(taddr + c0, ra);
-          tmem_ld_wait();
-          tmem_ld_fence(ra);
-          softmax_chunk(ra, need_mask, k0 + c0, lim, scale_log2e, m_run, z_run);
+          bool slow = no_ref || need_mask;      // the same in every lane
+          float zc = 0.f;
+          if (!slow) {
+            uint32_t ra[32];
+            tmem_ld32(taddr + c0, ra);
+            tmem_ld_wait();
+            tmem_ld_fence(ra);
+            zc = chunk_expsum(ra, scale_log2e, m_run);
+            slow = __any_sync(0xffffffffu, !(zc < kChunkSumLimit));
+          }
+          if (slow) {
+            const float2 mz =
+                softmax_chunk_ref(taddr + c0, need_mask, k0 + c0, lim, scale_log2e, m_run, z_run);
+            m_run = mz.x;
+            z_run = mz.y;
+            no_ref = false;
+          } else {
+            z_run += zc;
+          }
         }
       }
       tc_fence_before();
-      mbar_arrive(&bars->tempty[ts]);
+      __syncwarp();   // one arrival per warp: 512 single arrivals on one word cost more than a chunk
+      if (lane == 0) mbar_arrive(&bars->tempty[ts]);
       if (seg_start && row < NQ)
         ws.rowstat[((size_t)seg_first * NU + unit) * NQ + row] = make_float2(m_run, z_run);
       ++it;
@@ -581,6 +656,24 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
 }
 
 // ======================================================================== pass 2
+// Pass 2 streams K and V and sits at the HBM bound with sixteen warps: K/Q producer, MMA, V
+// producer, 1 idle, two epilogue warpgroups that own alternate tiles (every thread one key and all
+// of its G*W logit columns, so nothing is exchanged between warps), 4 value-norm warps.  More
+// epilogue warps splitting the columns of a tile were measured slower (C3: 13.4 against 11.7 us per
+// layer): the exchange of partial sums and the extra warps cost more than they hide.
+constexpr int kP2Threads = 16 * 32;
+constexpr int kP2EpiWarps = 8;                   // warps 4..11
+constexpr int kP2AuxWarp0 = 12;                  // warps 12..15: value norms
+
+// Named barrier among n threads that also agrees on whether to stop: the leader samples the
+// CTA abort flag before the barrier and everybody reads that sample after it, so a group
+// never splits around a later barrier.
+__device__ __forceinline__ bool group_sync_stop(int id, int n, bool leader, volatile int* abort,
+                                                volatile int* slots, int it) {
+  if (leader) slots[it & 1] = *abort;
+  named_bar_sync(id, n);
+  return slots[it & 1] != 0;
+}
 constexpr int kP2KStages = 3;              // K tiles (32 KB each)
 constexpr int kP2VStagesMax = 4;           // V half tiles: 64 rows, 16 KB each
 constexpr int kVSubBytes = 64 * 256;
@@ -591,13 +684,12 @@ struct P2Bars {
   uint64_t vempty[kP2VStagesMax];
   uint64_t tfull[2];
   uint64_t tempty[2];
-  uint64_t xfull[2];    // the sixteen epilogue warps have left their partial sums of a tile
-  uint64_t xempty[2];   // the four value-norm warps have added them up
   uint64_t qfull;
   uint64_t qfree;
   uint64_t kbready;
   uint32_t tmem_base;
   int abort;
+  int vote[3][2];
 };
 
 // N logit columns of one key (registers r[0..N)): adds exp2(logit * scale - normaliser of the
@@ -619,18 +711,8 @@ __device__ __forceinline__ void colsum_chunk(const uint32_t (&r)[N], const float
   }
 }
 
-// registers per thread: at launch, then per role (6 warpgroups: 40 + 4 * 88 + 88 = 6 * 80; a
-// value-norm thread keeps the sixteen 16-byte loads of its row in flight)
-#ifndef P2_LEAD
-#define P2_LEAD 40
-#define P2_EPI 88
-#define P2_AUX 88
-#endif
-constexpr int kP2RegsLaunch = 80, kP2RegsLead = P2_LEAD, kP2RegsEpi = P2_EPI, kP2RegsAux = P2_AUX;
-
-// grid = g2 persistent CTAs of 24 warps: K producer, V producer, 1 idle, MMA, 16 epilogue,
-// 4 value-norm warps.
-__global__ void __launch_bounds__(kThreads2, 1)
+// grid = g2 persistent CTAs: K producer, MMA, V producer, 1 idle, 8 epilogue, 4 value-norm warps.
+__global__ void __launch_bounds__(kP2Threads, 1)
 k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
         const __grid_constant__ CUtensorMap tmQ, const SeqTable st, const Workspace ws,
         float* __restrict__ s_div_out, const float scale_log2e,
@@ -644,15 +726,14 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
   unsigned char* sK = sQ + 2 * NB * 128;      // kP2KStages x 32 KB
   unsigned char* sV = sK + kP2KStages * kTileBytes;   // vstages x 16 KB
   float* sbq = reinterpret_cast<float*>(sV + vstages * kVSubBytes);  // [2][256] negated normalisers
-  float* sx = sbq + 512;                      // [2 stages][4 warpgroups][128] partial column sums
-  float* sred = sx + 1024;                    // [64]: 16 diversity, 16 value norms / attention
+  float* sred = sbq + 512;                    // [64]: 2 x 16 epilogue, 16 value norms + 4 mean key
   P2Bars* bars = reinterpret_cast<P2Bars*>(sred + 64);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int lo = cta_first_tile(blockIdx.x, split2(st));
   const int hi = cta_first_tile(blockIdx.x + 1, split2(st));
   volatile int* abort = &bars->abort;
-  constexpr int kWarpTmaV = 1, kP2WarpMma = 3;
+  constexpr int kWarpTmaV = 2;
 
   pdl_launch_dependents();
   if (tid == 0) {
@@ -666,9 +747,7 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(&bars->tfull[s], 1);
-      mbar_init(&bars->tempty[s], kEpiThreads);   // every epilogue thread reads every tile
-      mbar_init(&bars->xfull[s], kEpiWarps);
-      mbar_init(&bars->xempty[s], 4);
+      mbar_init(&bars->tempty[s], 128);    // the warpgroup that owns the accumulator stage
     }
     mbar_init(&bars->qfull, 1);
     mbar_init(&bars->qfree, 1);
@@ -676,7 +755,7 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
     bars->abort = 0;
     mbar_init_fence();
   }
-  if (warp == kP2WarpMma) tmem_alloc(&bars->tmem_base, 512);
+  if (warp == kWarpMma) tmem_alloc(&bars->tmem_base, 512);
   if (warp == kWarpTma && lane == 0) {
     tma_prefetch_desc(&tmK);
     tma_prefetch_desc(&tmQ);
@@ -688,217 +767,204 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
   const uint32_t tmem = bars->tmem_base;
   pdl_wait();
 
-  if (warp < kEpiWarp0) {
-    set_regs<kP2RegsLead, kP2RegsLaunch>();
-    if (warp == kWarpTma) {
-      // ---------------------------------------------------------------- K / Q producer
-      if (lane == 0) {
-        int it = 0, segn = 0;
-        bool seg_start = true;
-        for (TileIter ti(st.tile2_start, st.batch, H, st.nt2, lo, hi); ti.valid(); ti.next()) {
-          if (seg_start) {
-            if (segn > 0 && !mbar_wait(&bars->qfree, (segn - 1) & 1, abort)) break;
-            mbar_expect_tx(&bars->qfull, NQ * 256);
-            tma_load_3d(sQ, &tmQ, 0, ti.bh() * NQ, ti.layer, &bars->qfull);
-            tma_load_3d(sQ + NB * 128, &tmQ, 64, ti.bh() * NQ, ti.layer, &bars->qfull);
-            ++segn;
-          }
-          seg_start = ti.seg_last();
-          const int s = it % kP2KStages, ph = (it / kP2KStages) & 1;
-          if (!mbar_wait(&bars->kempty[s], ph ^ 1, abort)) break;
-          mbar_expect_tx(&bars->kfull[s], kTileBytes);
-          const int y = st.cu[ti.b] + ti.t * kTile;
-          tma_load_4d(sK + s * kTileBytes, &tmK, 0, y, ti.h, ti.layer, &bars->kfull[s]);
-          tma_load_4d(sK + s * kTileBytes + kHalfBytes, &tmK, 64, y, ti.h, ti.layer, &bars->kfull[s]);
-          ++it;
+  if (warp == kWarpTma) {
+    // ------------------------------------------------------------------ K / Q producer
+    if (lane == 0) {
+      int it = 0, segn = 0;
+      bool seg_start = true;
+      for (TileIter ti(st.tile2_start, st.batch, H, st.nt2, lo, hi); ti.valid(); ti.next()) {
+        if (seg_start) {
+          if (segn > 0 && !mbar_wait(&bars->qfree, (segn - 1) & 1, abort)) break;
+          mbar_expect_tx(&bars->qfull, NQ * 256);
+          tma_load_3d(sQ, &tmQ, 0, ti.bh() * NQ, ti.layer, &bars->qfull);
+          tma_load_3d(sQ + NB * 128, &tmQ, 64, ti.bh() * NQ, ti.layer, &bars->qfull);
+          ++segn;
         }
-        if (*abort) {
-          raise(status, abort);
-          drain_ring(bars->kfull, kP2KStages, it);
-        }
+        seg_start = ti.seg_last();
+        const int s = it % kP2KStages, ph = (it / kP2KStages) & 1;
+        if (!mbar_wait(&bars->kempty[s], ph ^ 1, abort)) break;
+        mbar_expect_tx(&bars->kfull[s], kTileBytes);
+        const int y = st.cu[ti.b] + ti.t * kTile;
+        tma_load_4d(sK + s * kTileBytes, &tmK, 0, y, ti.h, ti.layer, &bars->kfull[s]);
+        tma_load_4d(sK + s * kTileBytes + kHalfBytes, &tmK, 64, y, ti.h, ti.layer, &bars->kfull[s]);
+        ++it;
       }
-    } else if (warp == kWarpTmaV) {
-      // ---------------------------------------------------------------- V producer
-      if (lane == 0 && use_vnorm == MIXKV_INTRINSIC_VNORM) {
-        int vit = 0;
-        bool ok = true;
-        for (TileIter ti(st.tile2_start, st.batch, H, st.nt2, lo, hi); ti.valid() && ok; ti.next()) {
-          const int y = st.cu[ti.b] + ti.t * kTile;
-          for (int sub = 0; sub < 2; ++sub) {
-            const int vs = vit % vstages, vph = (vit / vstages) & 1;
-            if (!mbar_wait(&bars->vempty[vs], vph ^ 1, abort)) {
-              ok = false;
-              break;
-            }
-            mbar_expect_tx(&bars->vfull[vs], kVSubBytes);
-            unsigned char* dst = sV + vs * kVSubBytes;
-            tma_load_4d(dst, &tmV, 0, y + sub * 64, ti.h, ti.layer, &bars->vfull[vs]);
-            tma_load_4d(dst + kVSubBytes / 2, &tmV, 64, y + sub * 64, ti.h, ti.layer, &bars->vfull[vs]);
-            ++vit;
-          }
-        }
-        if (*abort) {
-          raise(status, abort);
-          drain_ring(bars->vfull, vstages, vit);
-        }
-      }
-    } else if (warp == kP2WarpMma) {
-      // ---------------------------------------------------------------- MMA issuer
-      if (lane == 0) {
-        const uint32_t idesc = umma_idesc_bf16(128, NB);
-        const uint32_t q_lo = umma_desc_lo(smem_u32(sQ));
-        const uint32_t k_lo = umma_desc_lo(smem_u32(sK));
-        const uint32_t q_half = (uint32_t)(NB * 128) >> 4;   // second 64-column half of the B rows
-        int it = 0, segn = 0;
-        bool seg_start = true;
-        for (TileIter ti(st.tile2_start, st.batch, H, st.nt2, lo, hi); ti.valid(); ti.next()) {
-          if (seg_start) {
-            if (!mbar_wait(&bars->qfull, segn & 1, abort)) break;
-            if (!mbar_wait(&bars->kbready, segn & 1, abort)) break;
-            ++segn;
-          }
-          seg_start = ti.seg_last();
-          const int s = it % kP2KStages, ph = (it / kP2KStages) & 1, ts = it & 1, tph = (it >> 1) & 1;
-          if (!mbar_wait(&bars->kfull[s], ph, abort)) break;
-          if (!mbar_wait(&bars->tempty[ts], tph ^ 1, abort)) break;
-          tc_fence_after();
-          const uint32_t kb_lo = k_lo + (uint32_t)s * (kTileBytes >> 4);
-#pragma unroll
-          for (int ks = 0; ks < 8; ++ks) {
-            const uint32_t a_lo = kb_lo + (uint32_t)((ks >> 2) * (kHalfBytes >> 4) + (ks & 3) * 2);
-            const uint32_t b_lo = q_lo + (ks >> 2) * q_half + (uint32_t)((ks & 3) * 2);
-            if (ks == 0)
-              umma_bf16_lo<0>(tmem + ts * 256, a_lo, b_lo, idesc);
-            else
-              umma_bf16_lo<1>(tmem + ts * 256, a_lo, b_lo, idesc);
-          }
-          umma_commit(&bars->kempty[s]);
-          umma_commit(&bars->tfull[ts]);
-          if (seg_start) umma_commit(&bars->qfree);
-          ++it;
-        }
-        if (*abort) raise(status, abort);
+      if (*abort) {
+        raise(status, abort);
+        drain_ring(bars->kfull, kP2KStages, it);
       }
     }
-  } else if (warp < kAuxWarp0) {
+  } else if (warp == kWarpTmaV) {
+    // ------------------------------------------------------------------ V producer
+    if (lane == 0 && use_vnorm == MIXKV_INTRINSIC_VNORM) {
+      int vit = 0;
+      bool ok = true;
+      for (TileIter ti(st.tile2_start, st.batch, H, st.nt2, lo, hi); ti.valid() && ok; ti.next()) {
+        const int y = st.cu[ti.b] + ti.t * kTile;
+        for (int sub = 0; sub < 2; ++sub) {
+          const int vs = vit % vstages, vph = (vit / vstages) & 1;
+          if (!mbar_wait(&bars->vempty[vs], vph ^ 1, abort)) {
+            ok = false;
+            break;
+          }
+          mbar_expect_tx(&bars->vfull[vs], kVSubBytes);
+          unsigned char* dst = sV + vs * kVSubBytes;
+          tma_load_4d(dst, &tmV, 0, y + sub * 64, ti.h, ti.layer, &bars->vfull[vs]);
+          tma_load_4d(dst + kVSubBytes / 2, &tmV, 64, y + sub * 64, ti.h, ti.layer, &bars->vfull[vs]);
+          ++vit;
+        }
+      }
+      if (*abort) {
+        raise(status, abort);
+        drain_ring(bars->vfull, vstages, vit);
+      }
+    }
+  } else if (warp == kWarpMma) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc = umma_idesc_bf16(128, NB);
+      int it = 0, segn = 0;
+      bool seg_start = true;
+      for (TileIter ti(st.tile2_start, st.batch, H, st.nt2, lo, hi); ti.valid(); ti.next()) {
+        if (seg_start) {
+          if (!mbar_wait(&bars->qfull, segn & 1, abort)) break;
+          if (!mbar_wait(&bars->kbready, segn & 1, abort)) break;
+          ++segn;
+        }
+        seg_start = ti.seg_last();
+        const int s = it % kP2KStages, ph = (it / kP2KStages) & 1, ts = it & 1, tph = (it >> 1) & 1;
+        if (!mbar_wait(&bars->kfull[s], ph, abort)) break;
+        if (!mbar_wait(&bars->tempty[ts], tph ^ 1, abort)) break;
+        tc_fence_after();
+        const uint32_t kaddr = smem_u32(sK + s * kTileBytes);
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+          const uint64_t da = umma_desc_sw128(kaddr + (ks >> 2) * kHalfBytes + (ks & 3) * 32);
+          const uint64_t db = umma_desc_sw128(smem_u32(sQ) + (ks >> 2) * NB * 128 + (ks & 3) * 32);
+          umma_bf16(tmem + ts * 256, da, db, idesc, ks > 0);
+        }
+        umma_commit(&bars->kempty[s]);
+        umma_commit(&bars->tfull[ts]);
+        if (seg_start) umma_commit(&bars->qfree);
+        ++it;
+      }
+      if (*abort) raise(status, abort);
+    }
+  } else if (warp >= kEpiWarp0 && warp < kEpiWarp0 + kP2EpiWarps) {
     // ------------------------------------------------------------------ epilogue
-    // All sixteen warps read every tile (two accumulator stages: the MMA of the next tile fills
-    // the other stage meanwhile); a thread is one key.  The four warpgroups split the G*W logit
-    // columns of the key: each leaves its partial sum in shared memory, where the value-norm
-    // warps add the four up.  Warpgroup 0 also takes the three mean-key columns and owns the
-    // diversity score.  After an abort the waits fail at once and every warp still walks the
-    // same tiles, so the per-segment barriers stay matched.
-    set_regs<kP2RegsEpi, kP2RegsLaunch>();
-    const int wg = (warp - kEpiWarp0) >> 2, quarter = warp & 3;
-    const int et = tid - kEpiWarp0 * 32;           // 0..511
+    // The two warpgroups take alternate tiles (warpgroup g owns accumulator stage g), one key
+    // per thread and all G*W columns of it, so a tile needs no exchange between warpgroups and
+    // the groups never wait for each other: each keeps its own copy of the normaliser table
+    // and leaves its own partial score statistics.
+    const int quarter = warp & 3, wg = (warp - kEpiWarp0) >> 2;
+    const int gt = (tid - kEpiWarp0 * 32) & 127;   // thread inside the warpgroup
+    const int gw = gt >> 5;                        // warp inside the warpgroup
     const int key = quarter * 32 + lane;
-    const int nch = NQ / 16;                       // 16-column chunks of a key's logits
-    const int ch0 = (nch * wg) >> 2, ch1 = (nch * (wg + 1)) >> 2;   // this warpgroup's chunks
-    const int n32 = (ch1 - ch0) >> 1;
-    const bool rest16 = ((ch1 - ch0) & 1) != 0;
+    const int nch = NQ / 16;
+    float* mybq = sbq + wg * 256;
+    const int barid = 1 + wg;                      // named barriers 1, 2: one per warpgroup
     const f32x2 sc2 = pack2(scale_log2e, scale_log2e);
-    float dmin = INFINITY, dmax = -INFINITY, dsum = 0.f;
-    int it = 0, segn = 0, seg_first = lo;
+    float dmin = INFINITY, dmax = -INFINITY, dsum = 0.f, exw = 0.f;
+    int it = 0, seg_first = lo;
     bool seg_start = true;
-    const float* mybq = sbq;
     for (TileIter ti(st.tile2_start, st.batch, H, st.nt2, lo, hi); ti.valid(); ti.next()) {
       const int L = st.cu[ti.b + 1] - st.cu[ti.b], P = L - W;
       if (seg_start) {
-        // pass 1 left one negated log2 normaliser per window row of this (layer, b, h); the
-        // table alternates between two buffers, so the previous segment's readers are never
-        // overtaken
-        float* tb = sbq + (segn & 1) * 256;
-        if (et < NQ) tb[et] = ws.bq[(size_t)ti.unit() * NQ + et];
-        mybq = tb;
-        ++segn;
-        dmin = INFINITY, dmax = -INFINITY, dsum = 0.f;
+        // pass 1 left one negated log2 normaliser per window row of this (layer, b, h)
+        named_bar_sync(barid, 128);   // the previous segment's readers of mybq are done
+        for (int q = gt; q < NQ; q += 128) mybq[q] = ws.bq[(size_t)ti.unit() * NQ + q];
+        dmin = INFINITY, dmax = -INFINITY, dsum = 0.f, exw = 0.f;
         seg_first = ti.id;
-        named_bar_sync(2, kEpiThreads);
+        named_bar_sync(barid, 128);
       }
       seg_start = ti.seg_last();
-      const int ts = it & 1, use = it >> 1;
-      const int ikey = ti.t * kTile + key;
-      float kinv_i = 0.f;
-      if (wg == 0 && ikey < P) kinv_i = ws.kinv[kpos(st, ti.layer, ti.h, ti.b, ikey)];
-      const bool ok = mbar_wait(&bars->tfull[ts], use & 1, abort);
-      tc_fence_after();
-      const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + ts * 256;
-      f32x2 acc = pack2(0.f, 0.f);
-      float dot = 0.f;
-      if (ok) {
-        uint32_t rd[4];
-        if (wg == 0) tmem_ld4(taddr + NQ, rd);
-        // 32-column chunks, then a 16-column rest; kept rolled: the body must stay in the i-cache
+      const int ts = it & 1;
+      if (ts == wg) {   // this warpgroup's tile
+        const int tph = (it >> 1) & 1;
+        const int ikey = ti.t * kTile + key;
+        float kinv_i = 0.f;
+        if (ikey < P) kinv_i = ws.kinv[kpos(st, ti.layer, ti.h, ti.b, ikey)];
+        const bool ok = mbar_wait(&bars->tfull[ts], tph, abort);
+        tc_fence_after();
+        const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + ts * 256;
+        f32x2 acc = pack2(0.f, 0.f);
+        float dot = 0.f;
+        if (ok) {
+          uint32_t rd[4];
+          tmem_ld4(taddr + NQ, rd);
+          // 32-column chunks (the other warpgroup's tile keeps the SM busy while this load is
+          // in flight), then a 16-column rest; kept rolled: the body must stay in the i-cache
+          const int n32 = nch >> 1;
 #pragma unroll 1
-        for (int ci = 0; ci < n32; ++ci) {
-          uint32_t ra[32];
-          tmem_ld32(taddr + ch0 * 16 + ci * 32, ra);
-          tmem_ld_wait();
-          tmem_ld_fence(ra);
-          colsum_chunk<32>(ra, mybq + ch0 * 16 + ci * 32, sc2, acc);
-        }
-        if (rest16) {
-          uint32_t rb[16];
-          tmem_ld16(taddr + ch0 * 16 + n32 * 32, rb);
-          tmem_ld_wait();
-          tmem_ld_fence(rb);
-          colsum_chunk<16>(rb, mybq + ch0 * 16 + n32 * 32, sc2, acc);
-        }
-        if (wg == 0) {
+          for (int ci = 0; ci < n32; ++ci) {
+            uint32_t ra[32];
+            tmem_ld32(taddr + ci * 32, ra);
+            tmem_ld_wait();
+            tmem_ld_fence(ra);
+            colsum_chunk<32>(ra, mybq + ci * 32, sc2, acc);
+          }
+          if (nch & 1) {
+            uint32_t rb[16];
+            tmem_ld16(taddr + n32 * 32, rb);
+            tmem_ld_wait();
+            tmem_ld_fence(rb);
+            colsum_chunk<16>(rb, mybq + n32 * 32, sc2, acc);
+          }
           tmem_ld_wait();
           tmem_ld_fence(rd);
           dot = (__uint_as_float(rd[0]) + __uint_as_float(rd[1])) + __uint_as_float(rd[2]);
         }
+        tc_fence_before();
+        mbar_arrive(&bars->tempty[ts]);
+        if (ok && ikey < P) {
+          float acc0, acc1;
+          unpack2(acc, acc0, acc1);
+          const size_t poff = ppos(st, ti.layer, ti.h, ti.b, 0);
+          const float ex = acc0 + acc1;
+          ws.s_ex_raw[poff + ikey] = ex;
+          const float sd = -dot * kinv_i;
+          s_div_out[poff + ikey] = sd;
+          dmin = fminf(dmin, sd);
+          dmax = fmaxf(dmax, sd);
+          dsum += sd;
+          // number of pooling windows (centres in [0, P)) that cover this position
+          const int cover = min(ikey, pool_half) + min(P - 1 - ikey, pool_half) + 1;
+          exw = fmaf(ex, (float)cover, exw);
+        }
       }
-      tc_fence_before();
-      mbar_arrive(&bars->tempty[ts]);
-      // hand the partial sum to the value-norm warps (the slot was read two tiles ago)
-      if (use > 0) mbar_wait(&bars->xempty[ts], (use - 1) & 1, abort);
-      float acc0, acc1;
-      unpack2(acc, acc0, acc1);
-      sx[(ts * 4 + wg) * 128 + key] = acc0 + acc1;
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&bars->xfull[ts]);
-      if (wg == 0 && ok && ikey < P) {
-        const float sd = -dot * kinv_i;
-        s_div_out[ppos(st, ti.layer, ti.h, ti.b, 0) + ikey] = sd;
-        dmin = fminf(dmin, sd);
-        dmax = fmaxf(dmax, sd);
-        dsum += sd;
-      }
-      if (seg_start && wg == 0) {
-        // the segment's diversity statistics (the attention-score sum comes from the value-norm warps)
-        const float a = warp_min(dmin), b2 = warp_max(dmax), c2 = warp_sum(dsum);
+      if (group_sync_stop(barid, 128, gt == 0, abort, bars->vote[wg], it)) break;
+      if (seg_start) {
+        // this warpgroup's share of the segment's score statistics (neutral if it had no tile)
+        const float a = warp_min(dmin), b2 = warp_max(dmax), c2 = warp_sum(dsum),
+                    d2 = warp_sum(exw);
+        float* sr = sred + wg * 16;
         if (lane == 0) {
-          sred[quarter] = a;
-          sred[4 + quarter] = b2;
-          sred[8 + quarter] = c2;
+          sr[gw] = a;
+          sr[4 + gw] = b2;
+          sr[8 + gw] = c2;
+          sr[12 + gw] = d2;
         }
-        named_bar_sync(1, 128);
-        if (et == 0) {
-          ws.dstat[(size_t)seg_first * 2] = make_float4(
-              fminf(fminf(sred[0], sred[1]), fminf(sred[2], sred[3])),
-              fmaxf(fmaxf(sred[4], sred[5]), fmaxf(sred[6], sred[7])),
-              (sred[8] + sred[9]) + (sred[10] + sred[11]), 0.f);
+        named_bar_sync(barid, 128);
+        if (gt == 0) {
+          ws.dstat[(size_t)seg_first * 2 + wg] = make_float4(
+              fminf(fminf(sr[0], sr[1]), fminf(sr[2], sr[3])),
+              fmaxf(fmaxf(sr[4], sr[5]), fmaxf(sr[6], sr[7])),
+              (sr[8] + sr[9]) + (sr[10] + sr[11]), (sr[12] + sr[13]) + (sr[14] + sr[15]));
         }
-        named_bar_sync(1, 128);
       }
       ++it;
     }
-  } else {
+  } else if (warp >= kP2AuxWarp0) {
     // ------------------------------------------------------------------ mean key, value norms
     // At the start of a segment: write the bf16 hi / lo / lo2 split of the head's mean unit key
-    // (pass 1) into the three extra B rows.  Per tile: warps 0, 1 of the four read the first 64
-    // rows of the V tile, warps 2, 3 the last 64; one row per thread from the swizzled half tile;
-    // then thread vt adds the four partial attention sums of key vt.
-    set_regs<kP2RegsAux, kP2RegsLaunch>();
-    const int vt = tid - kAuxWarp0 * 32;         // 0..127
+    // (pass 1) into the three extra B rows.  Per tile: warps 12, 13 read the first 64 rows of the V
+    // tile, warps 14, 15 the last 64; one row per thread from the swizzled half tile.
+    const int vt = tid - kP2AuxWarp0 * 32;         // 0..127
     const int sub = vt >> 6, vr = vt & 63;
-    float vmin = INFINITY, vmax = -INFINITY, vsum = 0.f, exw = 0.f;
+    float vmin = INFINITY, vmax = -INFINITY, vsum = 0.f;
     int it = 0, segn = 0, seg_first = lo;
     bool seg_start = true;
     for (TileIter ti(st.tile2_start, st.batch, H, st.nt2, lo, hi); ti.valid(); ti.next()) {
-      const int P = st.cu[ti.b + 1] - st.cu[ti.b] - W;
       if (seg_start) {
         const float kb = ws.kbar[(size_t)ti.unit() * kHeadDim + vt];   // mean unit key (pass 1)
         __nv_bfloat16 parts[3];
@@ -924,13 +990,14 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
         __syncwarp();
         if (lane == 0) mbar_arrive(&bars->kbready);
         ++segn;
-        vmin = INFINITY, vmax = -INFINITY, vsum = 0.f, exw = 0.f;
+        vmin = INFINITY, vmax = -INFINITY, vsum = 0.f;
         seg_first = ti.id;
       }
       seg_start = ti.seg_last();
       if (use_vnorm == MIXKV_INTRINSIC_KNORM) {
         // key-norm ablation: the intrinsic term is minus the key norm, which pass 1 left as its
         // reciprocal; no V tile is loaded
+        const int P = st.cu[ti.b + 1] - st.cu[ti.b] - W;
         const int i = ti.t * kTile + vt;
         if (i < P) {
           const float ki = ws.kinv[kpos(st, ti.layer, ti.h, ti.b, i)];
@@ -941,6 +1008,7 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
           vsum += n;
         }
       } else if (use_vnorm) {
+        const int P = st.cu[ti.b + 1] - st.cu[ti.b] - W;
         const int vit = 2 * it + sub;
         const int vs = vit % vstages, vph = (vit / vstages) & 1;
         const bool ok = mbar_wait(&bars->vfull[vs], vph, abort);
@@ -977,42 +1045,21 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
           vsum += n;
         }
       }
-      {
-        // attention score of key vt of this tile: the four warpgroups' partial sums, in order
-        const int ts = it & 1, use = it >> 1;
-        const bool okx = mbar_wait(&bars->xfull[ts], use & 1, abort);
-        const float* px = sx + ts * 512 + vt;
-        const float ex = (px[0] + px[128]) + (px[256] + px[384]);
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&bars->xempty[ts]);
-        const int ikey = ti.t * kTile + vt;
-        if (okx && ikey < P) {
-          ws.s_ex_raw[ppos(st, ti.layer, ti.h, ti.b, 0) + ikey] = ex;
-          // number of pooling windows (centres in [0, P)) that cover this position
-          const int cover = min(ikey, pool_half) + min(P - 1 - ikey, pool_half) + 1;
-          exw = fmaf(ex, (float)cover, exw);
-        }
-      }
-      if (seg_start) {
-        const float a = warp_min(vmin), b2 = warp_max(vmax), c2 = warp_sum(vsum),
-                    d2 = warp_sum(exw);
-        const int vw = warp - kAuxWarp0;
+      if (group_sync_stop(3, 128, vt == 0, abort, bars->vote[2], it)) break;
+      if (seg_start && use_vnorm) {
+        const float a = warp_min(vmin), b2 = warp_max(vmax), c2 = warp_sum(vsum);
+        const int vw = warp - kP2AuxWarp0;
         if (lane == 0) {
           sred[32 + vw] = a;
           sred[36 + vw] = b2;
           sred[40 + vw] = c2;
-          sred[44 + vw] = d2;
         }
         named_bar_sync(4, 128);
         if (vt == 0) {
-          if (use_vnorm)
-            ws.vstat[seg_first] = make_float4(
-                fminf(fminf(sred[32], sred[33]), fminf(sred[34], sred[35])),
-                fmaxf(fmaxf(sred[36], sred[37]), fmaxf(sred[38], sred[39])),
-                (sred[40] + sred[41]) + (sred[42] + sred[43]), 0.f);
-          // neutral diversity statistics, the window-count-weighted sum of the attention scores
-          ws.dstat[(size_t)seg_first * 2 + 1] = make_float4(
-              INFINITY, -INFINITY, 0.f, (sred[44] + sred[45]) + (sred[46] + sred[47]));
+          ws.vstat[seg_first] = make_float4(
+              fminf(fminf(sred[32], sred[33]), fminf(sred[34], sred[35])),
+              fmaxf(fmaxf(sred[36], sred[37]), fmaxf(sred[38], sred[39])),
+              (sred[40] + sred[41]) + (sred[42] + sred[43]), 0.f);
         }
         named_bar_sync(4, 128);
       }
@@ -1021,7 +1068,7 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == kP2WarpMma) tmem_dealloc(tmem, 512);
+  if (warp == kWarpMma) tmem_dealloc(tmem, 512);
   if (tid == 0 && bars->abort && status) atomicExch(status, MIXKV_ERR_TIMEOUT);
 }
 
@@ -1082,7 +1129,7 @@ size_t pass1_smem(int MB, int NQ) {
 }
 size_t pass2_smem(int NQ, int vstages) {
   return 1024 + (size_t)2 * (NQ + kExtraRows) * 128 + kP2KStages * kTileBytes +
-         (size_t)vstages * kVSubBytes + 512 * 4 + 1024 * 4 + 64 * 4 + sizeof(P2Bars) + 64;
+         (size_t)vstages * kVSubBytes + 512 * 4 + 64 * 4 + sizeof(P2Bars) + 64;
 }
 
 // cudaFuncSetAttribute once per (kernel, device).
@@ -1145,7 +1192,7 @@ cudaError_t launch_pass2(const LaunchCtx& c, const void* K, const void* V, const
   int vstages = kP2VStagesMax;
   while (vstages > 2 && pass2_smem(c.st.NQ, vstages) > kSmemLimit) --vstages;
   const size_t smem = pass2_smem(c.st.NQ, vstages);
-  return launch_pdl(k_pass2, dim3(c.st.g2), dim3(kThreads2), smem, c.stream, 1, tmK, tmV, tmQ, c.st,
+  return launch_pdl(k_pass2, dim3(c.st.g2), dim3(kP2Threads), smem, c.stream, 1, tmK, tmV, tmQ, c.st,
                     c.ws, s_div_out, c.scale_log2e, c.p.use_vnorm, c.p.pool_kernel >> 1,
                     vstages, status);
 }
