@@ -283,8 +283,8 @@ def run_mixkv(args):
                         ada_floor=wl.ada_floor)
     cu_list = None if wl.batch == 1 else [int(c) for c in wl.cu_seqlens]
     H, Ltot, NL = wl.kv_heads, wl.total_tokens, wl.layers
-    n_stage = binding.launches_per_layer(pg)
-    stage_names = binding.stage_names(pg)
+    stage_names = binding.stage_names_for(pg, NL, wl.batch, max(wl.seq_lens))
+    n_stage = len(stage_names)
 
     # ---- inputs: K, V [layers, H, Ltot, d] and Q [layers, batch, H*G, W, d] in pinned host
     # memory; enough device copies ("sets") that the bytes streamed between two uses of a

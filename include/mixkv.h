@@ -29,10 +29,17 @@
  *      rbar      [batch, H] fp32.
  *  - cu_seqlens_host: HOST pointer to batch+1 ascending int32 offsets, read during the
  *    call (not retained).  NULL means one sequence of length L (batch must be 1).
- *  - Return value: 0 on success, a negative mixkv_status otherwise; on error nothing has
- *    been enqueued.  Conditions only the device can see (a bounded wait inside a kernel
- *    expired) are written to *status_dev (device int32, optional, must be zeroed by the
- *    caller) as MIXKV_ERR_TIMEOUT; kernels never trap.
+ *  - Return value: 0 on success, a negative mixkv_status otherwise.  Argument errors
+ *    (INVALID_ARG, UNSUPPORTED, WORKSPACE_TOO_SMALL) enqueue nothing; MIXKV_ERR_CUDA means a
+ *    launch failed, earlier kernels of the call may already be enqueued and the outputs are
+ *    undefined.  A device whose compute capability is not 10.x gives MIXKV_ERR_UNSUPPORTED (the
+ *    kernels use tcgen05 / tensor memory; see mixkv_device_check).  Conditions only the
+ *    device can see (a bounded wait inside a kernel expired) are written to *status_dev
+ *    (device int32, optional, must be zeroed by the caller) as MIXKV_ERR_TIMEOUT; kernels
+ *    never trap.
+ *  - CUDA graphs: a call may be recorded into a stream capture and replayed, provided the
+ *    same entry point ran once on that device outside capture (its first use sets function
+ *    attributes); the host arrays (cu_seqlens_host) are read at capture time only.
  *  - Limits: head_dim == 128; 16 <= G*W <= 240 and G*W % 16 == 0; batch <= 64;
  *    every sequence needs L_b >= W + 1; budget > W; odd pool_kernel <= 63.
  */
@@ -127,12 +134,14 @@ int mixkv_scores(const void* K, const void* V, const void* Qwin,
  * MIXKV_STATIC_SCRATCH_BYTES that lives in the library's device image, so every GPU that
  * loads the library sets that much memory aside until the process exits.
  *  - Problems whose workspace (mixkv_workspace_size) would exceed the array are refused with
- *    MIXKV_ERR_STATIC_SCRATCH_EXCEEDED and nothing is enqueued.  As a guide the array covers
+ *    MIXKV_ERR_STATIC_SCRATCH_EXCEEDED before anything is enqueued (the size is worked out on
+ *    the host; the only CUDA calls before the refusal are attribute queries).  As a guide the array covers
  *    about 128k (head, token) pairs, e.g. H = 4 at L = 32768 or H = 8 at L = 16384.
  *  - The call performs no cudaMalloc / cudaFree and calls no allocating library routine.
  *  - The first call on each device looks up the array's device address (once per device, with
  *    that device current) and keeps it for later calls; make that first call outside any
- *    stream capture.
+ *    stream capture.  The kept address does not survive cudaDeviceReset: a process that resets
+ *    a device must not call this entry point on it afterwards.
  *  - All calls on one device share the one array, and it keeps whatever the previous call
  *    left in it.  Nothing in it needs to start from zero (every cell is written before it is
  *    read inside a call), but two calls whose kernels overlap on the GPU (different streams
@@ -154,7 +163,9 @@ int mixkv_scores_static(const void* K, const void* V, const void* Qwin,
  *   idx          out, packed in (b, h) order; capacity batch * H * (B - W) int32 is always
  *                enough
  *   counts       out, [batch * H], b_h
- *   idx_offsets  out, [batch * H + 1], exclusive prefix sum of counts */
+ *   idx_offsets  out, [batch * H + 1], exclusive prefix sum of counts
+ * status_dev is accepted for symmetry and never written: the kernels of this entry point
+ * contain no bounded waits. */
 int mixkv_select(const float* scores, const int32_t* cu_seqlens_host, int32_t batch, int32_t L,
                  const mixkv_params* p, void* workspace, size_t workspace_bytes,
                  int32_t* idx, int32_t* counts, int32_t* idx_offsets,
@@ -288,10 +299,25 @@ int mixkv_decode_attention(const void* K_cache, const void* V_cache,
                            int32_t head_dim, float softmax_scale, int32_t max_rows, float* out,
                            void* stream);
 
-/* Number of kernels one mixkv_compress_layer call enqueues for these parameters, and the
- * name of the i-th of them (NULL when i is out of range). */
+/* Number of kernels one mixkv_compress_layer[s] call enqueues, and the name of the i-th of
+ * them (NULL when i is out of range), for the measurement hook.  The route depends on the
+ * shape: fixed budgets take three kernels (pass1, pass2, tail; max pooling adds poolsum) while
+ * the candidates of the longest sequence fit the tail kernel's shared memory (P_b <= 131072)
+ * and add the unfused mix kernel beyond that; adaptive budgets always take the unfused route
+ * with the budget kernel.  The _for variants take the shape and follow the route the call
+ * takes; the short forms assume the fused route where it exists. */
 int mixkv_launches_per_layer(const mixkv_params* p);
 const char* mixkv_stage_name(const mixkv_params* p, int32_t i);
+int mixkv_launches_for(const mixkv_params* p, int32_t n_layers, int32_t batch,
+                       int32_t max_seq_len);
+const char* mixkv_stage_name_for(const mixkv_params* p, int32_t n_layers, int32_t batch,
+                                 int32_t max_seq_len, int32_t i);
+
+/* Whether the current device can run the library (no counterpart in the paper): MIXKV_OK for
+ * compute capability 10.x, MIXKV_ERR_UNSUPPORTED for any other device, MIXKV_ERR_CUDA when no
+ * device can be queried.  *cc_major_opt receives the major compute capability (0 when unknown).
+ * Every enqueueing entry point performs the same check (cached per device). */
+int mixkv_device_check(int32_t* cc_major_opt);
 
 /* Diagnostic (no counterpart in the paper): enqueues a one-CTA kernel that waits, through the
  * same bounded-wait helper as the pass kernels, on a barrier nothing arrives on.  After the

@@ -23,7 +23,8 @@ EXPORTS = ("mixkv_default_params", "mixkv_workspace_size", "mixkv_scores", "mixk
            "mixkv_workspace_size_layers", "mixkv_compress_layers",
            "mixkv_compress_layers_budgeted", "mixkv_layer_budget_schedule",
            "mixkv_similarity_workspace_size", "mixkv_similarity_map", "mixkv_decode_attention",
-           "mixkv_selftest_bounded_wait")
+           "mixkv_selftest_bounded_wait", "mixkv_launches_for", "mixkv_stage_name_for",
+           "mixkv_device_check")
 
 
 class MixKVError(RuntimeError):
@@ -86,6 +87,10 @@ def load_library() -> C.CDLL:
         lib.mixkv_workspace_size_layers.argtypes = [C.POINTER(_CParams), i32, i32, C.c_int64, i32,
                                                     C.POINTER(sz)]
         lib.mixkv_launches_per_layer.argtypes = [C.POINTER(_CParams)]
+        lib.mixkv_launches_for.argtypes = [C.POINTER(_CParams), i32, i32, i32]
+        lib.mixkv_stage_name_for.argtypes = [C.POINTER(_CParams), i32, i32, i32, i32]
+        lib.mixkv_stage_name_for.restype = C.c_char_p
+        lib.mixkv_device_check.argtypes = [C.POINTER(i32)]
         lib.mixkv_scores.argtypes = [vp, vp, vp, C.POINTER(i32), i32, i32, C.POINTER(_CParams),
                                      vp, sz, vp, vp, vp, vp, vp, vp, vp]
         lib.mixkv_scores_static.argtypes = [vp, vp, vp, C.POINTER(i32), i32, i32,
@@ -170,6 +175,23 @@ def stage_names(params: Params):
     pc = params.c()
     lib = load_library()
     return [lib.mixkv_stage_name(C.byref(pc), i).decode() for i in range(launches_per_layer(params))]
+
+
+def stage_names_for(params: Params, n_layers: int, batch: int, max_seq_len: int):
+    """Names of the kernels a call of this shape enqueues (mixkv_launches_for /
+    mixkv_stage_name_for): the route depends on the longest sequence and the number of units."""
+    pc = params.c()
+    lib = load_library()
+    n = int(lib.mixkv_launches_for(C.byref(pc), n_layers, batch, max_seq_len))
+    return [lib.mixkv_stage_name_for(C.byref(pc), n_layers, batch, max_seq_len, i).decode()
+            for i in range(n)]
+
+
+def device_check():
+    """mixkv_device_check: (status, major compute capability of the current device)."""
+    major = C.c_int32(0)
+    rc = int(load_library().mixkv_device_check(C.byref(major)))
+    return rc, int(major.value)
 
 
 def _workspace(params, cu, Ltot, device, workspace):

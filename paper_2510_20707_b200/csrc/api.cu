@@ -10,14 +10,34 @@
 
 namespace mixkv {
 
+// MIXKV_OK when the current device has compute capability 10.x (tcgen05, tensor memory), else
+// UNSUPPORTED; CUDA when the device cannot be queried.  Looked up once per device.
+int classify_cc(int major) { return major == 10 ? MIXKV_OK : MIXKV_ERR_UNSUPPORTED; }
+int device_check(int* major_out) {
+  static std::atomic<int> cached[64];   // 0 = unknown, else major + 1
+  int dev = 0;
+  if (major_out) *major_out = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return MIXKV_ERR_CUDA;
+  int major = 0;
+  if (dev >= 0 && dev < 64 && cached[dev].load(std::memory_order_relaxed) != 0) {
+    major = cached[dev].load(std::memory_order_relaxed) - 1;
+  } else {
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
+      return MIXKV_ERR_CUDA;
+    if (dev >= 0 && dev < 64) cached[dev].store(major + 1, std::memory_order_relaxed);
+  }
+  if (major_out) *major_out = major;
+  return classify_cc(major);
+}
+
 namespace {
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // A new 48-bit tag for every call.  The arrival counters pass 1 keeps in the caller's workspace
 // carry it, so counts left by an earlier call (or memory never written) read as "not this call"
-// and the workspace needs no clearing.  The sequence starts at a clock-derived value and steps by
-// an odd constant: no tag repeats within 2^48 calls of a process.
+// and the workspace needs no clearing.  Tags are 48 bits of a mixed 64-bit counter: random for
+// practical purposes, so a stale word matches a new call's tag with probability 2^-48.
 unsigned long long next_call_tag() {
   static std::atomic<unsigned long long> state{0};
   unsigned long long cur = state.load(std::memory_order_relaxed);
@@ -305,6 +325,8 @@ int mixkv_scores(const void* K, const void* V, const void* Qwin, const int32_t* 
   if (!K || !Qwin || !s_comp || (p->use_vnorm == MIXKV_INTRINSIC_VNORM && !V))
     return MIXKV_ERR_INVALID_ARG;
   if (!aligned16(K) || !aligned16(Qwin) || (V && !aligned16(V))) return MIXKV_ERR_INVALID_ARG;
+  rc = device_check(nullptr);   // last: every argument error is reported without a device
+  if (rc != MIXKV_OK) return rc;
   return enqueue_scores(c, K, V, Qwin, s_comp, s_ex_opt, s_div_opt, rbar_opt, rbar_in_opt,
                         status_dev);
 }
@@ -317,6 +339,8 @@ int mixkv_select(const float* scores, const int32_t* cu_seqlens_host, int32_t ba
   int rc = make_ctx(p, cu_seqlens_host, batch, L, workspace, workspace_bytes, stream, &c);
   if (rc != MIXKV_OK) return rc;
   if (!scores || !idx || !counts || !idx_offsets) return MIXKV_ERR_INVALID_ARG;
+  rc = device_check(nullptr);
+  if (rc != MIXKV_OK) return rc;
   TailArgs t;
   memset(&t, 0, sizeof(t));
   t.idx = idx;
@@ -345,6 +369,9 @@ int compress_impl(const void* K, const void* V, const void* Qwin, int n_layers,
   if (!K || !V || !Qwin || !K_out || !V_out || !out_row_offsets) return MIXKV_ERR_INVALID_ARG;
   if (!aligned16(K) || !aligned16(V) || !aligned16(Qwin) || !aligned16(K_out) || !aligned16(V_out))
     return MIXKV_ERR_INVALID_ARG;
+  if (head_budgets && p->budget_mode != MIXKV_BUDGET_FIXED) return MIXKV_ERR_INVALID_ARG;
+  rc = device_check(nullptr);
+  if (rc != MIXKV_OK) return rc;
   float* s_comp = s_comp_opt ? s_comp_opt : c.ws.s_comp;
   int* counts = counts_opt ? counts_opt : c.ws.counts;
   TailArgs t;
@@ -507,7 +534,8 @@ int mixkv_scores_static(const void* K, const void* V, const void* Qwin,
                         const mixkv_params* p, float* s_comp, float* s_ex_opt, float* s_div_opt,
                         float* rbar_opt, const float* rbar_in_opt, int32_t* status_dev,
                         void* stream) {
-  // size the problem on the host first: too large a problem is refused before any CUDA call
+  // size the problem on the host first: too large a problem is refused before anything is
+  // enqueued (only attribute queries have run by then)
   {
     int rc = check_params(p);
     if (rc != MIXKV_OK) return rc;
@@ -525,6 +553,41 @@ int mixkv_scores_static(const void* K, const void* V, const void* Qwin,
   return mixkv_scores(K, V, Qwin, cu_seqlens_host, batch, L, p, scratch,
                       (size_t)MIXKV_STATIC_SCRATCH_BYTES, s_comp, s_ex_opt, s_div_opt, rbar_opt,
                       rbar_in_opt, status_dev, stream);
+}
+
+namespace {
+// Whether a call of this shape takes the fused tail (what tail_can_fuse decides at launch).
+bool fused_route(const mixkv_params* p, int n_layers, int batch, int max_seq_len) {
+  LaunchCtx c;
+  memset(&c, 0, sizeof(c));
+  c.st.layers = n_layers;
+  c.st.batch = batch;
+  c.st.H = p->kv_heads;
+  c.max_prefix = max_seq_len - p->window;
+  return p->budget_mode == MIXKV_BUDGET_FIXED && tail_can_fuse(c);
+}
+}  // namespace
+
+int mixkv_launches_for(const mixkv_params* p, int32_t n_layers, int32_t batch,
+                       int32_t max_seq_len) {
+  if (!p || n_layers < 1 || batch < 1 || max_seq_len <= p->window) return 0;
+  const char* names[8];
+  return layer_stages(p, fused_route(p, n_layers, batch, max_seq_len), names);
+}
+
+const char* mixkv_stage_name_for(const mixkv_params* p, int32_t n_layers, int32_t batch,
+                                 int32_t max_seq_len, int32_t i) {
+  if (!p || n_layers < 1 || batch < 1 || max_seq_len <= p->window) return nullptr;
+  const char* names[8];
+  const int n = layer_stages(p, fused_route(p, n_layers, batch, max_seq_len), names);
+  return (i >= 0 && i < n) ? names[i] : nullptr;
+}
+
+int mixkv_device_check(int32_t* cc_major_opt) {
+  int major = 0;
+  const int rc = device_check(&major);
+  if (cc_major_opt) *cc_major_opt = major;
+  return rc;
 }
 
 const char* mixkv_stage_name(const mixkv_params* p, int32_t i) {

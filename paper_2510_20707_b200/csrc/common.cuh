@@ -99,6 +99,9 @@ cudaError_t launch_pass1(const LaunchCtx& c, const void* K, const void* Q, float
 cudaError_t launch_pass2(const LaunchCtx& c, const void* K, const void* V, const void* Q,
                          float* s_div_out, int* status);
 int device_sm_count();
+// MIXKV_OK on a compute-capability 10.x device, MIXKV_ERR_UNSUPPORTED on any other,
+// MIXKV_ERR_CUDA when none can be queried; *major_out (optional) receives the major number.
+int device_check(int* major_out);
 cudaError_t launch_poolsum(const LaunchCtx& c);
 cudaError_t launch_mixpool(const LaunchCtx& c, const float* s_div, const float* rbar_in,
                            float* s_ex_out, float* s_comp);

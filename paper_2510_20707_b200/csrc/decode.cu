@@ -123,6 +123,10 @@ extern "C" int mixkv_decode_attention(const void* K_cache, const void* V_cache,
     return MIXKV_ERR_INVALID_ARG;
   const size_t smem = ((size_t)gqa_ratio * kHeadDim + (size_t)gqa_ratio * max_rows) * 4;
   if (smem > 160 * 1024) return MIXKV_ERR_UNSUPPORTED;
+  {
+    const int rc = device_check(nullptr);
+    if (rc != MIXKV_OK) return rc;
+  }
   if (smem > 48 * 1024) {
     static bool done[64] = {false};
     int dev = 0;

@@ -192,6 +192,10 @@ int mixkv_similarity_map(const void* X, int32_t heads, int32_t L, int32_t head_d
   const long long T = ((long long)L + block - 1) / block;
   const long long S = ((long long)block + kSimRows - 1) / kSimRows;
   if (T > 65535 || heads > 65535 || T * S > 0x7fffffffLL) return MIXKV_ERR_UNSUPPORTED;   // grid limits
+  {
+    const int rc = device_check(nullptr);
+    if (rc != MIXKV_OK) return rc;
+  }
   unsigned char* wsb = reinterpret_cast<unsigned char*>(workspace);
   float* u = reinterpret_cast<float*>(wsb);
   wsb += align256((size_t)heads * T * kHeadDim * 4);

@@ -77,3 +77,25 @@ def test_entry_points_validate_before_any_cuda_call(lib):
                             None, None, None, None, None) == -1
     assert lib.mixkv_select(None, None, 1, 1024, C.byref(p), wsp, 1 << 19, one, one, one, None,
                             None) == -1
+
+
+def test_stage_names_follow_the_route(lib):
+    p = binding.Params(kv_heads=4, gqa_ratio=7, budget=256)
+    assert binding.stage_names_for(p, 28, 1, 32768) == ["pass1", "pass2", "tail"]
+    # one head-layer of 140000 candidates does not fit the tail kernel's shared memory
+    assert binding.stage_names_for(p, 1, 1, 140032) == ["pass1", "pass2", "mixpool", "tail"]
+    # 112 units of 65504 candidates: too long for one CTA per head, clusters of eight keep them
+    assert binding.stage_names_for(p, 28, 1, 65536) == ["pass1", "pass2", "tail"]
+    pa = binding.Params(kv_heads=4, gqa_ratio=7, budget=128, budget_mode=1)
+    assert binding.stage_names_for(pa, 28, 8, 8192) == ["pass1", "pass2", "mixpool", "budget", "tail"]
+    assert binding.stage_names(p) == ["pass1", "pass2", "tail"]
+
+
+def test_device_check_without_a_device_or_with_one(lib):
+    # no GPU here: the query fails and the entry point says so; on a B200 it reports 10.x
+    import torch
+    rc, major = binding.device_check()
+    if torch.cuda.is_available():
+        assert (rc, major) == (0, 10)
+    else:
+        assert rc == -4 and major == 0

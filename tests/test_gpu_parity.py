@@ -6,8 +6,8 @@ import torch
 
 import oracle
 from paper_2510_20707_b200 import binding, synth
-from parity import (check_rbar, check_scores, check_selection, params_pair, run_layer_parity,
-                    run_layers_parity, to_bits, to_dev)
+from parity import (check_gather, check_rbar, check_scores, check_selection, params_pair,
+                    run_layer_parity, run_layers_parity, to_bits, to_dev)
 
 pytestmark = pytest.mark.gpu
 
@@ -308,6 +308,45 @@ def test_workspace_needs_no_clearing():
         assert torch.equal(first["idx"][:n_idx], out["idx"][:n_idx])
         assert torch.equal(first["K_out"][:n_rows].view(torch.int16), out["K_out"][:n_rows].view(torch.int16))
         assert torch.equal(first["V_out"][:n_rows].view(torch.int16), out["V_out"][:n_rows].view(torch.int16))
+
+
+def test_graph_capture_and_replay():
+    # A call recorded into a CUDA graph keeps its host-side call tag, so every replay meets the
+    # arrival counters of the run before it in the workspace: the last arrival of a head leaves
+    # its counter at zero under the tag, and a replay counts afresh.  Two replays on new K / V /
+    # Q (copied into the captured buffers) must each match the oracle.
+    wl = synth.small_workload(H=3, G=4, W=16, seq_lens=(2600, 900), pool_kernel=5, budget=80,
+                              seed=71, centroids=8)
+    po, pg = params_pair(wl)
+    cu = wl.cu_seqlens
+    cu_list = [int(c) for c in cu]
+    xs = [synth.make_layer(wl, layer, "calibrated") for layer in range(3)]
+    K, V, Q = (to_dev(xs[0][k]).clone() for k in ("K", "V", "Q"))
+    ws = torch.empty(binding.workspace_size(pg, wl.batch, wl.total_tokens, max(wl.seq_lens)),
+                     dtype=torch.uint8, device="cuda")
+    out = binding.compress_layer(K, V, Q, pg, cu_seqlens=cu_list, workspace=ws)   # outside capture
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.graph(graph, stream=side):
+        binding.compress_layer(K, V, Q, pg, cu_seqlens=cu_list, workspace=ws, out=out)
+    H, W = wl.kv_heads, wl.window
+    for x in xs[1:]:
+        K.copy_(to_dev(x["K"])), V.copy_(to_dev(x["V"])), Q.copy_(to_dev(x["Q"]))
+        out["status"].zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert int(out["status"].item()) == 0
+        ref_s = oracle.scores(x["K"], x["V"], x["Q"], po, cu=cu)
+        ref = oracle.select(ref_s["s_comp"], po, cu=cu)
+        check_scores("s_comp", out["s_comp"].cpu().numpy(), ref_s["s_comp"], cu, W)
+        offs = out["idx_offsets"].cpu().numpy()
+        idx = out["idx"].cpu().numpy()
+        check_selection(idx, offs, out["counts"].cpu().numpy(), ref, ref_s["s_comp"], cu, W, H)
+        ro = out["out_row_offsets"].cpu().numpy()
+        check_gather(x["K"], to_bits(out["K_out"]), ro, idx, offs, cu, W, H)
+        check_gather(x["V"], to_bits(out["V_out"]), ro, idx, offs, cu, W, H)
 
 
 def test_given_head_budgets_ragged():
