@@ -146,9 +146,7 @@ void carve(const mixkv_params* p, const SeqTable& st, unsigned char* base, Works
   ws->s_ex_raw = (float*)take(NL * H * st.Ptot * 4);
   ws->s_div = (float*)take(NL * H * st.Ptot * 4);
   ws->s_comp = (float*)take(NL * H * st.Ptot * 4);
-  // partial softmax statistics per segment and window row: one per epilogue group, and per key
-  // half where the query tile is a single 128-row block
-  ws->rowstat = (float2*)take(NL * st.nt1 * (st.NQ <= 128 ? 4 : 2) * st.NQ * 8);
+  ws->rowstat = (float2*)take(NL * st.nt1 * st.NQ * 8);
   ws->ksum = (float*)take(NL * st.nt1 * kHeadDim * 4);
   ws->vstat = (float4*)take(NL * st.nt2 * 16);
   ws->dstat = (float4*)take(NL * st.nt2 * 2 * 16);

@@ -52,7 +52,7 @@ struct Workspace {
   float* s_comp;      // [H, Ptot]
   // per-segment partial results; a segment is a run of tiles of one (b, h) inside one CTA's
   // range and its slot is the id of its first tile
-  float2* rowstat;    // [nt1, 2 or 4, NQ]  softmax (max, sum) of each window row, log2 units
+  float2* rowstat;    // [nt1, NQ]  softmax (reference, sum) of each window row, log2 units
   float* ksum;        // [nt1, d]      sum of unit keys
   float4* vstat;      // [nt2]         (min, max, sum, -) of |V_i| over candidates
   float4* dstat;      // [nt2, 2]      per epilogue warpgroup: (min, max, sum) of s_div, window-count-weighted sum of s_ex_raw

@@ -158,9 +158,11 @@ constexpr size_t kSmemLimit = 227 * 1024;   // dynamic shared memory a CTA may a
 __host__ __device__ constexpr int p1_aux_warps(int MB) { return 8; }
 __host__ __device__ constexpr int p1_threads(int MB) { return (kAuxWarp0 + p1_aux_warps(MB)) * 32; }
 constexpr int kP1MaxStages = 6;
+constexpr int kP1XRows = 3 * 128;   // row statistics exchanged between the warpgroups of a query row
 // K tile ring: as deep as shared memory allows next to the query tile (the deeper the ring, the
 // more bytes in flight towards HBM)
-__host__ __device__ constexpr int p1_stages(int MB) { return 5; }
+// (the widest query tiles leave room for four)
+__host__ __device__ constexpr int p1_stages(int NQ) { return NQ > 224 ? 4 : 5; }
 // registers per thread: at launch, then per role (7 warpgroups: 40 + 4 * 72 + 2 * 88 = 7 * 72;
 // the key-statistics warps hold a batch of eight key rows in registers between their two sweeps)
 #ifndef P1_LEAD
@@ -185,21 +187,19 @@ struct P1Bars {
 // ---- per-head folds at the end of pass 1 (once per (layer, sequence, head), in the CTA that
 // delivers the head's last segment)
 //
-// All segments' softmax (max, sum) of window row q -> minus the log2 of the row's normaliser.
-// NU partial results per segment and row.
-template <int NU>
-__device__ __forceinline__ float fold_row_stats(const float2* rowstat, const SegList& sl,
-                                                const int NQ, const int q) {
-  const int total = sl.nseg * NU;
+// Softmax (reference, sum) pairs of window row q over the segments e = half, half + 2, ... of
+// the head: the caller's partner thread takes the other half.
+__device__ __forceinline__ float2 fold_row_stats(const float2* rowstat, const SegList& sl,
+                                                 const int NQ, const int q, const int half) {
   float Mx = -1e30f, Zs = 0.f;
 #pragma unroll 1
-  for (int i0 = 0; i0 < total; i0 += 12) {   // twelve loads in flight
+  for (int e0 = half; e0 < sl.nseg; e0 += 24) {   // twelve loads in flight
     float2 v[12];
 #pragma unroll
     for (int k = 0; k < 12; ++k) {
-      const int i = i0 + k;
+      const int e = e0 + 2 * k;
       v[k] = make_float2(-1e30f, 0.f);
-      if (i < total) v[k] = __ldcg(rowstat + ((size_t)sl.start(i / NU) * NU + (i % NU)) * NQ + q);
+      if (e < sl.nseg) v[k] = __ldcg(rowstat + (size_t)sl.start(e) * NQ + q);
     }
 #pragma unroll
     for (int k = 0; k < 12; ++k) {
@@ -208,34 +208,39 @@ __device__ __forceinline__ float fold_row_stats(const float2* rowstat, const Seg
       Mx = mn;
     }
   }
-  return -(Mx + log2f(Zs));
+  return make_float2(Mx, Zs);
 }
-// Sum over the head's segments of component kt of their unit-key sums.
-__device__ __forceinline__ float fold_key_sums(const float* ksum, const SegList& sl, const int kt) {
+// (m, z) pairs of the same row merged: z0 2^m0 + z1 2^m1 under the larger reference.
+__device__ __forceinline__ float2 merge_stats(const float2 a, const float2 b) {
+  const float mn = fmaxf(a.x, b.x);
+  return make_float2(mn, a.y * ex2(a.x - mn) + b.y * ex2(b.x - mn));
+}
+// Component kt of the unit-key sums over the segments e = half, half + 2, ... of the head.
+__device__ __forceinline__ float fold_key_sums(const float* ksum, const SegList& sl, const int kt,
+                                               const int half) {
   float sum = 0.f;
 #pragma unroll 1
-  for (int e0 = 0; e0 < sl.nseg; e0 += 12) {   // twelve loads in flight
+  for (int e0 = half; e0 < sl.nseg; e0 += 24) {   // twelve loads in flight
     float v[12];
 #pragma unroll
-    for (int e = 0; e < 12; ++e)
-      v[e] = e0 + e < sl.nseg ? __ldcg(ksum + (size_t)sl.start(e0 + e) * kHeadDim + kt) : 0.f;
+    for (int k = 0; k < 12; ++k)
+      v[k] = e0 + 2 * k < sl.nseg ? __ldcg(ksum + (size_t)sl.start(e0 + 2 * k) * kHeadDim + kt) : 0.f;
 #pragma unroll
-    for (int e = 0; e < 12; ++e) sum += v[e];
+    for (int k = 0; k < 12; ++k) sum += v[k];
   }
   return sum;
 }
-// Walks the segments of the CTA's tile range [lo, hi); every epilogue thread (et = 0 .. 511)
-// calls it after the barrier that ends the tile loops.  Threads 0 .. NQ-1 fold the row
-// statistics, threads 256 .. 383 the key sums.  `red` is shared scratch of four floats, `flag` a
-// shared int.  Named barrier 5 joins the epilogue threads.
-template <int MB>
+constexpr int kFoldThreads = kEpiThreads + 256;   // the epilogue and the key-statistics warps
+// Walks the segments of the CTA's tile range [lo, hi); the epilogue threads (et = 0 .. 511, else
+// -1) and the key-statistics threads (at = 0 .. 255, else -1) call it after the barrier that
+// ends the tile loops.  Two epilogue threads per window row fold the row statistics, two
+// key-statistics threads per dimension the key sums.  `red` is shared scratch of eight floats,
+// `flag` a shared int.  Named barrier 5 joins the callers.
 __device__ __forceinline__ void finish_heads(const SeqTable& st, const Workspace& ws, const int lo,
                                              const int hi, const unsigned long long call_tag,
                                              float* __restrict__ rbar_out, float* red, int* flag,
-                                             const int et) {
-  const int lane = et & 31;
+                                             const int et, const int at) {
   const int NQ = st.NQ, H = st.H;
-  constexpr int NU = MB == 2 ? 2 : 4;
   int id = lo;
   while (id < hi) {
     const TileIter ti(st.tile1_start, st.batch, H, st.nt1, id, hi);
@@ -245,24 +250,31 @@ __device__ __forceinline__ void finish_heads(const SeqTable& st, const Workspace
     const SegList sl(ti.layer * st.nt1 + st.tile1_start[ti.b] + ti.h * per_head, per_head,
                      split1(st));
     if (et == 0) *flag = arrive_last(ws.headcnt + unit, call_tag, sl.nseg);
-    named_bar_sync(5, kEpiThreads);
+    named_bar_sync(5, kFoldThreads);
     const bool last = *flag != 0;
     if (last) {
-      if (et < NQ)
-        ws.bq[(size_t)unit * NQ + et] =
-            fold_row_stats<NU>(ws.rowstat, sl, NQ, et) - log2f((float)st.W);
-      const int kt = et - 256;
-      float sum = 0.f;
-      if (kt >= 0 && kt < kHeadDim) {
-        sum = fold_key_sums(ws.ksum, sl, kt);
-        ws.kbar[(size_t)unit * kHeadDim + kt] = sum / (float)L;
-        const float n2 = warp_sum(sum * sum);
-        if (lane == 0) red[kt >> 5] = n2;
+      if (et >= 0 && et < 2 * NQ) {   // 2 NQ is a multiple of 32: whole warps, partners in adjacent lanes
+        float2 mz = fold_row_stats(ws.rowstat, sl, NQ, et >> 1, et & 1);
+        const float2 other = make_float2(__shfl_xor_sync(0xffffffffu, mz.x, 1),
+                                         __shfl_xor_sync(0xffffffffu, mz.y, 1));
+        mz = (et & 1) ? merge_stats(other, mz) : merge_stats(mz, other);
+        if ((et & 1) == 0)
+          ws.bq[(size_t)unit * NQ + (et >> 1)] = -(mz.x + log2f(mz.y)) - log2f((float)st.W);
+      }
+      if (at >= 0) {
+        const int kt = at >> 1;
+        float sum = fold_key_sums(ws.ksum, sl, kt, at & 1);
+        const float o = __shfl_xor_sync(0xffffffffu, sum, 1);
+        sum = (at & 1) ? o + sum : sum + o;
+        if ((at & 1) == 0) ws.kbar[(size_t)unit * kHeadDim + kt] = sum / (float)L;
+        const float n2 = warp_sum((at & 1) ? 0.f : sum * sum);
+        if ((at & 31) == 0) red[at >> 5] = n2;
       }
     }
-    named_bar_sync(5, kEpiThreads);   // `flag` may be rewritten; the four partial norms are in `red`
-    if (last && et == 256) {
-      const double nn = ((double)red[0] + (double)red[1]) + ((double)red[2] + (double)red[3]);
+    named_bar_sync(5, kFoldThreads);   // `flag` may be rewritten; the eight partial norms are in `red`
+    if (last && at == 0) {
+      double nn = 0.0;
+      for (int w = 0; w < 8; ++w) nn += (double)red[w];
       const double T = (double)L;
       const float r = (float)((nn - T) / (T * (T - 1.0)));   // Eq. 4
       ws.rbar[unit] = r;
@@ -271,7 +283,7 @@ __device__ __forceinline__ void finish_heads(const SeqTable& st, const Workspace
       // so that a replay of the same launch (a captured graph keeps its tag) counts afresh
       ws.headcnt[unit] = call_tag << 16;
     }
-    named_bar_sync(5, kEpiThreads);   // `red` is free again
+    named_bar_sync(5, kFoldThreads);   // `red` is free again
     id += min(hi - id, per_head - ti.t);
   }
 }
@@ -348,9 +360,9 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* base =
       reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
-  constexpr int kP1Stages = p1_stages(MB);
+  const int kP1Stages = p1_stages(st.NQ);
   constexpr int kP1AuxWarps = p1_aux_warps(MB);
-  constexpr int NU = MB == 2 ? 2 : 4;   // partial row statistics per segment and row
+  constexpr int NU = MB == 2 ? 2 : 4;   // warpgroups that share a query row
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int NQ = st.NQ, W = st.W, H = st.H;
   // The query tile holds exactly NQ rows per 64-column half.  The MMA reads MB * 128 rows: the
@@ -359,7 +371,8 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
   unsigned char* sQ = base;                    // 2 halves x [NQ x 128 B]
   unsigned char* sK = sQ + 2 * NQ * 128;       // kP1Stages x 32 KB
   float* sks = reinterpret_cast<float*>(sK + kP1Stages * kTileBytes);  // [aux warps][128] key-sum exchange
-  P1Bars* bars = reinterpret_cast<P1Bars*>(sks + kP1AuxWarps * 128);
+  float2* sxs = reinterpret_cast<float2*>(sks + kP1AuxWarps * 128);    // [kP1XRows] row statistics handed over
+  P1Bars* bars = reinterpret_cast<P1Bars*>(sxs + kP1XRows);
   {
     // the carve-up above must fit behind the (1 KB aligned) base
     unsigned dyn;
@@ -486,8 +499,13 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
     const int col0 = blk * 128 + unit * NC;
     const bool warp_on = blk * 128 + quarter * 32 < NQ;
     const int jrow = row % W;
+    // The NU warpgroups that share a query row merge their statistics at the end of a segment:
+    // units 1 .. NU-1 hand theirs over through shared memory, unit 0 merges and writes one pair
+    // per row.  Named barriers 6 + blk ("handed over") and 8 + blk ("read").
+    const int xrow = (unit > 0 ? unit - 1 : 0) * 128 + (MB == 2 ? blk * 128 : 0) + quarter * 32 + lane;
+    constexpr int kXThreads = NU * 128;
     float m_run = -1e30f, z_run = 0.f;
-    int it = 0, seg_first = lo;
+    int it = 0, seg_first = lo, segs_done = 0;
     bool seg_start = true, no_ref = true;
     for (TileIter ti(st.tile1_start, st.batch, H, st.nt1, lo, hi); ti.valid(); ti.next()) {
       if (seg_start) {
@@ -499,9 +517,11 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
       seg_start = ti.seg_last();
       const int L = st.cu[ti.b + 1] - st.cu[ti.b], P = L - W;
       const int ts = it & 1, tph = (it >> 1) & 1;
-      if (!mbar_wait(&bars->tfull[ts], tph, abort)) break;
+      // (after an abort the waits fail at once; the loop goes on without work so that the
+      // segment-end barriers below stay matched)
+      const bool ok = mbar_wait(&bars->tfull[ts], tph, abort);
       tc_fence_after();
-      if (warp_on) {
+      if (ok && warp_on) {
         const int k0 = ti.t * kTile + unit * NC;
         const bool need_mask = ti.t * kTile + kTile > P;
         const int lim = P + jrow;   // last key this row may see
@@ -532,8 +552,21 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
       tc_fence_before();
       __syncwarp();   // one arrival per warp: 512 single arrivals on one word cost more than a chunk
       if (lane == 0) mbar_arrive(&bars->tempty[ts]);
-      if (seg_start && row < NQ)
-        ws.rowstat[((size_t)seg_first * NU + unit) * NQ + row] = make_float2(m_run, z_run);
+      if (seg_start) {   // (here: this was the segment's last tile)
+        if (unit > 0) {
+          if (segs_done > 0) named_bar_sync(8 + blk, kXThreads);   // the last hand-over was read
+          sxs[xrow] = make_float2(m_run, z_run);
+          named_bar_arrive(6 + blk, kXThreads);
+        } else {
+          named_bar_sync(6 + blk, kXThreads);
+          float2 mz = make_float2(m_run, z_run);
+#pragma unroll
+          for (int u = 1; u < NU; ++u) mz = merge_stats(mz, sxs[xrow + (u - 1) * 128]);
+          named_bar_arrive(8 + blk, kXThreads);
+          if (row < NQ) ws.rowstat[(size_t)seg_first * NQ + row] = mz;
+        }
+        ++segs_done;
+      }
       ++it;
     }
   } else {
@@ -647,12 +680,10 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
   // what pass 2 reads: one log2 normaliser per window row (the 1/W of the window mean folded
   // in), the mean unit key, the redundancy of Eq. 4.  The epilogue warps do it (they hold the
   // registers).
-#ifndef DIAG_NO_FINISH
-  if (warp >= kEpiWarp0 && warp < kAuxWarp0)
-#else
-  if (warp > 1000)
-#endif
-    finish_heads<MB>(st, ws, lo, hi, call_tag, rbar_out, sks, &bars->last, tid - kEpiWarp0 * 32);
+  if (warp >= kEpiWarp0)
+    finish_heads(st, ws, lo, hi, call_tag, rbar_out, sks, &bars->last,
+                 warp < kAuxWarp0 ? tid - kEpiWarp0 * 32 : -1,
+                 warp < kAuxWarp0 ? -1 : tid - kAuxWarp0 * 32);
 }
 
 // ======================================================================== pass 2
@@ -1122,8 +1153,8 @@ bool map_q(const LaunchCtx& c, const void* Q, CUtensorMap* tm) {
 size_t pass1_smem(int MB, int NQ) {
   // up to 1023 bytes of alignment slack in front of the carve-up; never beyond the limit (the
   // kernel checks that its carve-up fits behind the aligned base)
-  const size_t need = (size_t)2 * NQ * 128 + (size_t)p1_stages(MB) * kTileBytes + p1_aux_warps(MB) * 128 * 4 +
-                      sizeof(P1Bars);
+  const size_t need = (size_t)2 * NQ * 128 + (size_t)p1_stages(NQ) * kTileBytes + p1_aux_warps(MB) * 128 * 4 +
+                      kP1XRows * 8 + sizeof(P1Bars);
   const size_t want = need + 1024;
   return want < kSmemLimit ? want : kSmemLimit;
 }

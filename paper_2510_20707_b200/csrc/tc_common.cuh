@@ -231,6 +231,13 @@ __device__ __forceinline__ void named_bar_sync(int id, int threads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
 
+// Arrives at a named barrier without waiting (the other side calls named_bar_sync with the
+// same thread count); shared-memory writes before it are visible to the threads that sync.
+__device__ __forceinline__ void named_bar_arrive(int id, int threads) {
+  __threadfence_block();
+  asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
 // Byte offset of element (row r, 16-byte chunk c in 0..7) inside a [rows x 128 B] half tile
 // written with the 128-byte swizzle (tile base 1024-byte aligned).
 __device__ __forceinline__ uint32_t sw128_offset(int r, int c) {
