@@ -274,8 +274,12 @@ int mixkv_layer_budget_schedule(int32_t n_layers, int32_t budget, int32_t window
  *   mean_opt   device, [heads] fp32 or NULL: mean over all ordered pairs i != j of the head,
  *              the redundancy of Eq. 4
  *   workspace  device, mixkv_similarity_workspace_size bytes, 16-byte aligned, caller-owned
- * A zero row has cosine 0 with every row.  Enqueues three small kernels on `stream`; reads X
- * once.  Errors as for the other entry points. */
+ * A zero row has cosine 0 with every row.  Two routes: for block = 1, 2, 4, 8 or 16 the dense
+ * matrix X^ X^T of Eq. 3 is formed on the tensor cores (rows normalised once into two bf16
+ * halves, upper triangle of 128 x 128 tiles, cells reduced in the epilogue); for every other
+ * block size the cells come from the Gram matrix of the per-block sums of unit rows (one
+ * streaming pass over X).  The workspace size depends on the route.  Errors as for the other
+ * entry points. */
 int mixkv_similarity_workspace_size(int32_t heads, int32_t L, int32_t block, size_t* bytes);
 int mixkv_similarity_map(const void* X, int32_t heads, int32_t L, int32_t head_dim, int32_t block,
                          void* workspace, size_t workspace_bytes, float* cells, float* mean_opt,
@@ -289,8 +293,11 @@ int mixkv_similarity_map(const void* X, int32_t heads, int32_t L, int32_t head_d
  *   out_row_offsets    device, [n_layers, batch * H + 1]: rows of (b, h) inside a layer's slice
  *   rows_cap           rows between the slices of consecutive layers (batch * H * B)
  *   q                  device, [n_layers, batch, H * G, d] bf16: the token's query per layer
- *   max_rows           upper bound on the rows of one (layer, b, h), e.g. B; sizes shared memory
- *                      (G * (128 + max_rows) floats <= 160 KB); rows beyond it are not read
+ *   max_rows           upper bound on the rows of one (layer, b, h), e.g. B, or L for a cache
+ *                      that was not compressed; rows beyond it are not read.  It only steers
+ *                      how many CTAs share one head (a cluster of 1, 2, 4 or 8 splits the rows;
+ *                      each CTA walks its share in blocks of 256 with a running softmax), so
+ *                      any length is accepted
  *   out                device, [n_layers, batch, H * G, d] fp32; a head without rows gets zeros
  * softmax_scale 0 means 1 / sqrt(d).  d must be 128, G <= 16 (else MIXKV_ERR_UNSUPPORTED). */
 int mixkv_decode_attention(const void* K_cache, const void* V_cache,

@@ -99,6 +99,10 @@ cudaError_t launch_pass1(const LaunchCtx& c, const void* K, const void* Q, float
 cudaError_t launch_pass2(const LaunchCtx& c, const void* K, const void* V, const void* Q,
                          float* s_div_out, int* status);
 int device_sm_count();
+// Fills a CUtensorMap (passed as void*) for a bf16 tensor of the given rank: dims innermost first,
+// strides in bytes of dimensions 1 .. rank-1, box extents; 128-byte swizzle, zero fill outside.
+bool encode_bf16_map(void* tm, const void* base, int rank, const unsigned long long* dims,
+                     const unsigned long long* strides_bytes, const unsigned* box);
 // MIXKV_OK on a compute-capability 10.x device, MIXKV_ERR_UNSUPPORTED on any other,
 // MIXKV_ERR_CUDA when none can be queried; *major_out (optional) receives the major number.
 int device_check(int* major_out);
@@ -119,6 +123,13 @@ __host__ __device__ __forceinline__ size_t ppos(const SeqTable& st, int layer, i
                                                 int i) {
   return ((size_t)layer * st.H + h) * st.Ptot + (st.cu[b] - b * st.W) + i;
 }
+
+// Dense (tensor-core) route of the similarity map for block = 1, 2, 4, 8, 16 (similarity_tc.cu).
+bool similarity_dense_block(int block);
+size_t similarity_dense_workspace(int heads, int L);
+cudaError_t launch_similarity_dense(const void* X, int heads, int L, int block, void* workspace,
+                                    float* cells, float** u_out, int** nz_out, int* slices_out,
+                                    cudaStream_t s);
 
 struct TailArgs {
   const float* scores;

@@ -3,7 +3,9 @@
 // one tensor.  The mean of cos(x_i, x_j) over a cell (i in block I, j in block J) is
 // u_I . u_J / (n_I n_J) with u_I the sum of the unit rows of block I, the same identity that
 // turns the mean of the whole matrix into Eq. 4; so the map needs one streaming pass over the
-// rows (HBM bound) and a small Gram matrix of the block sums, not the L x L matrix.
+// rows (HBM bound) and a small Gram matrix of the block sums, not the L x L matrix.  That is the
+// route for coarse maps; with 1 .. 16 rows per cell the Gram of block sums is the L x L
+// contraction itself and runs on the tensor cores (similarity_tc.cu).
 #include "common.cuh"
 
 namespace mixkv {
@@ -172,6 +174,10 @@ extern "C" {
 
 int mixkv_similarity_workspace_size(int32_t heads, int32_t L, int32_t block, size_t* bytes) {
   if (!bytes || heads < 1 || L < 1 || block < 1) return MIXKV_ERR_INVALID_ARG;
+  if (similarity_dense_block(block)) {
+    *bytes = similarity_dense_workspace(heads, L);
+    return MIXKV_OK;
+  }
   const size_t T = ((size_t)L + block - 1) / block;
   const size_t S = ((size_t)block + kSimRows - 1) / kSimRows;   // slices per block
   *bytes = align256((size_t)heads * T * kHeadDim * 4) + align256((size_t)heads * T * 4);
@@ -196,12 +202,22 @@ int mixkv_similarity_map(const void* X, int32_t heads, int32_t L, int32_t head_d
     const int rc = device_check(nullptr);
     if (rc != MIXKV_OK) return rc;
   }
+  cudaStream_t s = (cudaStream_t)stream;
+  if (similarity_dense_block(block)) {
+    float* ud = nullptr;
+    int* nzd = nullptr;
+    int slices = 0;
+    if (launch_similarity_dense(X, heads, L, block, workspace, cells, &ud, &nzd, &slices, s) !=
+        cudaSuccess)
+      return MIXKV_ERR_CUDA;
+    if (mean_opt) k_head_mean<<<(unsigned)heads, 1024, 0, s>>>(ud, nzd, L, slices, mean_opt);
+    return cudaGetLastError() == cudaSuccess ? MIXKV_OK : MIXKV_ERR_CUDA;
+  }
   unsigned char* wsb = reinterpret_cast<unsigned char*>(workspace);
   float* u = reinterpret_cast<float*>(wsb);
   wsb += align256((size_t)heads * T * kHeadDim * 4);
   int* nz = reinterpret_cast<int*>(wsb);
   wsb += align256((size_t)heads * T * 4);
-  cudaStream_t s = (cudaStream_t)stream;
   if (S == 1) {
     k_block_unit_sums<<<dim3((unsigned)T, (unsigned)heads), kSimThreads, 0, s>>>(
         reinterpret_cast<const __nv_bfloat16*>(X), L, block, 1, u, nz);

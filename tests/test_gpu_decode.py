@@ -56,6 +56,27 @@ def test_ragged_adaptive_cache():
     run(synth.with_budget(wl, 96, budget_mode=1), 2)
 
 
+@pytest.mark.parametrize("rows,G", [((4096, 1000, 4096, 37), 7), ((20000, 513), 4), ((256, 257), 16)])
+def test_long_rows_split_over_a_cluster(rows, G):
+    # heads with thousands of rows (a large budget, or a cache that was not compressed): the rows
+    # of a head are split over the CTAs of a cluster and walked in blocks of 256 with a running
+    # softmax; two layers, ragged heads, a sharp row so that the running reference moves
+    H, NL = len(rows), 2
+    rng = np.random.default_rng(sum(rows))
+    cap = int(sum(rows))
+    K = rng.standard_normal((NL, cap, 128)).astype(np.float32)
+    V = rng.standard_normal((NL, cap, 128)).astype(np.float32)
+    q = rng.standard_normal((NL, 1, H * G, 128)).astype(np.float32)
+    K[0, rows[0] - 3] = 6.0 * q[0, 0, 0]          # one key far above the rest, late in head 0
+    Kb, Vb, qb = (synth.f32_to_bf16_bits(a) for a in (K, V, q))
+    offs = np.tile(np.concatenate([[0], np.cumsum(rows)]).astype(np.int32), (NL, 1))
+    out = binding.decode_attention(bits_to_dev(Kb), bits_to_dev(Vb), torch.from_numpy(offs).cuda(),
+                                   bits_to_dev(qb), H, G, max_rows=max(rows)).cpu().numpy()
+    for l in range(NL):
+        ref = decode_plain.decode_attention(Kb[l], Vb[l], offs[l], qb[l], H, G)
+        assert np.allclose(out[l], ref, rtol=RTOL, atol=ATOL), f"layer {l}"
+
+
 def test_empty_head_short_rows_and_bad_arguments():
     H, G = 2, 2
     rng = np.random.default_rng(3)

@@ -31,6 +31,52 @@ def test_random_rows_with_shared_component(H, L, block):
     run(synth.f32_to_bf16_bits(X.astype(np.float32)), block)
 
 
+@pytest.mark.parametrize("H,L,block", [(2, 1000, 16), (1, 700, 4), (3, 300, 2), (2, 257, 1),
+                                       (1, 130, 8), (2, 2049, 16), (1, 128, 1), (2, 391, 4)])
+def test_dense_route_small_maps(H, L, block):
+    # block = 1, 2, 4, 8, 16 takes the tensor-core route: ragged last tile and last block, a zero
+    # row, diagonal cells without the i == j pairs
+    rng = np.random.default_rng(1000 * block + L)
+    X = rng.standard_normal((H, L, 128)) + 0.8 * rng.standard_normal((H, 1, 128))
+    X[0, 3] = 0.0
+    cells, _ = run(synth.f32_to_bf16_bits(X.astype(np.float32)), block)
+    c = cells.cpu().numpy()
+    # mirrored tiles are the same numbers; inside a diagonal tile (i, j) and (j, i) are summed in
+    # a different order
+    assert np.allclose(c, c.transpose(0, 2, 1), rtol=0, atol=1e-6)
+    if block == 1:
+        assert (np.diagonal(c, axis1=1, axis2=2) == 0).all()
+
+
+@pytest.mark.parametrize("L,block", [(8192, 1), (32768, 16)])
+def test_dense_route_full_size_sampled(L, block):
+    # The dense map of the keys of two heads at full size.  The pairwise oracle needs the L x L
+    # matrix in fp64, so it checks sampled 128-row tiles: a cell depends only on the rows of its
+    # two blocks, and the oracle run on the rows of tiles a and b gives the cells of (a, a),
+    # (a, b), (b, a), (b, b).  The whole map is checked for symmetry and range, its mean against
+    # Eq. 4 from the oracle's key geometry.
+    import oracle
+    wl = synth.replace(synth.CONFIGS["C3"], seq_lens=(L,), vision_tokens=(L - 256,),
+                       frame_tokens=(L - 256) // 32)
+    K = synth.make_layer(wl, 3, "calibrated")["K"][:2]
+    X = torch.from_numpy(K.view(np.int16)).cuda().view(torch.bfloat16)
+    cells, mean = binding.similarity_map(X, block)
+    torch.cuda.synchronize()
+    nT, per = L // 128, 128 // block
+    for h in range(2):
+        for a, b in ((0, 1), (5, nT - 1), (nT // 2, nT // 2 + 7), (nT - 2, nT - 1)):
+            rows = np.concatenate([np.arange(a * 128, a * 128 + 128), np.arange(b * 128, b * 128 + 128)])
+            ref, _ = similarity_plain.block_cosine_map(K[h:h + 1, rows], block)
+            ia, ib = slice(a * per, a * per + per), slice(b * per, b * per + per)
+            got = torch.cat([torch.cat([cells[h, ia, ia], cells[h, ia, ib]], 1),
+                             torch.cat([cells[h, ib, ia], cells[h, ib, ib]], 1)], 0).cpu().numpy()
+            assert np.allclose(got, ref[0], rtol=RTOL, atol=ATOL), (h, a, b)
+        assert torch.allclose(cells[h], cells[h].T, rtol=0, atol=1e-6)
+        assert float(cells[h].abs().max()) <= 1.0 + 1e-4
+    rbar = np.array([oracle.key_geometry(K[h])[1] for h in range(2)])
+    assert np.allclose(mean.cpu().numpy(), rbar, rtol=RTOL, atol=ATOL)
+
+
 def test_keys_and_values_of_a_c2_layer():
     wl = synth.CONFIGS["C2"]
     x = synth.make_layer(wl, 7, "calibrated")
