@@ -543,10 +543,103 @@ def run_e2e(args, wl, pg, cu_list, host, dev, world, barrier, binding):
                     "mixkv_compress_layers per group, compact cache -> pinned host"}
 
 
+def run_widened(args):
+    """Builder-run lines for the rows widened after the hot path (not the driver's metric):
+    --workload SIM     the dense redundancy-analysis map (block 16) of the keys of a C3 layer, a
+                       tensor-core contraction: roofline bound "tensor" against the measured bf16
+                       peak, algorithmic flops = 2 L^2 d per head;
+    --workload DECODE  one decode token over the C3b compact cache (28 layers x 4 heads x 512
+                       rows): bytes of cache read per second against the measured copy peak."""
+    import torch
+
+    from paper_2510_20707_b200 import binding, build, synth
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(0)
+    build.build()
+    binding.load_library()
+    with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+        pk = json.load(f)
+    stream = torch.cuda.current_stream()
+
+    def timed(fn, n):
+        for _ in range(max(3, args.warmup)):
+            fn()
+        torch.cuda.synchronize()
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0.record(stream)
+        for _ in range(n):
+            fn()
+        t1.record(stream)
+        torch.cuda.synchronize()
+        return t0.elapsed_time(t1) / n
+
+    if args.workload == "SIM":
+        wl = synth.CONFIGS["C3"]
+        H, L, block = wl.kv_heads, wl.total_tokens, 16
+        # keys of four layers in turn: 134 MB of input, larger than L2
+        Xs = [torch.from_numpy(synth.make_layer(wl, l, args.variant)["K"].view(np.int16)).cuda()
+              .view(torch.bfloat16) for l in range(4)]
+        it = [0]
+
+        def fn():
+            binding.similarity_map(Xs[it[0] % 4], block)
+            it[0] += 1
+
+        ms = timed(fn, max(4, min(args.steps, 20)))
+        flops = 2.0 * L * L * 128 * H
+        ach = flops / (ms * 1e-3) / 1e12
+        line = {"metric": "similarity_rows_per_s", "value": H * L / (ms * 1e-3), "unit": "rows/s",
+                "n_gpus": 1, "ms_per_step": ms, "higher_is_better": True, "dtype": "bf16 hi/lo in, f32 accumulate",
+                "data": "synthetic",
+                "config": {"workload": f"SIM: block-{block} cosine map of the keys of a C3 layer, "
+                                       f"H={H}, L={L}, d=128, {args.variant} keys; inputs of 4 layers cycled"},
+                "roofline": {"bound": "tensor", "achieved": ach, "peak": pk["bf16_tflops"],
+                             "unit": "TFLOP/s", "frac": ach / pk["bf16_tflops"], "traffic": None,
+                             "peak_source": "measured cuBLAS bf16 (burst)",
+                             "algorithmic_flops_per_launch": flops,
+                             "executed_flops_per_launch": flops * 1.5,
+                             "note": "executed = upper triangle (x 1/2) of three bf16 products "
+                                     "(hi.hi, hi.lo, lo.hi: x 3)"}}
+    else:
+        NL, H, G, B = 28, 4, 7, 512
+        rows = H * B
+        K = torch.randn((NL, rows, 128), device="cuda", dtype=torch.bfloat16)
+        V = torch.randn_like(K)
+        offs = (torch.arange(H + 1, dtype=torch.int32) * B).repeat(NL, 1).contiguous().cuda()
+        q = torch.randn((NL, 1, H * G, 128), device="cuda", dtype=torch.bfloat16)
+        big = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+
+        def fn():
+            big.zero_()          # flushes L2 between two reads of the 29 MB cache
+            binding.decode_attention(K, V, offs, q, H, G, B)
+
+        n = max(4, min(args.steps, 20))
+        ms_both = timed(fn, n)
+        ms_flush = timed(lambda: big.zero_(), n)
+        ms = ms_both - ms_flush
+        nbytes = 2.0 * NL * rows * 256
+        ach = nbytes / (ms * 1e-3) / 1e9
+        line = {"metric": "decode_tokens_per_s", "value": 1.0 / (ms * 1e-3), "unit": "tokens/s",
+                "n_gpus": 1, "ms_per_step": ms, "higher_is_better": True, "dtype": "bf16 in, f32 accumulate",
+                "data": "synthetic",
+                "config": {"workload": f"DECODE: one token over a compact cache of {NL} layers x {H} KV "
+                                       f"heads x {B} rows, G={G}, d=128; L2 flushed between calls "
+                                       f"(flush time {ms_flush * 1e3:.1f} us subtracted)"},
+                "roofline": {"bound": "hbm", "achieved": ach, "peak": pk["hbm_gbs"], "unit": "GB/s",
+                             "frac": ach / pk["hbm_gbs"], "traffic": None,
+                             "peak_source": "measured copy bandwidth",
+                             "algorithmic_bytes_per_launch": nbytes}}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload in ("SIM", "DECODE"):
+        run_widened(args)
     else:
         run_mixkv(args)
 
