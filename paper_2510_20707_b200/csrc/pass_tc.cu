@@ -395,7 +395,10 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(&bars->tfull[s], 1);
-      mbar_init(&bars->tempty[s], kEpiWarps);        // every epilogue warp reads every tile
+      // every epilogue warp that owns query rows reads every tile; warps on padding rows (the
+      // last lane quarters of the last block) neither wait nor arrive: a warp that polls a
+      // barrier takes issue slots from the scheduler it shares with the MMA issuer
+      mbar_init(&bars->tempty[s], (kEpiWarps / (MB * 4)) * ((NQ + 31) / 32));
     }
     mbar_init(&bars->qfull, 1);
     mbar_init(&bars->qfree, 1);
@@ -519,9 +522,9 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
       const int ts = it & 1, tph = (it >> 1) & 1;
       // (after an abort the waits fail at once; the loop goes on without work so that the
       // segment-end barriers below stay matched)
-      const bool ok = mbar_wait(&bars->tfull[ts], tph, abort);
-      tc_fence_after();
-      if (ok && warp_on) {
+      const bool ok = warp_on && mbar_wait(&bars->tfull[ts], tph, abort);
+      if (ok) {
+        tc_fence_after();
         const int k0 = ti.t * kTile + unit * NC;
         const bool need_mask = ti.t * kTile + kTile > P;
         const int lim = P + jrow;   // last key this row may see
@@ -549,9 +552,11 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
           }
         }
       }
-      tc_fence_before();
-      __syncwarp();   // one arrival per warp: 512 single arrivals on one word cost more than a chunk
-      if (lane == 0) mbar_arrive(&bars->tempty[ts]);
+      if (warp_on) {
+        tc_fence_before();
+        __syncwarp();   // one arrival per warp: 512 single arrivals on one word cost more than a chunk
+        if (lane == 0) mbar_arrive(&bars->tempty[ts]);
+      }
       if (seg_start) {   // (here: this was the segment's last tile)
         if (unit > 0) {
           if (segs_done > 0) named_bar_sync(8 + blk, kXThreads);   // the last hand-over was read
