@@ -430,6 +430,11 @@ def run_mixkv(args):
         "timing": {"blocks": len(blocks), "steps_per_block": args.steps,
                    "ms_per_step_median_block": ms_per_step, "ms_per_step_best_block": min(blocks),
                    "ms_per_step_first_block": blocks[0],
+                   # context only: the median block rescaled from the median sampled SM clock to the
+                   # maximum one (the HBM-bound share of a step does not follow the SM clock)
+                   "ms_per_step_scaled_to_max_sm_clock": (
+                       ms_per_step * clocks["sm_mhz"] / clocks["sm_max_mhz"]
+                       if clocks and clocks.get("sm_mhz") and clocks.get("sm_max_mhz") else None),
                    "regime": ("sustained: sw_power_cap seen during the timed blocks"
                               if clocks and "sw_power_cap" in clocks.get("reasons", [])
                               else "no throttle reason seen during the timed blocks")},
