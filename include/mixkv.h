@@ -14,10 +14,10 @@
  *    device memory and never synchronises the stream: every call only enqueues kernels
  *    on `stream` (a cudaStream_t passed as void*; NULL is the default stream).  Host
  *    state kept between calls is limited to per-device caches of attributes (SM count,
- *    shared-memory opt-in) and a process-wide call counter whose value tags the
- *    bookkeeping a call leaves in its workspace.  The workspace needs no initialisation
- *    and no clearing between calls, and may be reused for other shapes; two calls that
- *    may overlap in time need a workspace each.
+ *    compute capability, shared-memory opt-in).  The workspace needs no initialisation
+ *    and no clearing between calls (every word a kernel reads was written earlier in the
+ *    same call; nothing is counted across CTAs), and may be reused for other shapes; two
+ *    calls that may overlap in time need a workspace each.
  *  - Shapes.  H = kv_heads, G = gqa_ratio, d = head_dim (128), W = window.
  *      K, V      [H, Ltot, d] bf16, row-major.  Ltot = L for one sequence, else
  *                cu_seqlens_host[batch]; sequence b owns rows cu[b] .. cu[b+1]-1.

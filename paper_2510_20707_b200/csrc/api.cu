@@ -3,7 +3,6 @@
 #include <string.h>
 
 #include <atomic>
-#include <chrono>
 #include <mutex>
 
 #include "common.cuh"
@@ -33,29 +32,6 @@ int device_check(int* major_out) {
 namespace {
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
-
-// A new 48-bit tag for every call.  The arrival counters pass 1 keeps in the caller's workspace
-// carry it, so counts left by an earlier call (or memory never written) read as "not this call"
-// and the workspace needs no clearing.  Tags are 48 bits of a mixed 64-bit counter: random for
-// practical purposes, so a stale word matches a new call's tag with probability 2^-48.
-unsigned long long next_call_tag() {
-  static std::atomic<unsigned long long> state{0};
-  unsigned long long cur = state.load(std::memory_order_relaxed);
-  if (cur == 0) {
-    unsigned long long seed =
-        (unsigned long long)std::chrono::steady_clock::now().time_since_epoch().count();
-    seed ^= reinterpret_cast<uintptr_t>(&state) * 0x9e3779b97f4a7c15ull;
-    seed |= 1ull;
-    state.compare_exchange_strong(cur, seed, std::memory_order_relaxed);
-  }
-  const unsigned long long v =
-      state.fetch_add(0x9e3779b97f4a7c15ull, std::memory_order_relaxed);
-  unsigned long long z = v;   // splitmix64 finaliser: consecutive calls get unrelated tags
-  z = (z ^ (z >> 30)) * 0xbf58476d1ce4e5b9ull;
-  z = (z ^ (z >> 27)) * 0x94d049bb133111ebull;
-  z ^= z >> 31;
-  return z & 0xffffffffffffull;
-}
 
 int check_params(const mixkv_params* p) {
   if (!p) return MIXKV_ERR_INVALID_ARG;
@@ -152,9 +128,6 @@ void carve(const mixkv_params* p, const SeqTable& st, unsigned char* base, Works
   ws->dstat = (float4*)take(NL * st.nt2 * 2 * 16);
   ws->exsum = (float*)take(NL * H * st.pchunks_total * 4);
   ws->rbar = (float*)take(NL * BH * 4);
-  ws->bq = (float*)take(NL * BH * st.NQ * 4);
-  ws->kbar = (float*)take(NL * BH * kHeadDim * 4);
-  ws->headcnt = (unsigned long long*)take(NL * BH * 8);
   ws->counts = (int*)take(NL * BH * 4);
   ws->idx_offsets = (int*)take(NL * (BH + 1) * 4);
   ws->idx = (int*)take(NL * (size_t)idx_capacity(p, st) * 4);
@@ -187,7 +160,6 @@ int make_ctx(const mixkv_params* p, const int32_t* cu, int batch, int L, void* w
   c->p = *p;
   const float scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)kHeadDim);
   c->scale_log2e = scale * kLog2e;
-  c->call_tag = next_call_tag();
   c->max_seq_len = max_len;
   c->max_prefix = max_len - p->window;
   c->stream = (cudaStream_t)stream;
@@ -201,9 +173,9 @@ int make_ctx(const mixkv_params* p, const int32_t* cu, int batch, int L, void* w
 int enqueue_passes(const LaunchCtx& c, const void* K, const void* V, const void* Q, float* s_div,
                    float* rbar_out, int* status) {
   c.mark();
-  if (launch_pass1(c, K, Q, rbar_out, status) != cudaSuccess) return MIXKV_ERR_CUDA;
+  if (launch_pass1(c, K, Q, status) != cudaSuccess) return MIXKV_ERR_CUDA;
   c.mark();
-  if (launch_pass2(c, K, V, Q, s_div, status) != cudaSuccess) return MIXKV_ERR_CUDA;
+  if (launch_pass2(c, K, V, Q, s_div, rbar_out, status) != cudaSuccess) return MIXKV_ERR_CUDA;
   if (c.p.pool_mode == MIXKV_POOL_MAX) {
     c.mark();
     if (launch_poolsum(c) != cudaSuccess) return MIXKV_ERR_CUDA;

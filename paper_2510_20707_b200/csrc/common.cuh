@@ -57,11 +57,7 @@ struct Workspace {
   float4* vstat;      // [nt2]         (min, max, sum, -) of |V_i| over candidates
   float4* dstat;      // [nt2, 2]      per epilogue warpgroup: (min, max, sum) of s_div, window-count-weighted sum of s_ex_raw
   float* exsum;       // [H, pchunks_total]   per-chunk sum of pooled s_ex (max pooling only)
-  float* rbar;        // [batch*H]
-  // merged once per (sequence, head) by the pass-1 CTA that delivers its last segment
-  float* bq;          // [batch*H, NQ]  per window row: -(log2 of its softmax normaliser) - log2 W
-  float* kbar;        // [batch*H, d]   mean unit key
-  unsigned long long* headcnt;   // [batch*H]  (call tag << 16 | segments delivered)
+  float* rbar;        // [batch*H]   redundancy of Eq. 4, left by pass 2
   int* counts;        // [batch*H]
   int* idx_offsets;   // [batch*H + 1]
   int* idx;           // [batch*H*(B-W)]
@@ -77,7 +73,6 @@ struct LaunchCtx {
   int idx_cap;                 // selected rows one layer can produce (capacity of its index list)
   int out_rows_cap;            // output rows reserved per layer: batch * H * B
   float scale_log2e;   // softmax scale * log2(e)
-  unsigned long long call_tag;   // 48 bits, new for every call: marks this call's arrival counters
   int max_seq_len;
   int max_prefix;
   cudaStream_t stream;
@@ -94,10 +89,9 @@ struct LaunchCtx {
 };
 
 // ---- kernels (defined in the .cu files) ------------------------------------------
-cudaError_t launch_pass1(const LaunchCtx& c, const void* K, const void* Q, float* rbar_out,
-                         int* status);
+cudaError_t launch_pass1(const LaunchCtx& c, const void* K, const void* Q, int* status);
 cudaError_t launch_pass2(const LaunchCtx& c, const void* K, const void* V, const void* Q,
-                         float* s_div_out, int* status);
+                         float* s_div_out, float* rbar_out, int* status);
 int device_sm_count();
 // Fills a CUtensorMap (passed as void*) for a bf16 tensor of the given rank: dims innermost first,
 // strides in bytes of dimensions 1 .. rank-1, box extents; 128-byte swizzle, zero fill outside.

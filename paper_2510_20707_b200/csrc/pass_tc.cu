@@ -5,12 +5,15 @@
 //
 //   pass 1  K from HBM.  Logits with the window queries on the M side (one query row per TMEM
 //           lane), so the running softmax (max, sum) of a row is thread-local; alongside, key
-//           norms and the sum of unit keys from the shared-memory tile.
-//           The CTA that delivers the last segment of a (layer, sequence, head) folds all of
-//           its segments: the softmax statistics become one log2 normaliser per window row,
-//           the unit-key sums become the mean unit key and the redundancy of Eq. 4.
-//   pass 2  K again, V from HBM.  Logits with the keys on the M side (one key per TMEM lane),
-//           normalised with the finished row statistics, so the column sum over window rows
+//           norms and the sum of unit keys from the shared-memory tile.  Every run of tiles
+//           of one (layer, sequence, head) inside a CTA (a segment) leaves its partial
+//           statistics.
+//   pass 2  K again, V from HBM.  A CTA that starts on a (layer, sequence, head) first folds
+//           that head's segments of pass 1: the softmax statistics become one log2 normaliser
+//           per window row, the unit-key sums the mean unit key and the redundancy of Eq. 4
+//           (every CTA that touches the head does this for itself: no CTA waits for another,
+//           nothing is counted).  Logits with the keys on the M side (one key per TMEM lane),
+//           normalised with those row statistics, so the column sum over window rows
 //           and query heads is thread-local -> s_ex_raw.  The mean unit key rides
 //           along as three extra bf16 "query" rows -> K_i . kbar -> s_div.  Value norms are
 //           computed from V tiles staged next to the K tiles.
@@ -28,14 +31,11 @@ constexpr int kTileBytes = kTile * 256;    // 128 keys x 128 bf16
 constexpr int kHalfBytes = kTile * 128;    // one 64-column half of a K tile
 
 // Warp roles.  Warpgroup 0 (warps 0..3) holds the single-thread roles: TMA producer, MMA
-// issuer, (pass 2) V producer; warps 4..19 are the epilogue: two groups of eight warps, group g
-// owns accumulator stage g of tensor memory and therefore every other tile, so the exponentials
-// of two tiles are in flight on every scheduler at any time (the exp2 unit is what bounds both
-// passes, and eight warps cannot keep it busy: their chains are too short to cover its latency);
-// the warps from 20 on compute key statistics (pass 1) or value norms (pass 2).  A warp's TMEM
-// lane quarter is warp % 4.  Register budgets per role are set with setmaxnreg: the kernels are
-// launched with 72 / 80 registers per thread and the single-thread roles hand most of theirs to
-// the epilogue warps.
+// issuer, (pass 2) V producer.  Pass 1: warps 4..19 are the epilogue (all sixteen work on every
+// tile), warps 20..27 compute the key statistics; register budgets per role are set with
+// setmaxnreg (the single-thread roles hand most of theirs to the others).  Pass 2: warps 4..11
+// are the epilogue (two warpgroups that own alternate tiles), warps 12..15 the value norms.  A
+// warp's TMEM lane quarter is warp % 4.
 constexpr int kWarpTma = 0, kWarpMma = 1;
 constexpr int kP1WarpMma = 3;                    // pass 1: see k_pass1
 constexpr int kEpiWarp0 = 4;
@@ -49,33 +49,6 @@ template <int N, int BASE>
 __device__ __forceinline__ void set_regs() {
   if constexpr (N < BASE) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
   if constexpr (N > BASE) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
-}
-
-// Counts a delivered segment of a (layer, sequence, head) whose partial results come from
-// `nseg` CTAs; true in the CTA that delivers the last one.  Called by one thread after a CTA
-// barrier that follows the writes of the partial results: the release half of the atomic
-// publishes them, the acquire half lets the last arrival read everybody's.  The word holds
-// (tag << 16 | arrivals).  A word with another tag is left over from an earlier call, or was
-// never written, and the first arrival of this call replaces it: the caller's workspace needs
-// no clearing between calls.  Once the word carries the tag an arrival is one atomic add (no
-// retries when the CTAs of a head finish together).
-__device__ __forceinline__ bool arrive_last(unsigned long long* word, const unsigned long long tag,
-                                            const int nseg) {
-  unsigned long long cur = *reinterpret_cast<volatile unsigned long long*>(word);
-  for (;;) {
-    if ((cur >> 16) == tag) {
-      unsigned long long old;
-      asm volatile("atom.add.acq_rel.gpu.global.u64 %0, [%1], %2;"
-                   : "=l"(old)
-                   : "l"(word), "l"(1ull)
-                   : "memory");
-      return (int)((old + 1ull) & 0xffffull) == nseg;
-    }
-    __threadfence();   // release for the plain compare-and-swap below
-    const unsigned long long seen = atomicCAS(word, cur, (tag << 16) | 1ull);
-    if (seen == cur) return nseg == 1;
-    cur = seen;   // another CTA replaced the stale word first (or it changed): look again
-  }
 }
 
 __device__ __forceinline__ void raise(int* status, volatile int* abort) {
@@ -181,111 +154,61 @@ struct P1Bars {
   uint64_t qfree;
   uint32_t tmem_base;
   int abort;
-  int last;   // this CTA delivered the last segment of the head at hand
 };
 
-// ---- per-head folds at the end of pass 1 (once per (layer, sequence, head), in the CTA that
-// delivers the head's last segment)
-//
-// Softmax (reference, sum) pairs of window row q over the segments e = half, half + 2, ... of
-// the head: the caller's partner thread takes the other half.
-__device__ __forceinline__ float2 fold_row_stats(const float2* rowstat, const SegList& sl,
-                                                 const int NQ, const int q, const int half) {
-  float Mx = -1e30f, Zs = 0.f;
-#pragma unroll 1
-  for (int e0 = half; e0 < sl.nseg; e0 += 24) {   // twelve loads in flight
-    float2 v[12];
-#pragma unroll
-    for (int k = 0; k < 12; ++k) {
-      const int e = e0 + 2 * k;
-      v[k] = make_float2(-1e30f, 0.f);
-      if (e < sl.nseg) v[k] = __ldcg(rowstat + (size_t)sl.start(e) * NQ + q);
-    }
-#pragma unroll
-    for (int k = 0; k < 12; ++k) {
-      const float mn = fmaxf(Mx, v[k].x);
-      Zs = Zs * ex2(Mx - mn) + v[k].y * ex2(v[k].x - mn);
-      Mx = mn;
-    }
-  }
-  return make_float2(Mx, Zs);
-}
 // (m, z) pairs of the same row merged: z0 2^m0 + z1 2^m1 under the larger reference.
 __device__ __forceinline__ float2 merge_stats(const float2 a, const float2 b) {
   const float mn = fmaxf(a.x, b.x);
   return make_float2(mn, a.y * ex2(a.x - mn) + b.y * ex2(b.x - mn));
 }
-// Component kt of the unit-key sums over the segments e = half, half + 2, ... of the head.
-__device__ __forceinline__ float fold_key_sums(const float* ksum, const SegList& sl, const int kt,
-                                               const int half) {
+
+// ---- per-head folds (pass 2, at the start of a segment): what the segments of pass 1 left
+// for a (layer, sequence, head) becomes what pass 2 needs of it.
+//
+// kFoldDepth loads are in flight per round: a head that a one-layer call spreads over a quarter
+// of the GPU's CTAs is folded in one round trip to L2.
+constexpr int kFoldDepth = 40;
+// Window row q: the (reference, sum) pairs of all segments merged under the largest reference,
+// returned as the negated log2 normaliser of the row with the 1/W of the window mean folded in.
+__device__ __forceinline__ float fold_row_stats(const float2* rowstat, const SegList& sl,
+                                                const int NQ, const int q, const float log2W) {
+  float M = -1e30f, Z = 0.f;
+#pragma unroll 1
+  for (int e0 = 0; e0 < sl.nseg; e0 += kFoldDepth) {
+    float2 v[kFoldDepth];
+#pragma unroll
+    for (int k = 0; k < kFoldDepth; ++k) {
+      v[k] = make_float2(-1e30f, 0.f);
+      if (e0 + k < sl.nseg) v[k] = __ldcg(rowstat + (size_t)sl.start(e0 + k) * NQ + q);
+    }
+    float mx = M;
+#pragma unroll
+    for (int k = 0; k < kFoldDepth; ++k) mx = fmaxf(mx, v[k].x);
+    Z *= ex2(M - mx);
+#pragma unroll
+    for (int k = 0; k < kFoldDepth; ++k) Z = fmaf(v[k].y, ex2(v[k].x - mx), Z);
+    M = mx;
+  }
+  return -(M + log2f(Z)) - log2W;
+}
+// Component kt of the unit-key sum over all segments of the head.
+__device__ __forceinline__ float fold_key_sums(const float* ksum, const SegList& sl, const int kt) {
   float sum = 0.f;
 #pragma unroll 1
-  for (int e0 = half; e0 < sl.nseg; e0 += 24) {   // twelve loads in flight
-    float v[12];
+  for (int e0 = 0; e0 < sl.nseg; e0 += kFoldDepth) {
+    float v[kFoldDepth];
 #pragma unroll
-    for (int k = 0; k < 12; ++k)
-      v[k] = e0 + 2 * k < sl.nseg ? __ldcg(ksum + (size_t)sl.start(e0 + 2 * k) * kHeadDim + kt) : 0.f;
+    for (int k = 0; k < kFoldDepth; ++k)
+      v[k] = e0 + k < sl.nseg ? __ldcg(ksum + (size_t)sl.start(e0 + k) * kHeadDim + kt) : 0.f;
 #pragma unroll
-    for (int k = 0; k < 12; ++k) sum += v[k];
+    for (int k = 0; k < kFoldDepth; ++k) sum += v[k];
   }
   return sum;
 }
-constexpr int kFoldThreads = kEpiThreads + 256;   // the epilogue and the key-statistics warps
-// Walks the segments of the CTA's tile range [lo, hi); the epilogue threads (et = 0 .. 511, else
-// -1) and the key-statistics threads (at = 0 .. 255, else -1) call it after the barrier that
-// ends the tile loops.  Two epilogue threads per window row fold the row statistics, two
-// key-statistics threads per dimension the key sums.  `red` is shared scratch of eight floats,
-// `flag` a shared int.  Named barrier 5 joins the callers.
-__device__ __forceinline__ void finish_heads(const SeqTable& st, const Workspace& ws, const int lo,
-                                             const int hi, const unsigned long long call_tag,
-                                             float* __restrict__ rbar_out, float* red, int* flag,
-                                             const int et, const int at) {
-  const int NQ = st.NQ, H = st.H;
-  int id = lo;
-  while (id < hi) {
-    const TileIter ti(st.tile1_start, st.batch, H, st.nt1, id, hi);
-    const int per_head = (st.tile1_start[ti.b + 1] - st.tile1_start[ti.b]) / H;
-    const int L = st.cu[ti.b + 1] - st.cu[ti.b];
-    const int unit = ti.unit();
-    const SegList sl(ti.layer * st.nt1 + st.tile1_start[ti.b] + ti.h * per_head, per_head,
-                     split1(st));
-    if (et == 0) *flag = arrive_last(ws.headcnt + unit, call_tag, sl.nseg);
-    named_bar_sync(5, kFoldThreads);
-    const bool last = *flag != 0;
-    if (last) {
-      if (et >= 0 && et < 2 * NQ) {   // 2 NQ is a multiple of 32: whole warps, partners in adjacent lanes
-        float2 mz = fold_row_stats(ws.rowstat, sl, NQ, et >> 1, et & 1);
-        const float2 other = make_float2(__shfl_xor_sync(0xffffffffu, mz.x, 1),
-                                         __shfl_xor_sync(0xffffffffu, mz.y, 1));
-        mz = (et & 1) ? merge_stats(other, mz) : merge_stats(mz, other);
-        if ((et & 1) == 0)
-          ws.bq[(size_t)unit * NQ + (et >> 1)] = -(mz.x + log2f(mz.y)) - log2f((float)st.W);
-      }
-      if (at >= 0) {
-        const int kt = at >> 1;
-        float sum = fold_key_sums(ws.ksum, sl, kt, at & 1);
-        const float o = __shfl_xor_sync(0xffffffffu, sum, 1);
-        sum = (at & 1) ? o + sum : sum + o;
-        if ((at & 1) == 0) ws.kbar[(size_t)unit * kHeadDim + kt] = sum / (float)L;
-        const float n2 = warp_sum((at & 1) ? 0.f : sum * sum);
-        if ((at & 31) == 0) red[at >> 5] = n2;
-      }
-    }
-    named_bar_sync(5, kFoldThreads);   // `flag` may be rewritten; the eight partial norms are in `red`
-    if (last && at == 0) {
-      double nn = 0.0;
-      for (int w = 0; w < 8; ++w) nn += (double)red[w];
-      const double T = (double)L;
-      const float r = (float)((nn - T) / (T * (T - 1.0)));   // Eq. 4
-      ws.rbar[unit] = r;
-      if (rbar_out) rbar_out[unit] = r;
-      // every segment of this head has arrived: leave the counter at zero under this call's tag,
-      // so that a replay of the same launch (a captured graph keeps its tag) counts afresh
-      ws.headcnt[unit] = call_tag << 16;
-    }
-    named_bar_sync(5, kFoldThreads);   // `red` is free again
-    id += min(hi - id, per_head - ti.t);
-  }
+// The pass-1 segments of the head that tile iterator `ti` (of either pass) stands on.
+__device__ __forceinline__ SegList pass1_segments(const SeqTable& st, const TileIter& ti) {
+  const int per_head = (st.tile1_start[ti.b + 1] - st.tile1_start[ti.b]) / st.H;
+  return SegList(ti.layer * st.nt1 + st.tile1_start[ti.b] + ti.h * per_head, per_head, split1(st));
 }
 
 // The running softmax statistics of a query row are a pair (m, z): z = sum over the keys seen
@@ -356,7 +279,7 @@ template <int MB>
 __global__ void __launch_bounds__(p1_threads(MB), 1)
 k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmQ,
         const SeqTable st, const Workspace ws, const float scale_log2e,
-        const unsigned long long call_tag, float* __restrict__ rbar_out, int* status) {
+        int* status) {
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* base =
       reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
@@ -676,19 +599,8 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
   tc_fence_before();
   __syncthreads();
   if (warp == kP1WarpMma) tmem_dealloc(tmem, MB * 256);
-  if (bars->abort) {
-    if (tid == 0 && status) atomicExch(status, MIXKV_ERR_TIMEOUT);
-    return;
-  }
-  // Every partial result of this CTA is written.  Its segments now count as delivered; the CTA
-  // that delivers the last segment of a (layer, sequence, head) folds all of them, once, into
-  // what pass 2 reads: one log2 normaliser per window row (the 1/W of the window mean folded
-  // in), the mean unit key, the redundancy of Eq. 4.  The epilogue warps do it (they hold the
-  // registers).
-  if (warp >= kEpiWarp0)
-    finish_heads(st, ws, lo, hi, call_tag, rbar_out, sks, &bars->last,
-                 warp < kAuxWarp0 ? tid - kEpiWarp0 * 32 : -1,
-                 warp < kAuxWarp0 ? -1 : tid - kAuxWarp0 * 32);
+  if (tid == 0 && bars->abort && status) atomicExch(status, MIXKV_ERR_TIMEOUT);
+  // every partial result of this CTA's segments is written: pass 2 folds them per head
 }
 
 // ======================================================================== pass 2
@@ -701,15 +613,6 @@ constexpr int kP2Threads = 16 * 32;
 constexpr int kP2EpiWarps = 8;                   // warps 4..11
 constexpr int kP2AuxWarp0 = 12;                  // warps 12..15: value norms
 
-// Named barrier among n threads that also agrees on whether to stop: the leader samples the
-// CTA abort flag before the barrier and everybody reads that sample after it, so a group
-// never splits around a later barrier.
-__device__ __forceinline__ bool group_sync_stop(int id, int n, bool leader, volatile int* abort,
-                                                volatile int* slots, int it) {
-  if (leader) slots[it & 1] = *abort;
-  named_bar_sync(id, n);
-  return slots[it & 1] != 0;
-}
 constexpr int kP2KStages = 3;              // K tiles (32 KB each)
 constexpr int kP2VStagesMax = 4;           // V half tiles: 64 rows, 16 KB each
 constexpr int kVSubBytes = 64 * 256;
@@ -725,7 +628,6 @@ struct P2Bars {
   uint64_t kbready;
   uint32_t tmem_base;
   int abort;
-  int vote[3][2];
 };
 
 // N logit columns of one key (registers r[0..N)): adds exp2(logit * scale - normaliser of the
@@ -751,7 +653,7 @@ __device__ __forceinline__ void colsum_chunk(const uint32_t (&r)[N], const float
 __global__ void __launch_bounds__(kP2Threads, 1)
 k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
         const __grid_constant__ CUtensorMap tmQ, const SeqTable st, const Workspace ws,
-        float* __restrict__ s_div_out, const float scale_log2e,
+        float* __restrict__ s_div_out, float* __restrict__ rbar_out, const float scale_log2e,
         const int use_vnorm, const int pool_half, const int vstages, int* status) {
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* base =
@@ -761,8 +663,8 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
   unsigned char* sQ = base;                   // 2 halves x [NB x 128 B]
   unsigned char* sK = sQ + 2 * NB * 128;      // kP2KStages x 32 KB
   unsigned char* sV = sK + kP2KStages * kTileBytes;   // vstages x 16 KB
-  float* sbq = reinterpret_cast<float*>(sV + vstages * kVSubBytes);  // [2][256] negated normalisers
-  float* sred = sbq + 512;                    // [64]: 2 x 16 epilogue, 16 value norms + 4 mean key
+  float* sbq = reinterpret_cast<float*>(sV + vstages * kVSubBytes);  // [256] negated normalisers (+ 256 spare)
+  float* sred = sbq + 512;                    // [64]: 2 x 16 epilogue, 12 value norms, 4 mean key
   P2Bars* bars = reinterpret_cast<P2Bars*>(sred + 64);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -890,14 +792,18 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
     // ------------------------------------------------------------------ epilogue
     // The two warpgroups take alternate tiles (warpgroup g owns accumulator stage g), one key
     // per thread and all G*W columns of it, so a tile needs no exchange between warpgroups and
-    // the groups never wait for each other: each keeps its own copy of the normaliser table
-    // and leaves its own partial score statistics.
+    // inside a segment the groups never wait for each other; each leaves its own partial score
+    // statistics.  At the start of a segment the 256 threads fold the row statistics of the
+    // head together, one window row per thread, into the normaliser table both groups read.
+    // Nobody leaves the tile loop early: after an abort every wait fails at once, so the
+    // named barriers of the segment boundaries stay matched.
     const int quarter = warp & 3, wg = (warp - kEpiWarp0) >> 2;
     const int gt = (tid - kEpiWarp0 * 32) & 127;   // thread inside the warpgroup
     const int gw = gt >> 5;                        // warp inside the warpgroup
     const int key = quarter * 32 + lane;
     const int nch = NQ / 16;
-    float* mybq = sbq + wg * 256;
+    const int et = tid - kEpiWarp0 * 32;           // thread inside the epilogue, 0..255
+    const float log2W = log2f((float)W);
     const int barid = 1 + wg;                      // named barriers 1, 2: one per warpgroup
     const f32x2 sc2 = pack2(scale_log2e, scale_log2e);
     float dmin = INFINITY, dmax = -INFINITY, dsum = 0.f, exw = 0.f;
@@ -906,12 +812,11 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
     for (TileIter ti(st.tile2_start, st.batch, H, st.nt2, lo, hi); ti.valid(); ti.next()) {
       const int L = st.cu[ti.b + 1] - st.cu[ti.b], P = L - W;
       if (seg_start) {
-        // pass 1 left one negated log2 normaliser per window row of this (layer, b, h)
-        named_bar_sync(barid, 128);   // the previous segment's readers of mybq are done
-        for (int q = gt; q < NQ; q += 128) mybq[q] = ws.bq[(size_t)ti.unit() * NQ + q];
+        named_bar_sync(5, kP2EpiWarps * 32);   // the previous segment's readers of sbq are done
+        if (et < NQ) sbq[et] = fold_row_stats(ws.rowstat, pass1_segments(st, ti), NQ, et, log2W);
         dmin = INFINITY, dmax = -INFINITY, dsum = 0.f, exw = 0.f;
         seg_first = ti.id;
-        named_bar_sync(barid, 128);
+        named_bar_sync(5, kP2EpiWarps * 32);
       }
       seg_start = ti.seg_last();
       const int ts = it & 1;
@@ -937,14 +842,14 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
             tmem_ld32(taddr + ci * 32, ra);
             tmem_ld_wait();
             tmem_ld_fence(ra);
-            colsum_chunk<32>(ra, mybq + ci * 32, sc2, acc);
+            colsum_chunk<32>(ra, sbq + ci * 32, sc2, acc);
           }
           if (nch & 1) {
             uint32_t rb[16];
             tmem_ld16(taddr + n32 * 32, rb);
             tmem_ld_wait();
             tmem_ld_fence(rb);
-            colsum_chunk<16>(rb, mybq + n32 * 32, sc2, acc);
+            colsum_chunk<16>(rb, sbq + n32 * 32, sc2, acc);
           }
           tmem_ld_wait();
           tmem_ld_fence(rd);
@@ -968,7 +873,6 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
           exw = fmaf(ex, (float)cover, exw);
         }
       }
-      if (group_sync_stop(barid, 128, gt == 0, abort, bars->vote[wg], it)) break;
       if (seg_start) {
         // this warpgroup's share of the segment's score statistics (neutral if it had no tile)
         const float a = warp_min(dmin), b2 = warp_max(dmax), c2 = warp_sum(dsum),
@@ -992,8 +896,10 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
     }
   } else if (warp >= kP2AuxWarp0) {
     // ------------------------------------------------------------------ mean key, value norms
-    // At the start of a segment: write the bf16 hi / lo / lo2 split of the head's mean unit key
-    // (pass 1) into the three extra B rows.  Per tile: warps 12, 13 read the first 64 rows of the V
+    // At the start of a segment: fold the unit-key sums of the head's pass-1 segments (one
+    // dimension per thread) and write the bf16 hi / lo / lo2 split of the mean unit key into the
+    // three extra B rows; the CTA that starts on the head's first tile also leaves the redundancy
+    // of Eq. 4, which needs nothing but the squared norm of that sum.  Per tile: warps 12, 13 read the first 64 rows of the V
     // tile, warps 14, 15 the last 64; one row per thread from the swizzled half tile.
     const int vt = tid - kP2AuxWarp0 * 32;         // 0..127
     const int sub = vt >> 6, vr = vt & 63;
@@ -1002,7 +908,21 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
     bool seg_start = true;
     for (TileIter ti(st.tile2_start, st.batch, H, st.nt2, lo, hi); ti.valid(); ti.next()) {
       if (seg_start) {
-        const float kb = ws.kbar[(size_t)ti.unit() * kHeadDim + vt];   // mean unit key (pass 1)
+        const int L = st.cu[ti.b + 1] - st.cu[ti.b];
+        const float ks = fold_key_sums(ws.ksum, pass1_segments(st, ti), vt);
+        const float kb = ks / (float)L;   // mean unit key
+        if (ti.t == 0) {                  // the same in all 128 threads
+          const float n2 = warp_sum(ks * ks);
+          if (lane == 0) sred[44 + (warp - kP2AuxWarp0)] = n2;
+          named_bar_sync(4, 128);
+          if (vt == 0) {
+            const double nn = ((double)sred[44] + (double)sred[45]) + ((double)sred[46] + (double)sred[47]);
+            const double T = (double)L;
+            const float r = (float)((nn - T) / (T * (T - 1.0)));   // Eq. 4
+            ws.rbar[ti.unit()] = r;
+            if (rbar_out) rbar_out[ti.unit()] = r;
+          }
+        }
         __nv_bfloat16 parts[3];
         parts[0] = __float2bfloat16_rn(kb);
         const float r1 = kb - __bfloat162float(parts[0]);
@@ -1081,7 +1001,6 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
           vsum += n;
         }
       }
-      if (group_sync_stop(3, 128, vt == 0, abort, bars->vote[2], it)) break;
       if (seg_start && use_vnorm) {
         const float a = warp_min(vmin), b2 = warp_max(vmax), c2 = warp_sum(vsum);
         const int vw = warp - kP2AuxWarp0;
@@ -1211,8 +1130,7 @@ int device_sm_count() {
   return cached[dev];
 }
 
-cudaError_t launch_pass1(const LaunchCtx& c, const void* K, const void* Q, float* rbar_out,
-                         int* status) {
+cudaError_t launch_pass1(const LaunchCtx& c, const void* K, const void* Q, int* status) {
   CUtensorMap tmK, tmQ;
   if (!map_kv(c, K, kTile, &tmK) || !map_q(c, Q, &tmQ)) return cudaErrorInvalidValue;
   static bool done1[64] = {false}, done2[64] = {false};
@@ -1221,17 +1139,17 @@ cudaError_t launch_pass1(const LaunchCtx& c, const void* K, const void* Q, float
     cudaError_t e = ensure_smem(k_pass1<1>, kSmemLimit, done1);
     if (e != cudaSuccess) return e;
     return launch_pdl(k_pass1<1>, dim3(c.st.g1), dim3(p1_threads(1)), smem, c.stream, 1, tmK, tmQ, c.st,
-                      c.ws, c.scale_log2e, c.call_tag, rbar_out, status);
+                      c.ws, c.scale_log2e, status);
   }
   const size_t smem = pass1_smem(2, c.st.NQ);
   cudaError_t e = ensure_smem(k_pass1<2>, kSmemLimit, done2);
   if (e != cudaSuccess) return e;
   return launch_pdl(k_pass1<2>, dim3(c.st.g1), dim3(p1_threads(2)), smem, c.stream, 1, tmK, tmQ, c.st,
-                    c.ws, c.scale_log2e, c.call_tag, rbar_out, status);
+                    c.ws, c.scale_log2e, status);
 }
 
 cudaError_t launch_pass2(const LaunchCtx& c, const void* K, const void* V, const void* Q,
-                         float* s_div_out, int* status) {
+                         float* s_div_out, float* rbar_out, int* status) {
   CUtensorMap tmK, tmV, tmQ;
   const void* Vsrc = c.p.use_vnorm == MIXKV_INTRINSIC_VNORM ? V : K;   // the V map is never used without VNorm
   if (!map_kv(c, K, kTile, &tmK) || !map_kv(c, Vsrc, 64, &tmV) || !map_q(c, Q, &tmQ))
@@ -1243,7 +1161,7 @@ cudaError_t launch_pass2(const LaunchCtx& c, const void* K, const void* V, const
   while (vstages > 2 && pass2_smem(c.st.NQ, vstages) > kSmemLimit) --vstages;
   const size_t smem = pass2_smem(c.st.NQ, vstages);
   return launch_pdl(k_pass2, dim3(c.st.g2), dim3(kP2Threads), smem, c.stream, 1, tmK, tmV, tmQ, c.st,
-                    c.ws, s_div_out, c.scale_log2e, c.p.use_vnorm, c.p.pool_kernel >> 1,
+                    c.ws, s_div_out, rbar_out, c.scale_log2e, c.p.use_vnorm, c.p.pool_kernel >> 1,
                     vstages, status);
 }
 
