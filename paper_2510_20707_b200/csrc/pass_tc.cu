@@ -1001,6 +1001,11 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
           vsum += n;
         }
       }
+      // The four warps stay within one tile of each other.  With an odd number of V stages the
+      // two pairs of warps take turns on the same stage: a pair that ran ahead would wait for
+      // a phase of vfull whose predecessor it never saw complete, and a parity wait on a
+      // barrier that is still one phase behind returns at once.
+      named_bar_sync(3, 128);
       if (seg_start && use_vnorm) {
         const float a = warp_min(vmin), b2 = warp_max(vmax), c2 = warp_sum(vsum);
         const int vw = warp - kP2AuxWarp0;

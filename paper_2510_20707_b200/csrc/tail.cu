@@ -248,6 +248,39 @@ __device__ __forceinline__ void count_digits(int* hist, const unsigned digit, co
   if (((left >> lane) & 1u) && digit != 0xffffffffu) atomicAdd(&hist[digit], 1);
 }
 
+// Adds eight digits per lane (0xffffffff = none) to a shared-memory histogram.  A lane first counts
+// how many of its own digits equal its first live one (the leading digits of a selection put
+// almost every key of a CTA into two or three bins: one add per key on those words would
+// serialise the CTA).  Then, as in count_digits, the first digit of the lowest lane and that of
+// the lowest lane left are added with one vote, one warp sum and one add each; the lanes left
+// after that add their own count, and the digits that differ from a lane's first go in one by
+// one.
+__device__ __forceinline__ void count_digits8(int* hist, const unsigned (&dg)[8], const int lane) {
+  unsigned d0 = 0xffffffffu;
+#pragma unroll
+  for (int e = 0; e < 8; ++e)
+    if (d0 == 0xffffffffu) d0 = dg[e];
+  int c0 = 0;
+#pragma unroll
+  for (int e = 0; e < 8; ++e) c0 += (dg[e] == d0);
+  unsigned left = 0xffffffffu;
+#pragma unroll
+  for (int round = 0; round < 2; ++round) {
+    const int src = __ffs(left) - 1;                       // lowest lane not counted yet
+    const unsigned d = __shfl_sync(0xffffffffu, d0, src);
+    const bool mine = d0 == d && ((left >> lane) & 1u);
+    const unsigned same = __ballot_sync(0xffffffffu, mine);
+    const int tot = __reduce_add_sync(0xffffffffu, mine ? c0 : 0);
+    if (lane == src && d != 0xffffffffu) atomicAdd(&hist[d], tot);
+    left &= ~same;
+    if (left == 0) break;                                  // uniform across the warp
+  }
+  if (((left >> lane) & 1u) && d0 != 0xffffffffu) atomicAdd(&hist[d0], c0);
+#pragma unroll
+  for (int e = 0; e < 8; ++e)
+    if (dg[e] != 0xffffffffu && dg[e] != d0) atomicAdd(&hist[dg[e]], 1);
+}
+
 // Threshold of the `want` largest keys of a set spread over the CTAs of a cluster (one CTA: a
 // cluster of one): the want-th largest key and how many keys equal to it are still needed.  All
 // threads of all CTAs take part; key_at(e), e < total, gives the keys of this CTA (any order).
@@ -694,9 +727,13 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
         for (int e = 0; e < 8; ++e)
           dg[e] = (e * T + tid < n && (rk[e] & mask) == prefix) ? (rk[e] >> shift) & 255u
                                                                 : 0xffffffffu;
+        if (R > 4) {   // R is the same in every thread
+          count_digits8(hist[buf], dg, lane);
+        } else {
 #pragma unroll
-        for (int e = 0; e < 8; ++e)
-          if (e < R) count_digit(dg[e], buf);   // R is the same in every thread
+          for (int e = 0; e < 4; ++e)
+            if (e < R) count_digit(dg[e], buf);
+        }
       } else {
         for (int e = 0; e < R; ++e) {   // same trip count in every lane: full-warp votes
           const int j = e * T + tid;

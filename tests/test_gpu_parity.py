@@ -266,10 +266,35 @@ def test_many_units_long_prefix_and_widest_query_tile():
     run_layers_parity(wl, range(40), check=(0, 17, 39))
 
 
+def test_repeated_calls_are_bit_identical_widest_query_tile():
+    # G*W = 240 leaves pass 2 room for three V stages only, which the two pairs of value-norm
+    # warps then share in turn (with four, each pair has its own): the same call thirty times
+    # over must give the same bits every time, value norms included (they reach s_comp through
+    # the intrinsic term).  A warp that read a V stage before its copy had landed would show
+    # here.
+    wl = synth.small_workload(H=2, G=15, W=16, seq_lens=(45016,), pool_kernel=5, budget=300,
+                              seed=33, centroids=16)
+    wl = synth.replace(wl, layers=6)
+    _, pg = params_pair(wl)
+    xs = [synth.make_layer(wl, l, "calibrated") for l in range(6)]
+    K, V, Q = (torch.stack([to_dev(x[k]) for x in xs]) for k in ("K", "V", "Q"))
+    first = None
+    for _ in range(30):
+        out = binding.compress_layers(K, V, Q, pg)
+        torch.cuda.synchronize()
+        assert int(out["status"].item()) == 0
+        if first is None:
+            first = out
+            continue
+        for key in ("s_comp", "idx", "idx_offsets", "out_row_offsets"):
+            assert torch.equal(first[key], out[key]), key
+        assert torch.equal(first["V_out"].view(torch.int16), out["V_out"].view(torch.int16))
+
+
 def test_workspace_needs_no_clearing():
-    # Pass 1 counts delivered segments in the caller's workspace under a per-call tag: whatever
-    # the workspace holds (all ones, all zeros, random bytes, the counters of an earlier call
-    # on another shape) the results are bit-identical.
+    # Every word of the workspace that a kernel reads was written earlier in the same call:
+    # whatever the workspace holds (all ones, all zeros, random bytes, what an earlier call on
+    # another shape left) the results are bit-identical.
     wl = synth.small_workload(H=3, G=4, W=16, seq_lens=(3000, 1500), pool_kernel=5, budget=96,
                               seed=41, centroids=8)
     x = synth.make_layer(wl, 0, "calibrated")
@@ -311,10 +336,9 @@ def test_workspace_needs_no_clearing():
 
 
 def test_graph_capture_and_replay():
-    # A call recorded into a CUDA graph keeps its host-side call tag, so every replay meets the
-    # arrival counters of the run before it in the workspace: the last arrival of a head leaves
-    # its counter at zero under the tag, and a replay counts afresh.  Two replays on new K / V /
-    # Q (copied into the captured buffers) must each match the oracle.
+    # A call recorded into a CUDA graph meets, at every replay, the workspace as the run before
+    # left it; nothing in it is counted or carried over.  Two replays on new K / V / Q (copied
+    # into the captured buffers) must each match the oracle.
     wl = synth.small_workload(H=3, G=4, W=16, seq_lens=(2600, 900), pool_kernel=5, budget=80,
                               seed=71, centroids=8)
     po, pg = params_pair(wl)
