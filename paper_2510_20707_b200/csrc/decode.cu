@@ -1,12 +1,15 @@
 // The step after compression: one new query token per sequence attends over the compact cache
 // (paper Sec. 3.1, Eq. 1: generation continues on the compressed K, V).  All layers of a model go
 // in one launch.  The rows of a (layer, sequence, KV head) unit are split over the CTAs of a
-// thread-block cluster (1, 2, 4 or 8: the fewest CTAs that fill the GPU once); a CTA walks its rows in blocks of 128 with a running softmax (reference, sum,
-// weighted value sum per query head of the group).  Per block: the V rows start towards shared
-// memory as one bulk copy, two threads per K row load its 256 bytes straight into registers (all
-// loads in flight at once) and leave the G logits, the softmax weights are formed while the V
-// copy lands, sixteen threads per V row add the weighted rows.  The cluster's partial results
-// are merged through distributed shared memory by its first CTA.  Every row is read once.
+// thread-block cluster (1, 2, 4 or 8: the fewest CTAs that fill the GPU once); a CTA walks its
+// rows in blocks of 128 with a running softmax (reference, sum, weighted value sum per query head
+// of the group).  The loads run ahead of the arithmetic: the V rows of two blocks are on their
+// way to shared memory (bulk copies into a two-stage ring) and the K rows of the next block are
+// on their way to registers (two threads per row, all eight 16-byte loads of a thread in flight)
+// while a block is worked on: logits from the registers, softmax weights, then sixteen threads
+// per V row add the weighted rows of all query heads in one sweep (packed fp32 pairs).  The
+// cluster's partial results are merged through distributed shared memory, every CTA taking a
+// slice of the outputs.  Every row is read once.
 #include <cooperative_groups.h>
 
 #include "tc_common.cuh"
@@ -19,12 +22,14 @@ namespace {
 constexpr int kDecThreads = 256;
 constexpr int kDecMaxG = 16;
 constexpr int kDecBlock = 128;   // rows per block: two threads per logit row
+constexpr int kDecSweep = 8;     // query heads whose value sums a thread holds at once
 
-// Floats of dynamic shared memory in front of the V block: sq [G][128] queries, sp [G][128]
+// Floats of dynamic shared memory in front of the V ring: sq [G][128] queries, sp [G][128]
 // logits then weights, part [8][G][128] per-warp value sums, xo [G][128] running weighted value
-// sum, xm / xz / sscale [16] each.
+// sum, xm / xz / sscale [16] each, then the merge's copy of every rank's xm and xz [2][8][16].
 __host__ __device__ constexpr size_t dec_floats(int G) {
-  return (size_t)G * (kHeadDim + kDecBlock + 8 * kHeadDim + kHeadDim) + 3 * kDecMaxG;
+  return (size_t)G * (kHeadDim + kDecBlock + 8 * kHeadDim + kHeadDim) + 3 * kDecMaxG +
+         2 * 8 * kDecMaxG;
 }
 
 __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
@@ -33,6 +38,26 @@ __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t b
           smem_u32(dst)),
       "l"(src), "r"(bytes), "r"(smem_u32(bar))
       : "memory");
+}
+
+// Packed fp32 pairs: one instruction for two lanes of arithmetic.
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float a, float b) {
+  f32x2 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float& a, float& b) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+  f32x2 d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+// The two bf16 of a 32-bit word as an fp32 pair (low half first).
+__device__ __forceinline__ f32x2 bf16x2_to_f32x2(uint32_t w) {
+  return pack2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
 }
 
 // grid: n_layers * batch * H * S, clusters of S.
@@ -49,8 +74,10 @@ k_decode_attention(const __nv_bfloat16* __restrict__ Kc, const __nv_bfloat16* __
   float* xm = xo + G * kHeadDim;                // [16]
   float* xz = xm + kDecMaxG;                    // [16]
   float* sscale = xz + kDecMaxG;                // [16] rescale of the running sums for this block
-  unsigned char* sV = reinterpret_cast<unsigned char*>(dsm + dec_floats(G));   // [128][256 B]
-  __shared__ __align__(8) uint64_t vbar;
+  float* allm = sscale + kDecMaxG;              // [8][16] merge: every rank's xm
+  float* allz = allm + 8 * kDecMaxG;            // [8][16] merge: every rank's xz
+  unsigned char* sV = reinterpret_cast<unsigned char*>(dsm + dec_floats(G));   // [2][128][256 B]
+  __shared__ __align__(8) uint64_t vbar[2];
   __shared__ int vabort;
   cg::cluster_group cluster = cg::this_cluster();
   const int S = (int)cluster.num_blocks(), crank = (int)cluster.block_rank();
@@ -58,7 +85,8 @@ k_decode_attention(const __nv_bfloat16* __restrict__ Kc, const __nv_bfloat16* __
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   pdl_launch_dependents();
   if (tid == 0) {
-    mbar_init(&vbar, 1);
+    mbar_init(&vbar[0], 1);
+    mbar_init(&vbar[1], 1);
     vabort = 0;
     mbar_init_fence();
   }
@@ -67,9 +95,32 @@ k_decode_attention(const __nv_bfloat16* __restrict__ Kc, const __nv_bfloat16* __
   const int r0 = ro[bh], n_unit = min(ro[bh + 1] - r0, max_rows);
   const int chunk = (n_unit + S - 1) / S;
   const int c0 = min(crank * chunk, n_unit), n = min(chunk, n_unit - c0);   // this CTA's rows
+  const int nblk = (n + kDecBlock - 1) / kDecBlock;
   const __nv_bfloat16* Kb = Kc + ((size_t)layer * rows_cap + r0 + c0) * kHeadDim;
   const __nv_bfloat16* Vb = Vc + ((size_t)layer * rows_cap + r0 + c0) * kHeadDim;
   const size_t qoff = (((size_t)layer * (BH / H) + b) * H + h) * (size_t)G * kHeadDim;
+  __syncthreads();   // the barriers are initialised
+  // ---- the V rows of the first two blocks start towards the ring
+  if (tid == 0) {
+    for (int k = 0; k < 2 && k < nblk; ++k) {
+      const uint32_t bytes = (uint32_t)min(kDecBlock, n - k * kDecBlock) * 256u;
+      mbar_expect_tx(&vbar[k], bytes);
+      bulk_load(sV + (size_t)k * kDecBlock * 256, Vb + (size_t)k * kDecBlock * kHeadDim, bytes, &vbar[k]);
+    }
+  }
+  // ---- the K rows of the first block start towards registers: row tid / 2, dimensions
+  // 64 * (tid & 1) .. + 63
+  const int row = tid >> 1, hf = tid & 1;
+  uint4 kv[8];
+  auto load_k = [&](const int blk) {
+    const int rr = blk * kDecBlock + row;
+    if (rr < n) {
+      const uint4* krow = reinterpret_cast<const uint4*>(Kb + (size_t)rr * kHeadDim + hf * 64);
+#pragma unroll
+      for (int c = 0; c < 8; ++c) kv[c] = __ldg(krow + c);
+    }
+  };
+  if (nblk > 0) load_k(0);
   for (int e = tid; e < G * kHeadDim; e += kDecThreads) {
     sq[e] = __bfloat162float(q[qoff + e]);
     xo[e] = 0.f;
@@ -77,48 +128,41 @@ k_decode_attention(const __nv_bfloat16* __restrict__ Kc, const __nv_bfloat16* __
   if (tid < kDecMaxG) xm[tid] = -INFINITY, xz[tid] = 0.f;
   __syncthreads();
 
-  int nblk = 0;
-  for (int blk0 = 0; blk0 < n; blk0 += kDecBlock, ++nblk) {
-    const int nb = min(kDecBlock, n - blk0);
-    // ---- the block's V rows start towards shared memory (the previous block's readers are done)
-    if (tid == 0) {
-      mbar_expect_tx(&vbar, (uint32_t)nb * 256u);
-      bulk_load(sV, Vb + (size_t)blk0 * kHeadDim, (uint32_t)nb * 256u, &vbar);
-    }
-    // ---- logits (log2 units): two threads per row, 64 dimensions each, all eight loads in flight
+  for (int blk = 0; blk < nblk; ++blk) {
+    const int nb = min(kDecBlock, n - blk * kDecBlock);
+    const int st = blk & 1;
+    // ---- logits (log2 units) from the K registers
     {
-      const int row = tid >> 1, hf = tid & 1;
-      float d[kDecMaxG];
+      f32x2 d[kDecMaxG];
 #pragma unroll
-      for (int g = 0; g < kDecMaxG; ++g) d[g] = 0.f;
+      for (int g = 0; g < kDecMaxG; ++g) d[g] = pack2(0.f, 0.f);
       if (row < nb) {
-        const uint4* krow = reinterpret_cast<const uint4*>(Kb + (size_t)(blk0 + row) * kHeadDim + hf * 64);
-        uint4 kv[8];
-#pragma unroll
-        for (int c = 0; c < 8; ++c) kv[c] = krow[c];
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
-          const float2 k0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&kv[c].x));
-          const float2 k1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&kv[c].y));
-          const float2 k2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&kv[c].z));
-          const float2 k3 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&kv[c].w));
+          const f32x2 k0 = bf16x2_to_f32x2(kv[c].x), k1 = bf16x2_to_f32x2(kv[c].y);
+          const f32x2 k2 = bf16x2_to_f32x2(kv[c].z), k3 = bf16x2_to_f32x2(kv[c].w);
 #pragma unroll
           for (int g = 0; g < kDecMaxG; ++g) {
             if (g < G) {
-              const float* qg = sq + g * kHeadDim + hf * 64 + 8 * c;
-              const float4 qa = *reinterpret_cast<const float4*>(qg);
-              const float4 qb = *reinterpret_cast<const float4*>(qg + 4);
-              d[g] = fmaf(k0.x, qa.x, fmaf(k0.y, qa.y, fmaf(k1.x, qa.z, fmaf(k1.y, qa.w, d[g]))));
-              d[g] = fmaf(k2.x, qb.x, fmaf(k2.y, qb.y, fmaf(k3.x, qb.z, fmaf(k3.y, qb.w, d[g]))));
+              const ulonglong2* qg =
+                  reinterpret_cast<const ulonglong2*>(sq + g * kHeadDim + hf * 64 + 8 * c);
+              const ulonglong2 qa = qg[0], qb = qg[1];
+              d[g] = fma2(k0, qa.x, fma2(k1, qa.y, d[g]));
+              d[g] = fma2(k2, qb.x, fma2(k3, qb.y, d[g]));
             }
           }
         }
       }
+      // the next block's K rows start towards the registers just read
+      if (blk + 1 < nblk) load_k(blk + 1);
 #pragma unroll
       for (int g = 0; g < kDecMaxG; ++g) {
         if (g < G) {
-          const float o = __shfl_xor_sync(0xffffffffu, d[g], 1);
-          const float t = hf ? o + d[g] : d[g] + o;   // first half + second half in both threads
+          float d0, d1;
+          unpack2(d[g], d0, d1);
+          const float mine = d0 + d1;
+          const float o = __shfl_xor_sync(0xffffffffu, mine, 1);
+          const float t = hf ? o + mine : mine + o;   // first half + second half in both threads
           if (hf == 0 && row < nb) sp[g * kDecBlock + row] = t * scale_log2e;
         }
       }
@@ -126,15 +170,15 @@ k_decode_attention(const __nv_bfloat16* __restrict__ Kc, const __nv_bfloat16* __
     __syncthreads();
     // ---- running softmax per query head: warp w takes heads w, w + 8, ...
     for (int g = warp; g < G; g += kDecThreads / 32) {
-      float* row = sp + g * kDecBlock;
+      float* prow = sp + g * kDecBlock;
       float mx = -INFINITY;
-      for (int r = lane; r < nb; r += 32) mx = fmaxf(mx, row[r]);
+      for (int r = lane; r < nb; r += 32) mx = fmaxf(mx, prow[r]);
       mx = warp_max(mx);
       const float m_old = xm[g], m_new = fmaxf(m_old, mx);
       float sum = 0.f;
       for (int r = lane; r < nb; r += 32) {
-        const float e = exp2f(row[r] - m_new);
-        row[r] = e;
+        const float e = exp2f(prow[r] - m_new);
+        prow[r] = e;
         sum += e;
       }
       sum = warp_sum(sum);
@@ -145,47 +189,58 @@ k_decode_attention(const __nv_bfloat16* __restrict__ Kc, const __nv_bfloat16* __
         xm[g] = m_new;
       }
     }
-    const bool vok = mbar_wait(&vbar, nblk & 1, &vabort);
+    const bool vok = mbar_wait(&vbar[st], (blk >> 1) & 1, &vabort);
     __syncthreads();
     // ---- weighted sum of the value rows from shared memory: sixteen threads per row (16 bytes
-    // each), sixteen rows per sweep, four query heads at a time
+    // each), sixteen rows per sweep over the block, up to eight query heads at a time
+    const unsigned char* vblk = sV + (size_t)st * kDecBlock * 256;
     const int c8 = tid & 15, rg = tid >> 4;
-    for (int g0 = 0; g0 < G; g0 += 4) {
-      float acc[4][8];
+    for (int g0 = 0; g0 < G; g0 += kDecSweep) {
+      f32x2 acc[kDecSweep][4];
 #pragma unroll
-      for (int k = 0; k < 4; ++k)
+      for (int k = 0; k < kDecSweep; ++k)
 #pragma unroll
-        for (int e = 0; e < 8; ++e) acc[k][e] = 0.f;
+        for (int e = 0; e < 4; ++e) acc[k][e] = pack2(0.f, 0.f);
       if (vok) {
 #pragma unroll 2
         for (int r = rg; r < nb; r += 16) {
-          const uint4 vv = *reinterpret_cast<const uint4*>(sV + (size_t)r * 256 + 16 * c8);
-          float v[8];
-          const float2 v0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&vv.x));
-          const float2 v1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&vv.y));
-          const float2 v2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&vv.z));
-          const float2 v3 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&vv.w));
-          v[0] = v0.x, v[1] = v0.y, v[2] = v1.x, v[3] = v1.y, v[4] = v2.x, v[5] = v2.y, v[6] = v3.x, v[7] = v3.y;
+          const uint4 vv = *reinterpret_cast<const uint4*>(vblk + (size_t)r * 256 + 16 * c8);
+          const f32x2 v0 = bf16x2_to_f32x2(vv.x), v1 = bf16x2_to_f32x2(vv.y);
+          const f32x2 v2 = bf16x2_to_f32x2(vv.z), v3 = bf16x2_to_f32x2(vv.w);
 #pragma unroll
-          for (int k = 0; k < 4; ++k) {
+          for (int k = 0; k < kDecSweep; ++k) {
             if (g0 + k < G) {
               const float wgt = sp[(g0 + k) * kDecBlock + r];
-#pragma unroll
-              for (int e = 0; e < 8; ++e) acc[k][e] = fmaf(wgt, v[e], acc[k][e]);
+              const f32x2 w2 = pack2(wgt, wgt);
+              acc[k][0] = fma2(w2, v0, acc[k][0]);
+              acc[k][1] = fma2(w2, v1, acc[k][1]);
+              acc[k][2] = fma2(w2, v2, acc[k][2]);
+              acc[k][3] = fma2(w2, v3, acc[k][3]);
             }
           }
         }
       }
 #pragma unroll
-      for (int k = 0; k < 4; ++k) {
+      for (int k = 0; k < kDecSweep; ++k) {
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          const float t = acc[k][e] + __shfl_xor_sync(0xffffffffu, acc[k][e], 16);
-          if (lane < 16 && g0 + k < G) part[(warp * G + g0 + k) * kHeadDim + 8 * c8 + e] = t;
+        for (int e = 0; e < 4; ++e) {
+          float a0, a1;
+          unpack2(acc[k][e], a0, a1);
+          a0 += __shfl_xor_sync(0xffffffffu, a0, 16);
+          a1 += __shfl_xor_sync(0xffffffffu, a1, 16);
+          if (lane < 16 && g0 + k < G)
+            *reinterpret_cast<float2*>(part + (warp * G + g0 + k) * kHeadDim + 8 * c8 + 2 * e) =
+                make_float2(a0, a1);
         }
       }
     }
-    __syncthreads();
+    __syncthreads();   // the block's V stage is free, `part` is complete
+    if (tid == 0 && blk + 2 < nblk) {
+      const uint32_t bytes = (uint32_t)min(kDecBlock, n - (blk + 2) * kDecBlock) * 256u;
+      mbar_expect_tx(&vbar[st], bytes);
+      bulk_load(sV + (size_t)st * kDecBlock * 256, Vb + (size_t)(blk + 2) * kDecBlock * kHeadDim, bytes,
+                &vbar[st]);
+    }
     for (int e = tid; e < G * kHeadDim; e += kDecThreads) {
       const int g = e / kHeadDim;
       float t = 0.f;
@@ -196,26 +251,32 @@ k_decode_attention(const __nv_bfloat16* __restrict__ Kc, const __nv_bfloat16* __
     __syncthreads();
   }
 
-  // ---- merge the cluster's partial results in its first CTA
+  // ---- merge the cluster's partial results: every CTA copies all ranks' (reference, sum) pairs,
+  // then takes a slice of the G * 128 outputs
   cluster.sync();
-  if (crank == 0) {
-    for (int e = tid; e < G * kHeadDim; e += kDecThreads) {
-      const int g = e / kHeadDim;
-      float M = -INFINITY;
-      for (int r = 0; r < S; ++r) M = fmaxf(M, *cluster.map_shared_rank(&xm[g], r));
-      float num = 0.f, den = 0.f;
-      if (M != -INFINITY) {
-        for (int r = 0; r < S; ++r) {
-          const float mr = *cluster.map_shared_rank(&xm[g], r);
-          const float sc = mr == -INFINITY ? 0.f : exp2f(mr - M);
-          num = fmaf(*cluster.map_shared_rank(&xo[e], r), sc, num);
-          den = fmaf(*cluster.map_shared_rank(&xz[g], r), sc, den);
-        }
-      }
-      out[qoff + e] = den > 0.f ? num / den : 0.f;
-    }
+  for (int e = tid; e < S * G; e += kDecThreads) {
+    const int r = e / G, g = e % G;
+    allm[r * kDecMaxG + g] = *cluster.map_shared_rank(&xm[g], r);
+    allz[r * kDecMaxG + g] = *cluster.map_shared_rank(&xz[g], r);
   }
-  cluster.sync();   // the peers' shared memory stays alive until the first CTA has read it
+  __syncthreads();
+  const int per = (G * kHeadDim + S - 1) / S;
+  for (int e = crank * per + tid; e < min((crank + 1) * per, G * kHeadDim); e += kDecThreads) {
+    const int g = e / kHeadDim;
+    float M = -INFINITY;
+    for (int r = 0; r < S; ++r) M = fmaxf(M, allm[r * kDecMaxG + g]);
+    float num = 0.f, den = 0.f;
+    if (M != -INFINITY) {
+      for (int r = 0; r < S; ++r) {
+        const float mr = allm[r * kDecMaxG + g];
+        const float sc = mr == -INFINITY ? 0.f : exp2f(mr - M);
+        num = fmaf(*cluster.map_shared_rank(&xo[e], r), sc, num);
+        den = fmaf(allz[r * kDecMaxG + g], sc, den);
+      }
+    }
+    out[qoff + e] = den > 0.f ? num / den : 0.f;
+  }
+  cluster.sync();   // a CTA's shared memory stays alive until its peers have read it
 }
 
 }  // namespace
@@ -237,7 +298,7 @@ extern "C" int mixkv_decode_attention(const void* K_cache, const void* V_cache,
   if ((reinterpret_cast<uintptr_t>(K_cache) & 15u) || (reinterpret_cast<uintptr_t>(V_cache) & 15u) ||
       (reinterpret_cast<uintptr_t>(q) & 15u))
     return MIXKV_ERR_INVALID_ARG;
-  const size_t smem = dec_floats(gqa_ratio) * 4 + (size_t)kDecBlock * 256;
+  const size_t smem = dec_floats(gqa_ratio) * 4 + 2 * (size_t)kDecBlock * 256;
   {
     const int rc = device_check(nullptr);
     if (rc != MIXKV_OK) return rc;
@@ -248,7 +309,7 @@ extern "C" int mixkv_decode_attention(const void* K_cache, const void* V_cache,
     if (cudaGetDevice(&dev) != cudaSuccess) return MIXKV_ERR_CUDA;
     if (dev < 0 || dev >= 64 || !done[dev]) {
       if (cudaFuncSetAttribute(k_decode_attention, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                               128 * 1024) != cudaSuccess)
+                               160 * 1024) != cudaSuccess)
         return MIXKV_ERR_CUDA;
       if (dev >= 0 && dev < 64) done[dev] = true;
     }
