@@ -295,9 +295,9 @@ int mixkv_similarity_map(const void* X, int32_t heads, int32_t L, int32_t head_d
  *   q                  device, [n_layers, batch, H * G, d] bf16: the token's query per layer
  *   max_rows           upper bound on the rows of one (layer, b, h), e.g. B, or L for a cache
  *                      that was not compressed; rows beyond it are not read.  It only steers
- *                      how many CTAs share one head (a cluster of 1, 2, 4 or 8 splits the rows;
- *                      each CTA walks its share in blocks of 256 with a running softmax), so
- *                      any length is accepted
+ *                      how many CTAs share one head (the warps of a cluster of 1, 2, 4 or 8
+ *                      CTAs take the rows 16 at a time, each with a running softmax), so any
+ *                      length is accepted
  *   out                device, [n_layers, batch, H * G, d] fp32; a head without rows gets zeros
  * softmax_scale 0 means 1 / sqrt(d).  d must be 128, G <= 16 (else MIXKV_ERR_UNSUPPORTED). */
 int mixkv_decode_attention(const void* K_cache, const void* V_cache,

@@ -1,15 +1,25 @@
 // The step after compression: one new query token per sequence attends over the compact cache
 // (paper Sec. 3.1, Eq. 1: generation continues on the compressed K, V).  All layers of a model go
-// in one launch.  The rows of a (layer, sequence, KV head) unit are split over the CTAs of a
-// thread-block cluster (1, 2, 4 or 8: the fewest CTAs that fill the GPU once); a CTA walks its
-// rows in blocks of 128 with a running softmax (reference, sum, weighted value sum per query head
-// of the group).  The loads run ahead of the arithmetic: the V rows of two blocks are on their
-// way to shared memory (bulk copies into a two-stage ring) and the K rows of the next block are
-// on their way to registers (two threads per row, all eight 16-byte loads of a thread in flight)
-// while a block is worked on: logits from the registers, softmax weights, then sixteen threads
-// per V row add the weighted rows of all query heads in one sweep (packed fp32 pairs).  The
-// cluster's partial results are merged through distributed shared memory, every CTA taking a
-// slice of the outputs.  Every row is read once.
+// in one launch.  With one query token and G query heads per KV head the two contractions have
+// 7 .. 16 rows on one side: too few for the 64- or 128-row tcgen05 tiles (nine tenths of such a
+// tile would be padding), too many multiply-adds for the fp32 pipe at HBM speed (2 * 2 * G * 128
+// per 512-byte row pair), so they run as warp-level mma.sync m16n8k16 (bf16 x bf16 -> fp32) with
+// every operand loaded from global memory straight into its fragment, no shared-memory staging:
+//
+//   * a warp takes 16 cache rows per step.  logits: D[head, row] = q[head, :] . K[row, :],
+//     A = q (held in registers for the whole kernel), B = K rows.  The contraction index may be
+//     permuted freely as long as A and B agree, so a lane takes 64 CONTIGUOUS bytes of its row
+//     (four 16-byte loads) and deals them out over the eight k-steps.
+//   * softmax weights with a running (reference, sum) per head in log2 units; the weights leave
+//     as TWO bf16 (value and remainder), so the value sum is fp32-grade.
+//   * values: D[head, dim] += P[head, row] . V[row, dim].  B wants two rows of one dim per
+//     register: a lane loads 32 contiguous bytes of four rows and byte-permutes pairs of rows
+//     together; which output column a lane's dim lands in is again a free permutation.
+//
+// The rows of a (layer, sequence, KV head) unit are dealt out in steps of 16 over the warps of a
+// thread-block cluster (1, 2, 4 or 8 CTAs of four warps; as many as fit the GPU in one wave), and
+// a warp keeps two register sets so that the loads of its next step fly while it works.  Warps merge through shared memory, the CTAs of a cluster through distributed
+// shared memory, every CTA taking a slice of the outputs.  Every row is read once.
 #include <cooperative_groups.h>
 
 #include "tc_common.cuh"
@@ -19,259 +29,277 @@ namespace cg = cooperative_groups;
 namespace mixkv {
 namespace {
 
-constexpr int kDecThreads = 256;
+constexpr int kDecWarps = 4;
+constexpr int kDecThreads = kDecWarps * 32;
 constexpr int kDecMaxG = 16;
-constexpr int kDecBlock = 128;   // rows per block: two threads per logit row
-constexpr int kDecSweep = 8;     // query heads whose value sums a thread holds at once
+constexpr int kDecStep = 16;     // cache rows per warp step
 
-// Floats of dynamic shared memory in front of the V ring: sq [G][128] queries, sp [G][128]
-// logits then weights, part [8][G][128] per-warp value sums, xo [G][128] running weighted value
-// sum, xm / xz / sscale [16] each, then the merge's copy of every rank's xm and xz [2][8][16].
-__host__ __device__ constexpr size_t dec_floats(int G) {
-  return (size_t)G * (kHeadDim + kDecBlock + 8 * kHeadDim + kHeadDim) + 3 * kDecMaxG +
-         2 * 8 * kDecMaxG;
+// Floats of dynamic shared memory for GP = 8 or 16 head slots: wacc [warps][GP][132] per-warp
+// value sums, xo [GP][128] the CTA's, wm / wz [warps][16], xm / xz [16], allm / allz [8][16]
+// every rank's (reference, sum) during the cluster merge.
+constexpr int kDecHeadPitch = kHeadDim + 4;   // floats between the heads of a warp's value sums
+__host__ __device__ constexpr size_t dec_floats(int GP) {
+  return (size_t)kDecWarps * GP * kDecHeadPitch + (size_t)GP * kHeadDim + 2 * kDecWarps * kDecMaxG +
+         2 * kDecMaxG + 2 * 8 * kDecMaxG;
 }
+// Slot of dimension `dim` inside a head of a warp's value sums: one pad word per 32 dimensions
+// and a head pitch of 132 put the 32 lanes of a fragment store (8 heads x 4 dimensions 32 apart)
+// into 32 different banks.
+__device__ __forceinline__ int dec_slot(int dim) { return dim + (dim >> 5); }
 
-__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+// D (16 x 8, fp32) += A (16 x 16, bf16, row) * B (16 x 8, bf16, col).  Lane l = 4 g + t holds
+//   A: a0 (row g, k 2t..2t+1)  a1 (row g+8, same k)  a2 (row g, k 2t+8..2t+9)  a3 (row g+8, ..)
+//   B: b0 (k 2t..2t+1, col g)  b1 (k 2t+8..2t+9, col g)
+//   D: d0 d1 (row g, cols 2t, 2t+1)  d2 d3 (row g+8, same cols)
+__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], const uint32_t b0,
+                                         const uint32_t b1) {
   asm volatile(
-      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-          smem_u32(dst)),
-      "l"(src), "r"(bytes), "r"(smem_u32(bar))
-      : "memory");
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, "
+      "{%8, %9}, {%0, %1, %2, %3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+// bf16 pair (x in the low half) of two floats, and what rounding left over.
+__device__ __forceinline__ uint32_t pack_bf16(const float x, const float y) {
+  const __nv_bfloat162 v = __floats2bfloat162_rn(x, y);
+  return *reinterpret_cast<const uint32_t*>(&v);
+}
+__device__ __forceinline__ void split_bf16(const float x, const float y, uint32_t& hi, uint32_t& lo) {
+  hi = pack_bf16(x, y);
+  lo = pack_bf16(x - __uint_as_float(hi << 16), y - __uint_as_float(hi & 0xffff0000u));
+}
+__device__ __forceinline__ uint32_t word_of(const uint4& v, const int i) {
+  return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w;
+}
+__device__ __forceinline__ float quad_max(float v) {
+  v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 1));
+  return fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 2));
+}
+__device__ __forceinline__ float quad_sum(float v) {
+  v += __shfl_xor_sync(0xffffffffu, v, 1);
+  return v + __shfl_xor_sync(0xffffffffu, v, 2);
 }
 
-// Packed fp32 pairs: one instruction for two lanes of arithmetic.
-typedef unsigned long long f32x2;
-__device__ __forceinline__ f32x2 pack2(float a, float b) {
-  f32x2 r;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
-  return r;
-}
-__device__ __forceinline__ void unpack2(f32x2 v, float& a, float& b) {
-  asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
-}
-__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
-  f32x2 d;
-  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-  return d;
-}
-// The two bf16 of a 32-bit word as an fp32 pair (low half first).
-__device__ __forceinline__ f32x2 bf16x2_to_f32x2(uint32_t w) {
-  return pack2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
-}
-
-// grid: n_layers * batch * H * S, clusters of S.
+// grid: n_layers * batch * H * S, clusters of S.  WIDE: more than eight query heads per KV head
+// (head slots 8..15 of the tiles carry data).
+template <bool WIDE>
 __global__ void __launch_bounds__(kDecThreads, 2)
 k_decode_attention(const __nv_bfloat16* __restrict__ Kc, const __nv_bfloat16* __restrict__ Vc,
                    const int* __restrict__ row_offsets, const long long rows_cap,
                    const __nv_bfloat16* __restrict__ q, const int BH, const int H, const int G,
                    const float scale_log2e, const int max_rows, float* __restrict__ out) {
+  constexpr int GP = WIDE ? 16 : 8;
   extern __shared__ __align__(16) float dsm[];
-  float* sq = dsm;                              // [G][128]
-  float* sp = sq + G * kHeadDim;                // [G][128]
-  float* part = sp + G * kDecBlock;             // [8][G][128]
-  float* xo = part + 8 * G * kHeadDim;          // [G][128]
-  float* xm = xo + G * kHeadDim;                // [16]
-  float* xz = xm + kDecMaxG;                    // [16]
-  float* sscale = xz + kDecMaxG;                // [16] rescale of the running sums for this block
-  float* allm = sscale + kDecMaxG;              // [8][16] merge: every rank's xm
-  float* allz = allm + 8 * kDecMaxG;            // [8][16] merge: every rank's xz
-  unsigned char* sV = reinterpret_cast<unsigned char*>(dsm + dec_floats(G));   // [2][128][256 B]
-  __shared__ __align__(8) uint64_t vbar[2];
-  __shared__ int vabort;
+  float* wacc = dsm;                                   // [warps][GP][kDecHeadPitch]
+  float* xo = wacc + kDecWarps * GP * kDecHeadPitch;   // [GP][128]
+  float* wm = xo + GP * kHeadDim;                      // [warps][16]
+  float* wz = wm + kDecWarps * kDecMaxG;               // [warps][16]
+  float* xm = wz + kDecWarps * kDecMaxG;               // [16]
+  float* xz = xm + kDecMaxG;                           // [16]
+  float* allm = xz + kDecMaxG;                         // [8][16]
+  float* allz = allm + 8 * kDecMaxG;                   // [8][16]
   cg::cluster_group cluster = cg::this_cluster();
   const int S = (int)cluster.num_blocks(), crank = (int)cluster.block_rank();
   const int unit = blockIdx.x / S, layer = unit / BH, bh = unit % BH, b = bh / H, h = bh % H;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int g = lane >> 2, t = lane & 3;
   pdl_launch_dependents();
-  if (tid == 0) {
-    mbar_init(&vbar[0], 1);
-    mbar_init(&vbar[1], 1);
-    vabort = 0;
-    mbar_init_fence();
-  }
   pdl_wait();
   const int* ro = row_offsets + (size_t)layer * (BH + 1);
-  const int r0 = ro[bh], n_unit = min(ro[bh + 1] - r0, max_rows);
-  const int chunk = (n_unit + S - 1) / S;
-  const int c0 = min(crank * chunk, n_unit), n = min(chunk, n_unit - c0);   // this CTA's rows
-  const int nblk = (n + kDecBlock - 1) / kDecBlock;
-  const __nv_bfloat16* Kb = Kc + ((size_t)layer * rows_cap + r0 + c0) * kHeadDim;
-  const __nv_bfloat16* Vb = Vc + ((size_t)layer * rows_cap + r0 + c0) * kHeadDim;
+  const int r0 = ro[bh], n = min(ro[bh + 1] - r0, max_rows);
+  const __nv_bfloat16* Kb = Kc + ((size_t)layer * rows_cap + r0) * kHeadDim;
+  const __nv_bfloat16* Vb = Vc + ((size_t)layer * rows_cap + r0) * kHeadDim;
   const size_t qoff = (((size_t)layer * (BH / H) + b) * H + h) * (size_t)G * kHeadDim;
-  __syncthreads();   // the barriers are initialised
-  // ---- the V rows of the first two blocks start towards the ring
-  if (tid == 0) {
-    for (int k = 0; k < 2 && k < nblk; ++k) {
-      const uint32_t bytes = (uint32_t)min(kDecBlock, n - k * kDecBlock) * 256u;
-      mbar_expect_tx(&vbar[k], bytes);
-      bulk_load(sV + (size_t)k * kDecBlock * 256, Vb + (size_t)k * kDecBlock * kHeadDim, bytes, &vbar[k]);
+
+  // ---- query fragments: k-step kt of lane (g, t) covers dimensions 32 t + 4 kt .. + 3 of heads
+  // g and g + 8, the first two as a0 / a1, the last two as a2 / a3
+  uint32_t qa[8][4];
+  {
+    const uint4* q0 = reinterpret_cast<const uint4*>(q + qoff + (size_t)g * kHeadDim + 32 * t);
+    const uint4* q1 = reinterpret_cast<const uint4*>(q + qoff + (size_t)(g + 8) * kHeadDim + 32 * t);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      uint4 u0 = make_uint4(0, 0, 0, 0), u1 = u0;
+      if (g < G) u0 = __ldg(q0 + i);
+      if (WIDE && g + 8 < G) u1 = __ldg(q1 + i);
+      qa[2 * i][0] = u0.x, qa[2 * i][2] = u0.y, qa[2 * i + 1][0] = u0.z, qa[2 * i + 1][2] = u0.w;
+      qa[2 * i][1] = u1.x, qa[2 * i][3] = u1.y, qa[2 * i + 1][1] = u1.z, qa[2 * i + 1][3] = u1.w;
     }
   }
-  // ---- the K rows of the first block start towards registers: row tid / 2, dimensions
-  // 64 * (tid & 1) .. + 63
-  const int row = tid >> 1, hf = tid & 1;
-  uint4 kv[8];
-  auto load_k = [&](const int blk) {
-    const int rr = blk * kDecBlock + row;
-    if (rr < n) {
-      const uint4* krow = reinterpret_cast<const uint4*>(Kb + (size_t)rr * kHeadDim + hf * 64);
+  // value sums: tile dt, registers 0 1 = head g, dimensions 16 (2t) + dt and 16 (2t + 1) + dt;
+  // registers 2 3 = head g + 8
+  float acc[16][4];
 #pragma unroll
-      for (int c = 0; c < 8; ++c) kv[c] = __ldg(krow + c);
+  for (int dt = 0; dt < 16; ++dt)
+#pragma unroll
+    for (int c = 0; c < 4; ++c) acc[dt][c] = 0.f;
+  float m0 = -INFINITY, m1 = -INFINITY, z0 = 0.f, z1 = 0.f;
+
+  const int nsteps = (n + kDecStep - 1) / kDecStep;
+  // All loads of a step: K rows rb + 8 j + g (64 bytes from 64 t), V rows rb + 2t, 2t + 1,
+  // 2t + 8, 2t + 9 (32 bytes from 32 g).  Rows past the end repeat the last row; their weights
+  // are zero.
+  auto load_step = [&](const int step, uint4 (&kq)[2][4], uint4 (&vq)[4][2]) {
+    const int rb = step * kDecStep;
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      const int row = min(rb + 8 * j + g, n - 1);
+      const uint4* p = reinterpret_cast<const uint4*>(Kb + (size_t)row * kHeadDim + 32 * t);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) kq[j][i] = __ldg(p + i);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int row = min(rb + 2 * t + (u & 1) + 8 * (u >> 1), n - 1);
+      const uint4* p = reinterpret_cast<const uint4*>(Vb + (size_t)row * kHeadDim + 16 * g);
+      vq[u][0] = __ldg(p);
+      vq[u][1] = __ldg(p + 1);
     }
   };
-  if (nblk > 0) load_k(0);
-  for (int e = tid; e < G * kHeadDim; e += kDecThreads) {
-    sq[e] = __bfloat162float(q[qoff + e]);
-    xo[e] = 0.f;
-  }
-  if (tid < kDecMaxG) xm[tid] = -INFINITY, xz[tid] = 0.f;
-  __syncthreads();
-
-  for (int blk = 0; blk < nblk; ++blk) {
-    const int nb = min(kDecBlock, n - blk * kDecBlock);
-    const int st = blk & 1;
-    // ---- logits (log2 units) from the K registers
+  auto work_step = [&](const int step, const uint4 (&kq)[2][4], const uint4 (&vq)[4][2]) {
+    const int rb = step * kDecStep;
+    // ---- logits: s[j] registers 0 1 = head g, rows rb + 8 j + 2t, + 1; 2 3 = head g + 8
+    float s[2][4];
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+#pragma unroll
+      for (int c = 0; c < 4; ++c) s[j][c] = 0.f;
+#pragma unroll
+      for (int kt = 0; kt < 8; ++kt)
+        mma_bf16(s[j], qa[kt], word_of(kq[j][kt >> 1], 2 * (kt & 1)),
+                 word_of(kq[j][kt >> 1], 2 * (kt & 1) + 1));
+    }
+    // ---- softmax weights under the running reference of each head (log2 units)
+    float p[2][4];
+#pragma unroll
+    for (int j = 0; j < 2; ++j)
+#pragma unroll
+      for (int c = 0; c < 4; ++c)
+        p[j][c] = rb + 8 * j + 2 * t + (c & 1) < n ? s[j][c] * scale_log2e : -INFINITY;
     {
-      f32x2 d[kDecMaxG];
+      const float mx = quad_max(fmaxf(fmaxf(p[0][0], p[0][1]), fmaxf(p[1][0], p[1][1])));
+      const float mn = fmaxf(m0, mx), f = exp2f(m0 - mn);   // mx is finite: the step has a row
+      if (f != 1.f) {
+        z0 *= f;
 #pragma unroll
-      for (int g = 0; g < kDecMaxG; ++g) d[g] = pack2(0.f, 0.f);
-      if (row < nb) {
-#pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          const f32x2 k0 = bf16x2_to_f32x2(kv[c].x), k1 = bf16x2_to_f32x2(kv[c].y);
-          const f32x2 k2 = bf16x2_to_f32x2(kv[c].z), k3 = bf16x2_to_f32x2(kv[c].w);
-#pragma unroll
-          for (int g = 0; g < kDecMaxG; ++g) {
-            if (g < G) {
-              const ulonglong2* qg =
-                  reinterpret_cast<const ulonglong2*>(sq + g * kHeadDim + hf * 64 + 8 * c);
-              const ulonglong2 qa = qg[0], qb = qg[1];
-              d[g] = fma2(k0, qa.x, fma2(k1, qa.y, d[g]));
-              d[g] = fma2(k2, qb.x, fma2(k3, qb.y, d[g]));
-            }
-          }
-        }
+        for (int dt = 0; dt < 16; ++dt) acc[dt][0] *= f, acc[dt][1] *= f;
       }
-      // the next block's K rows start towards the registers just read
-      if (blk + 1 < nblk) load_k(blk + 1);
+      m0 = mn;
 #pragma unroll
-      for (int g = 0; g < kDecMaxG; ++g) {
-        if (g < G) {
-          float d0, d1;
-          unpack2(d[g], d0, d1);
-          const float mine = d0 + d1;
-          const float o = __shfl_xor_sync(0xffffffffu, mine, 1);
-          const float t = hf ? o + mine : mine + o;   // first half + second half in both threads
-          if (hf == 0 && row < nb) sp[g * kDecBlock + row] = t * scale_log2e;
-        }
+      for (int j = 0; j < 2; ++j) {
+        p[j][0] = exp2f(p[j][0] - mn);
+        p[j][1] = exp2f(p[j][1] - mn);
+        z0 += p[j][0] + p[j][1];
       }
     }
-    __syncthreads();
-    // ---- running softmax per query head: warp w takes heads w, w + 8, ...
-    for (int g = warp; g < G; g += kDecThreads / 32) {
-      float* prow = sp + g * kDecBlock;
-      float mx = -INFINITY;
-      for (int r = lane; r < nb; r += 32) mx = fmaxf(mx, prow[r]);
-      mx = warp_max(mx);
-      const float m_old = xm[g], m_new = fmaxf(m_old, mx);
-      float sum = 0.f;
-      for (int r = lane; r < nb; r += 32) {
-        const float e = exp2f(prow[r] - m_new);
-        prow[r] = e;
-        sum += e;
+    if (WIDE) {
+      const float mx = quad_max(fmaxf(fmaxf(p[0][2], p[0][3]), fmaxf(p[1][2], p[1][3])));
+      const float mn = fmaxf(m1, mx), f = exp2f(m1 - mn);
+      if (f != 1.f) {
+        z1 *= f;
+#pragma unroll
+        for (int dt = 0; dt < 16; ++dt) acc[dt][2] *= f, acc[dt][3] *= f;
       }
-      sum = warp_sum(sum);
-      if (lane == 0) {
-        const float sc = m_old == -INFINITY ? 0.f : exp2f(m_old - m_new);
-        sscale[g] = sc;
-        xz[g] = xz[g] * sc + sum;
-        xm[g] = m_new;
+      m1 = mn;
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        p[j][2] = exp2f(p[j][2] - mn);
+        p[j][3] = exp2f(p[j][3] - mn);
+        z1 += p[j][2] + p[j][3];
       }
     }
-    const bool vok = mbar_wait(&vbar[st], (blk >> 1) & 1, &vabort);
-    __syncthreads();
-    // ---- weighted sum of the value rows from shared memory: sixteen threads per row (16 bytes
-    // each), sixteen rows per sweep over the block, up to eight query heads at a time
-    const unsigned char* vblk = sV + (size_t)st * kDecBlock * 256;
-    const int c8 = tid & 15, rg = tid >> 4;
-    for (int g0 = 0; g0 < G; g0 += kDecSweep) {
-      f32x2 acc[kDecSweep][4];
-#pragma unroll
-      for (int k = 0; k < kDecSweep; ++k)
-#pragma unroll
-        for (int e = 0; e < 4; ++e) acc[k][e] = pack2(0.f, 0.f);
-      if (vok) {
-#pragma unroll 2
-        for (int r = rg; r < nb; r += 16) {
-          const uint4 vv = *reinterpret_cast<const uint4*>(vblk + (size_t)r * 256 + 16 * c8);
-          const f32x2 v0 = bf16x2_to_f32x2(vv.x), v1 = bf16x2_to_f32x2(vv.y);
-          const f32x2 v2 = bf16x2_to_f32x2(vv.z), v3 = bf16x2_to_f32x2(vv.w);
-#pragma unroll
-          for (int k = 0; k < kDecSweep; ++k) {
-            if (g0 + k < G) {
-              const float wgt = sp[(g0 + k) * kDecBlock + r];
-              const f32x2 w2 = pack2(wgt, wgt);
-              acc[k][0] = fma2(w2, v0, acc[k][0]);
-              acc[k][1] = fma2(w2, v1, acc[k][1]);
-              acc[k][2] = fma2(w2, v2, acc[k][2]);
-              acc[k][3] = fma2(w2, v3, acc[k][3]);
-            }
-          }
-        }
-      }
-#pragma unroll
-      for (int k = 0; k < kDecSweep; ++k) {
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          float a0, a1;
-          unpack2(acc[k][e], a0, a1);
-          a0 += __shfl_xor_sync(0xffffffffu, a0, 16);
-          a1 += __shfl_xor_sync(0xffffffffu, a1, 16);
-          if (lane < 16 && g0 + k < G)
-            *reinterpret_cast<float2*>(part + (warp * G + g0 + k) * kHeadDim + 8 * c8 + 2 * e) =
-                make_float2(a0, a1);
-        }
-      }
+    // the weights as bf16 value + bf16 remainder: A fragments over the 16 rows of the step
+    uint32_t ahi[4] = {0, 0, 0, 0}, alo[4] = {0, 0, 0, 0};
+    split_bf16(p[0][0], p[0][1], ahi[0], alo[0]);
+    split_bf16(p[1][0], p[1][1], ahi[2], alo[2]);
+    if (WIDE) {
+      split_bf16(p[0][2], p[0][3], ahi[1], alo[1]);
+      split_bf16(p[1][2], p[1][3], ahi[3], alo[3]);
     }
-    __syncthreads();   // the block's V stage is free, `part` is complete
-    if (tid == 0 && blk + 2 < nblk) {
-      const uint32_t bytes = (uint32_t)min(kDecBlock, n - (blk + 2) * kDecBlock) * 256u;
-      mbar_expect_tx(&vbar[st], bytes);
-      bulk_load(sV + (size_t)st * kDecBlock * 256, Vb + (size_t)(blk + 2) * kDecBlock * kHeadDim, bytes,
-                &vbar[st]);
-    }
-    for (int e = tid; e < G * kHeadDim; e += kDecThreads) {
-      const int g = e / kHeadDim;
-      float t = 0.f;
+    // ---- values: tile dt takes dimension 16 g + dt of this lane's four rows
 #pragma unroll
-      for (int w = 0; w < 8; ++w) t += part[w * G * kHeadDim + e];
-      xo[e] = xo[e] * sscale[g] + t;
+    for (int dt = 0; dt < 16; ++dt) {
+      const int w = dt >> 1;
+      const uint32_t sel = (dt & 1) ? 0x7632u : 0x5410u;
+      const uint32_t b0 = __byte_perm(word_of(vq[0][w >> 2], w & 3), word_of(vq[1][w >> 2], w & 3), sel);
+      const uint32_t b1 = __byte_perm(word_of(vq[2][w >> 2], w & 3), word_of(vq[3][w >> 2], w & 3), sel);
+      mma_bf16(acc[dt], ahi, b0, b1);
+      mma_bf16(acc[dt], alo, b0, b1);
     }
-    __syncthreads();
+  };
+  // two register sets: the loads of a warp's next step are in flight while it works on this one
+  {
+    const int stride = S * kDecWarps;
+    uint4 kA[2][4], vA[4][2], kB[2][4], vB[4][2];
+    int step = crank * kDecWarps + warp;
+    if (step < nsteps) load_step(step, kA, vA);
+    while (step < nsteps) {
+      if (step + stride < nsteps) load_step(step + stride, kB, vB);
+      work_step(step, kA, vA);
+      step += stride;
+      if (step >= nsteps) break;
+      if (step + stride < nsteps) load_step(step + stride, kA, vA);
+      work_step(step, kB, vB);
+      step += stride;
+    }
   }
 
-  // ---- merge the cluster's partial results: every CTA copies all ranks' (reference, sum) pairs,
-  // then takes a slice of the G * 128 outputs
+  // ---- the warps of the CTA merge through shared memory
+  z0 = quad_sum(z0);
+  z1 = quad_sum(z1);
+#pragma unroll
+  for (int dt = 0; dt < 16; ++dt) {
+    float* w0 = wacc + ((size_t)warp * GP + g) * kDecHeadPitch;
+    w0[dec_slot(16 * (2 * t) + dt)] = acc[dt][0];
+    w0[dec_slot(16 * (2 * t + 1) + dt)] = acc[dt][1];
+    if (WIDE) {
+      w0[8 * kDecHeadPitch + dec_slot(16 * (2 * t) + dt)] = acc[dt][2];
+      w0[8 * kDecHeadPitch + dec_slot(16 * (2 * t + 1) + dt)] = acc[dt][3];
+    }
+  }
+  if (t == 0) {
+    wm[warp * kDecMaxG + g] = m0, wz[warp * kDecMaxG + g] = z0;
+    wm[warp * kDecMaxG + g + 8] = WIDE ? m1 : -INFINITY, wz[warp * kDecMaxG + g + 8] = WIDE ? z1 : 0.f;
+  }
+  __syncthreads();
+  for (int e = tid; e < GP * kHeadDim; e += kDecThreads) {
+    const int head = e / kHeadDim, dim = e % kHeadDim;
+    float M = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < kDecWarps; ++w) M = fmaxf(M, wm[w * kDecMaxG + head]);
+    float num = 0.f, den = 0.f;
+#pragma unroll
+    for (int w = 0; w < kDecWarps; ++w) {
+      const float mw = wm[w * kDecMaxG + head];
+      const float sc = mw == -INFINITY ? 0.f : exp2f(mw - M);
+      num = fmaf(wacc[((size_t)w * GP + head) * kDecHeadPitch + dec_slot(dim)], sc, num);
+      den = fmaf(wz[w * kDecMaxG + head], sc, den);
+    }
+    xo[e] = num;
+    if (dim == 0) xm[head] = M, xz[head] = den;
+  }
+
+  // ---- the CTAs of the cluster merge through distributed shared memory: every CTA copies all
+  // ranks' (reference, sum) pairs, then takes a slice of the G * 128 outputs
   cluster.sync();
   for (int e = tid; e < S * G; e += kDecThreads) {
-    const int r = e / G, g = e % G;
-    allm[r * kDecMaxG + g] = *cluster.map_shared_rank(&xm[g], r);
-    allz[r * kDecMaxG + g] = *cluster.map_shared_rank(&xz[g], r);
+    const int r = e / G, head = e % G;
+    allm[r * kDecMaxG + head] = *cluster.map_shared_rank(&xm[head], r);
+    allz[r * kDecMaxG + head] = *cluster.map_shared_rank(&xz[head], r);
   }
   __syncthreads();
   const int per = (G * kHeadDim + S - 1) / S;
   for (int e = crank * per + tid; e < min((crank + 1) * per, G * kHeadDim); e += kDecThreads) {
-    const int g = e / kHeadDim;
+    const int head = e / kHeadDim;
     float M = -INFINITY;
-    for (int r = 0; r < S; ++r) M = fmaxf(M, allm[r * kDecMaxG + g]);
+    for (int r = 0; r < S; ++r) M = fmaxf(M, allm[r * kDecMaxG + head]);
     float num = 0.f, den = 0.f;
     if (M != -INFINITY) {
       for (int r = 0; r < S; ++r) {
-        const float mr = allm[r * kDecMaxG + g];
+        const float mr = allm[r * kDecMaxG + head];
         const float sc = mr == -INFINITY ? 0.f : exp2f(mr - M);
         num = fmaf(*cluster.map_shared_rank(&xo[e], r), sc, num);
-        den = fmaf(allz[r * kDecMaxG + g], sc, den);
+        den = fmaf(allz[r * kDecMaxG + head], sc, den);
       }
     }
     out[qoff + e] = den > 0.f ? num / den : 0.f;
@@ -298,33 +326,25 @@ extern "C" int mixkv_decode_attention(const void* K_cache, const void* V_cache,
   if ((reinterpret_cast<uintptr_t>(K_cache) & 15u) || (reinterpret_cast<uintptr_t>(V_cache) & 15u) ||
       (reinterpret_cast<uintptr_t>(q) & 15u))
     return MIXKV_ERR_INVALID_ARG;
-  const size_t smem = dec_floats(gqa_ratio) * 4 + 2 * (size_t)kDecBlock * 256;
   {
     const int rc = device_check(nullptr);
     if (rc != MIXKV_OK) return rc;
   }
-  if (smem > 48 * 1024) {
-    static bool done[64] = {false};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return MIXKV_ERR_CUDA;
-    if (dev < 0 || dev >= 64 || !done[dev]) {
-      if (cudaFuncSetAttribute(k_decode_attention, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                               160 * 1024) != cudaSuccess)
-        return MIXKV_ERR_CUDA;
-      if (dev >= 0 && dev < 64) done[dev] = true;
-    }
-  }
   const long long units = (long long)n_layers * batch * kv_heads;
   if (units * 8 > 0x7fffffffLL) return MIXKV_ERR_UNSUPPORTED;
-  // rows of a unit over a cluster: the fewest CTAs that fill the GPU once (more CTAs than that
-  // were measured slower: the cost of a call is the serial latency of a CTA, and launching more
-  // of them adds to it), and no CTA with more than 1024 rows
+  // CTAs per unit: as many as still fit the GPU in one wave (two CTAs of four warps per SM: the
+  // two register sets of a warp hold 16 KB of loads in flight) while every warp keeps at least
+  // two steps to overlap
+  const long long steps = ((long long)max_rows + kDecStep - 1) / kDecStep;
   int S = 1;
-  while (S < 8 && units * S < device_sm_count()) S *= 2;
-  while (S < 8 && (max_rows + S - 1) / S > 8 * kDecBlock) S *= 2;
+  while (S < 8 && units * (2 * S) <= 2LL * device_sm_count() && 2LL * (2 * S) * kDecWarps <= steps)
+    S *= 2;
+  const bool wide = gqa_ratio > 8;
+  const size_t smem = dec_floats(wide ? 16 : 8) * 4;
   const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)kHeadDim);
   const cudaError_t e = launch_pdl(
-      k_decode_attention, dim3((unsigned)(units * S)), dim3(kDecThreads), smem, (cudaStream_t)stream, S,
+      wide ? k_decode_attention<true> : k_decode_attention<false>, dim3((unsigned)(units * S)),
+      dim3(kDecThreads), smem, (cudaStream_t)stream, S,
       reinterpret_cast<const __nv_bfloat16*>(K_cache), reinterpret_cast<const __nv_bfloat16*>(V_cache),
       out_row_offsets, (long long)rows_cap, reinterpret_cast<const __nv_bfloat16*>(q), batch * kv_heads,
       kv_heads, gqa_ratio, scale * kLog2e, max_rows, out);

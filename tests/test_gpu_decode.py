@@ -10,7 +10,7 @@ from paper_2510_20707_b200 import binding, synth
 from parity import params_pair
 
 pytestmark = pytest.mark.gpu
-RTOL, ATOL = 2e-4, 2e-5   # fp32 dot products of 128 terms, approximate exp2, sums over <= B rows
+RTOL, ATOL = 2e-4, 2e-5   # fp32 accumulation of exact bf16 products, weights carried as two bf16
 
 
 def bits_to_dev(a):
@@ -59,8 +59,9 @@ def test_ragged_adaptive_cache():
 @pytest.mark.parametrize("rows,G", [((4096, 1000, 4096, 37), 7), ((20000, 513), 4), ((256, 257), 16)])
 def test_long_rows_split_over_a_cluster(rows, G):
     # heads with thousands of rows (a large budget, or a cache that was not compressed): the rows
-    # of a head are split over the CTAs of a cluster and walked in blocks of 256 with a running
-    # softmax; two layers, ragged heads, a sharp row so that the running reference moves
+    # of a head are dealt out 16 at a time over the warps of a cluster, each with a running
+    # softmax; two layers, ragged heads (row counts that are no multiple of 16), G on both sides
+    # of 8 (the second half of the 16 head slots), a sharp row so that the running reference moves
     H, NL = len(rows), 2
     rng = np.random.default_rng(sum(rows))
     cap = int(sum(rows))
@@ -69,6 +70,24 @@ def test_long_rows_split_over_a_cluster(rows, G):
     q = rng.standard_normal((NL, 1, H * G, 128)).astype(np.float32)
     K[0, rows[0] - 3] = 6.0 * q[0, 0, 0]          # one key far above the rest, late in head 0
     Kb, Vb, qb = (synth.f32_to_bf16_bits(a) for a in (K, V, q))
+    offs = np.tile(np.concatenate([[0], np.cumsum(rows)]).astype(np.int32), (NL, 1))
+    out = binding.decode_attention(bits_to_dev(Kb), bits_to_dev(Vb), torch.from_numpy(offs).cuda(),
+                                   bits_to_dev(qb), H, G, max_rows=max(rows)).cpu().numpy()
+    for l in range(NL):
+        ref = decode_plain.decode_attention(Kb[l], Vb[l], offs[l], qb[l], H, G)
+        assert np.allclose(out[l], ref, rtol=RTOL, atol=ATOL), f"layer {l}"
+
+
+@pytest.mark.parametrize("G", [1, 8, 9, 13])
+def test_step_edges_and_head_counts(G):
+    # heads of 1, 15, 16, 17 and 33 rows (below, at and past one 16-row step) for group sizes at
+    # the edges of the 8 + 8 head slots of a tile
+    rows, NL = (1, 15, 16, 17, 33), 2
+    H = len(rows)
+    rng = np.random.default_rng(100 + G)
+    cap = int(sum(rows))
+    Kb, Vb, qb = (synth.f32_to_bf16_bits(rng.standard_normal(sh).astype(np.float32))
+                  for sh in ((NL, cap, 128), (NL, cap, 128), (NL, 1, H * G, 128)))
     offs = np.tile(np.concatenate([[0], np.cumsum(rows)]).astype(np.int32), (NL, 1))
     out = binding.decode_attention(bits_to_dev(Kb), bits_to_dev(Vb), torch.from_numpy(offs).cuda(),
                                    bits_to_dev(qb), H, G, max_rows=max(rows)).cpu().numpy()
