@@ -524,6 +524,7 @@ constexpr int kTailCluster = 8;
 constexpr int kTailThreads = 512;
 constexpr int kTailCacheCap = 16384;       // positions a CTA of a cluster keeps in shared memory
 constexpr int kTailCacheCapSolo = 40960;   // positions a CTA that owns a whole head keeps
+constexpr int kTailListCap = 2048;         // keys of the threshold bin a lone CTA lists after two digits
 
 struct TailKernelArgs {
   const float* scores;        // select on these (FUSED == false)
@@ -570,7 +571,8 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
   __shared__ int hist[2][256];
   __shared__ int s_scan[32][2];
   __shared__ __align__(8) int s_tot[2];
-  __shared__ int s_sel[2];      // digit, remaining
+  __shared__ int s_sel[3];      // digit, remaining, keys in the digit's bin
+  __shared__ int s_nlist;
   __shared__ int s_off;
   __shared__ float sc[8];
   cg::cluster_group cluster = cg::this_cluster();
@@ -594,7 +596,7 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
   const int c0 = min(crank * chunk, P);
   const int n = min(chunk, P - c0);
   unsigned* skeys = reinterpret_cast<unsigned*>(tail_smem);            // [kslot(chunk) + 1]
-  float* sraw = reinterpret_cast<float*>(skeys + kslot(chunk) + 1);    // FUSED: [8 T + 64] stage
+  float* sraw = reinterpret_cast<float*>(skeys + kslot(chunk) + 1);    // FUSED: [8 T + 64] stage; else [kTailListCap]
 
   pdl_launch_dependents();
   pdl_wait();
@@ -612,6 +614,7 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
     }
     if (lane == 0) {
       s_off = off;
+      s_nlist = 0;
       s_sel[1] = cnt;
       if (crank == 0) {
         idx_offsets[bh] = off;
@@ -719,6 +722,31 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
     auto count_digit = [&](const unsigned digit, const int buf) {
       count_digits(hist[buf], digit, lane);
     };
+    // Threads 0..255 bring the number of keys in their bin: the bin that holds the left-th
+    // largest key goes to s_sel[0], how many keys are still needed from inside it to s_sel[1],
+    // its size to s_sel[2].  All threads call it; it ends on a CTA barrier.
+    auto find_digit = [&](const int tot, const int left) {
+      int incl = tot;   // suffix sums over the 256 bins: this bin and those above it
+      if (tid < 256) {
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int v = __shfl_down_sync(0xffffffffu, incl, o);
+          if (lane + o < 32) incl += v;
+        }
+        if (lane == 0) s_scan[warp][0] = incl;
+      }
+      __syncthreads();
+      if (tid < 256) {
+        int above = incl - tot;
+        for (int w = warp + 1; w < 8; ++w) above += s_scan[w][0];
+        if (above < left && left <= above + tot) {
+          s_sel[0] = tid;
+          s_sel[1] = left - above;
+          s_sel[2] = tot;
+        }
+      }
+      __syncthreads();
+    };
     for (int pass = 0; pass < 4; ++pass) {
       const int shift = 24 - 8 * pass, buf = pass & 1;
       if (inreg) {
@@ -735,19 +763,23 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
             if (e < R) count_digit(dg[e], buf);
         }
       } else {
-        for (int e = 0; e < R; ++e) {   // same trip count in every lane: full-warp votes
-          const int j = e * T + tid;
-          unsigned digit = 0xffffffffu;
-          if (j < n) {
-            const unsigned key = key_at(j);
-            if ((key & mask) == prefix) digit = (key >> shift) & 255u;
+        for (int e0 = 0; e0 < R; e0 += 8) {   // same trip count in every lane: full-warp votes
+          unsigned dg[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            const int j = (e0 + e) * T + tid;
+            dg[e] = 0xffffffffu;
+            if (e0 + e < R && j < n) {
+              const unsigned key = key_at(j);
+              if ((key & mask) == prefix) dg[e] = (key >> shift) & 255u;
+            }
           }
-          count_digit(digit, buf);
+          count_digits8(hist[buf], dg, lane);
         }
       }
       cluster.sync();
       // every CTA adds up the cluster's histograms and finds the digit itself
-      int tot = 0, incl = 0;
+      int tot = 0;
       if (tid < 256) {
         int part[kTailCluster];
 #pragma unroll
@@ -756,28 +788,41 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
 #pragma unroll
         for (int r = 0; r < kTailCluster; ++r) tot += part[r];
         hist[buf ^ 1][tid] = 0;   // every CTA is past its reads of the other buffer
-        // suffix sums over the 256 bins: bins above this one
-        incl = tot;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          const int v = __shfl_down_sync(0xffffffffu, incl, o);
-          if (lane + o < 32) incl += v;
-        }
-        if (lane == 0) s_scan[warp][0] = incl;
       }
-      __syncthreads();
-      if (tid < 256) {
-        int above = incl - tot;
-        for (int w = warp + 1; w < 8; ++w) above += s_scan[w][0];
-        if (above < remaining && remaining <= above + tot) {
-          s_sel[0] = tid;
-          s_sel[1] = remaining - above;
-        }
-      }
-      __syncthreads();
+      find_digit(tot, remaining);
       prefix |= (unsigned)s_sel[0] << shift;
       remaining = s_sel[1];
       mask |= 255u << shift;
+      // A CTA that owns a whole head and keeps its keys in shared memory: two digits fix sign,
+      // exponent and seven mantissa bits, and the bin that holds the threshold is small.  Its
+      // keys (their low 16 bits) go to a list and the last two digits are searched there, two
+      // sweeps over a few hundred entries instead of two over all keys.  (With a cluster the
+      // sweeps are short already and a list costs as much as the two histogram exchanges.)
+      if (cs == 1 && pass == 1 && !inreg && cached && s_sel[2] <= kTailListCap) {
+        unsigned* list = reinterpret_cast<unsigned*>(sraw);   // after the keys; the pooling stage is free by now
+        for (int e = 0; e < R; ++e) {
+          const int j = e * T + tid;
+          if (j < n) {
+            const unsigned key = skeys[kslot(j)];
+            if ((key & mask) == prefix) list[atomicAdd(&s_nlist, 1)] = key & 0xffffu;
+          }
+        }
+        if (tid < 256) hist[1][tid] = 0;   // hist[0] is zero already
+        __syncthreads();
+        const int nl = s_nlist;
+        for (int e = tid; e < nl; e += T) atomicAdd(&hist[0][(list[e] >> 8) & 255u], 1);
+        __syncthreads();
+        find_digit(tid < 256 ? hist[0][tid] : 0, remaining);
+        const unsigned hi8 = (unsigned)s_sel[0];
+        remaining = s_sel[1];
+        for (int e = tid; e < nl; e += T)
+          if (((list[e] >> 8) & 255u) == hi8) atomicAdd(&hist[1][list[e] & 255u], 1);
+        __syncthreads();
+        find_digit(tid < 256 ? hist[1][tid] : 0, remaining);
+        prefix |= (hi8 << 8) | (unsigned)s_sel[0];
+        remaining = s_sel[1];
+        break;
+      }
     }
     tau = prefix;
     need_eq = remaining;
@@ -1033,7 +1078,8 @@ cudaError_t launch_tail(const LaunchCtx& c, const TailArgs& t) {
   if (fused && !a.cached) return cudaErrorInvalidValue;   // callers check tail_can_fuse() first
   size_t smem = 0;
   if (a.cached) smem += ((size_t)sh.chunk + (sh.chunk >> 5) + 1) * 4;
-  if (fused) smem += ((size_t)8 * sh.threads + 64) * 4;
+  if (fused) smem += ((size_t)8 * sh.threads + 64) * 4;          // pooling stage, later the key list
+  else if (a.cached) smem += (size_t)kTailListCap * 4;           // key list of a lone CTA
   if (sh.threads == 1024)
     return fused ? launch_tail_t<true, 1024>(c, a, sh, smem) : launch_tail_t<false, 1024>(c, a, sh, smem);
   return fused ? launch_tail_t<true, 512>(c, a, sh, smem) : launch_tail_t<false, 512>(c, a, sh, smem);
