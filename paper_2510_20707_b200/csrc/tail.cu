@@ -627,6 +627,7 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
       }
     }
   }
+  for (int t = tid; t < 256; t += T) hist[0][t] = 0;   // visible after the next CTA barrier
   const float* src = a.scores;
   const bool cached = FUSED || a.cached;
   float held[8];   // FUSED, R <= 8: mixed scores kept until the selection is done
@@ -677,23 +678,27 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
           ex[e] = avg ? ex[e] + w : fmaxf(ex[e], w);
         }
       }
+      unsigned top[8];   // leading digit of the block's keys: the first digit pass, taken here
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
         const int jb = e * T + tid;
         held[e] = 0.f;
+        top[e] = 0xffffffffu;
         if (jb < nb) {
           held[e] = mix_one(avg ? ex[e] * invk : ex[e], vn[e], dv[e], sc, a.mp.use_vnorm,
                             a.mp.mix_mode);
-          skeys[kslot(j0 + jb)] = order_key(held[e]);
+          const unsigned key = order_key(held[e]);
+          skeys[kslot(j0 + jb)] = key;
+          top[e] = key >> 24;
           if (R > 8) a.s_comp_out[poff + c0 + j0 + jb] = held[e];
         }
       }
+      count_digits8(hist[0], top, lane);
     }
     src = a.s_comp_out;
   } else if (a.cached) {
     for (int j = tid; j < n; j += T) skeys[kslot(j)] = order_key(src[poff + c0 + j]);
   }
-  for (int t = tid; t < 256; t += T) hist[0][t] = 0;
   __syncthreads();
   const int want = s_sel[1];
   int* out = a.idx + (size_t)layer * a.idx_cap + s_off;
@@ -749,7 +754,9 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
     };
     for (int pass = 0; pass < 4; ++pass) {
       const int shift = 24 - 8 * pass, buf = pass & 1;
-      if (inreg) {
+      if (FUSED && pass == 0) {
+        // the leading digits were counted while the keys were made
+      } else if (inreg) {
         unsigned dg[8];
 #pragma unroll
         for (int e = 0; e < 8; ++e)
@@ -868,7 +875,9 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
 #pragma unroll
       for (int r = 0; r < kTailCluster; ++r) gt_before += before[r].x, eq_before += before[r].y;
     }
-    for (int j = r0; j < r1; ++j) {
+    // most runs hold no kept position at all: their second walk is skipped
+    const bool writes = all || gt > 0 || (eq > 0 && eq_before < need_eq);
+    for (int j = r0; writes && j < r1; ++j) {
       const int i = c0 + j;
       if (all) {
         out[gt_before++] = i;
