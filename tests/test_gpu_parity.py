@@ -250,6 +250,33 @@ def test_adaptive_budgets_on_many_keys_are_exact(H, lens, levels):
     assert np.array_equal(got["idx"].cpu().numpy()[:offs[-1]], ref["idx"])
 
 
+@pytest.mark.parametrize("levels", [0, 50, 3000000])
+def test_whole_head_ctas_select_exactly(levels):
+    # 80 (sequence, head) units of 20000 candidates: one 1024-thread CTA per unit with the keys
+    # in shared memory.  Few score levels leave more keys in the bin after two digits than the
+    # key list takes (the four-pass search), many levels a few hundred (the list), levels = 0
+    # real-valued scores; a head of equal scores and negative zeros ride along.  Integer work:
+    # bit-identical to the oracle.
+    H, B, W, P = 8, 10, 16, 20000
+    rng = np.random.default_rng(levels + 3)
+    cu = (np.arange(B + 1) * (P + W)).astype(np.int32)
+    if levels:
+        s = (rng.integers(0, levels, size=(H, B * P)) / np.float32(levels)).astype(np.float32)
+    else:
+        s = rng.standard_normal((H, B * P)).astype(np.float32) ** 2
+    s[1, :P] = 0.25
+    s[2, ::5] = -0.0
+    po = oracle.Params(kv_heads=H, gqa_ratio=1, window=W, budget=W + 333)
+    pg = binding.Params(kv_heads=H, gqa_ratio=1, window=W, budget=W + 333)
+    ref = oracle.select(s, po, cu=cu)
+    got = binding.select(torch.from_numpy(s).cuda(), pg, cu_seqlens=[int(c) for c in cu])
+    assert int(got["status"].item()) == 0
+    offs = got["idx_offsets"].cpu().numpy()
+    assert np.array_equal(got["counts"].cpu().numpy(), ref["counts"].reshape(-1))
+    assert np.array_equal(offs, ref["idx_offsets"])
+    assert np.array_equal(got["idx"].cpu().numpy()[:offs[-1]], ref["idx"])
+
+
 def test_long_sequence_cluster_tail():
     # 65536 keys per head: the cluster shape of the tail kernel with 16 positions per thread
     wl = synth.small_workload(H=2, G=4, W=32, seq_lens=(65536,), pool_kernel=7, budget=512,
