@@ -641,29 +641,37 @@ k_tail(const SeqTable st, const Workspace ws, const TailKernelArgs a) {
     if (warp == 1)
       head_scalars(st, ws, layer, b, h, a.mp.pool_k, a.mp.pool_mode, a.mp.use_vnorm, a.mp.eps,
                    a.rbar_in, lane, sc);
-    for (int j0 = 0; j0 < n; j0 += 8 * T) {
-      const int nb = min(8 * T, n - j0);   // positions of this block
-      __syncthreads();                     // the previous block's readers of sraw are done
-      // every load of the block is issued before the first use; the block and its pooling halo
-      // (62 positions at most) are nine rounds of T raw scores
-      float raw[9], vn[8], dv[8];
-      const int nstage = nb + 2 * half;
+    // The block and its pooling halo (62 positions at most) are nine rounds of T raw scores.
+    // They are loaded one block ahead: the raw scores of block b + 1 fly while block b is pooled
+    // and mixed, and the two per-position terms of a block are asked for before its pooling and
+    // used after it.
+    float raw[9];
+    auto load_raw = [&](const int j0) {
+      const int nstage = min(8 * T, n - j0) + 2 * half;
 #pragma unroll
       for (int e = 0; e < 9; ++e) {
         const int t = e * T + tid, i = c0 + j0 - half + t;
-        raw[e] = (t < nstage && i >= 0 && i < P) ? ws.s_ex_raw[poff + i] : pad;
+        raw[e] = (j0 < n && t < nstage && i >= 0 && i < P) ? ws.s_ex_raw[poff + i] : pad;
       }
+    };
+    load_raw(0);
+    for (int j0 = 0; j0 < n; j0 += 8 * T) {
+      const int nb = min(8 * T, n - j0);   // positions of this block
+      float vn[8], dv[8];
+      const int nstage = nb + 2 * half;
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
         const int jb = e * T + tid;
         vn[e] = (a.mp.use_vnorm && jb < nb) ? ws.vnorm[poff + c0 + j0 + jb] : 0.f;
         dv[e] = jb < nb ? a.s_div[poff + c0 + j0 + jb] : 0.f;
       }
+      __syncthreads();                     // the previous block's readers of sraw are done
 #pragma unroll
       for (int e = 0; e < 9; ++e) {
         const int t = e * T + tid;
         if (t < nstage) sraw[t] = raw[e];
       }
+      load_raw(j0 + 8 * T);
       __syncthreads();
       // the eight pooling windows advance together (same order of additions as pool_window),
       // so their shared-memory loads overlap instead of forming eight serial chains
