@@ -123,6 +123,12 @@ __device__ __forceinline__ f32x2 ex2_pair(f32x2 t2, const bool poly) {
   return pack2(ex2(a0), ex2(a1));
 }
 
+// The two bf16 of a word as a packed fp32 pair (low half first), built in place in the 64-bit
+// register (a pair assembled from two separate floats costs moves).
+__device__ __forceinline__ f32x2 bf16x2_wide(const uint32_t w) {
+  return ((unsigned long long)(w & 0xffff0000u) << 32) | (unsigned long long)(w << 16);
+}
+
 constexpr size_t kSmemLimit = 227 * 1024;   // dynamic shared memory a CTA may ask for
 
 // ======================================================================== pass 1
@@ -532,12 +538,11 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
 #pragma unroll
         for (int rr = 0; rr < 8; ++rr) {
           u[rr] = *reinterpret_cast<const uint4*>(tile + sw128_offset(row0 + rr, cc));
-          const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&u[rr]);
+          const uint32_t* p2 = reinterpret_cast<const uint32_t*>(&u[rr]);
           f32x2 sq = pack2(0.f, 0.f);
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
-            const float2 f = __bfloat1622float2(p2[e]);
-            const f32x2 f2 = pack2(f.x, f.y);
+            const f32x2 f2 = bf16x2_wide(p2[e]);
             sq = fma2(f2, f2, sq);
           }
           float s0, s1;
@@ -564,13 +569,10 @@ k_pass1(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
 #pragma unroll
         for (int rr = 0; rr < 8; ++rr) {
           const float w = __shfl_sync(0xffffffffu, inv, (lane & 16) | (rr << 1));
-          const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&u[rr]);
+          const uint32_t* p2 = reinterpret_cast<const uint32_t*>(&u[rr]);
           const f32x2 w2 = pack2(w, w);
 #pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const float2 f = __bfloat1622float2(p2[e]);
-            acc2[e] = fma2(pack2(f.x, f.y), w2, acc2[e]);
-          }
+          for (int e = 0; e < 4; ++e) acc2[e] = fma2(bf16x2_wide(p2[e]), w2, acc2[e]);
         }
       }
       // (no barrier per tile: after an abort the waits fail at once and every warp still walks
@@ -977,11 +979,10 @@ k_pass2(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtenso
             for (int c = 0; c < 8; ++c) {
               const uint4 u =
                   *reinterpret_cast<const uint4*>(tile + half * (kVSubBytes / 2) + sw128_offset(vr, c));
-              const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&u);
+              const uint32_t* p2 = reinterpret_cast<const uint32_t*>(&u);
 #pragma unroll
               for (int e = 0; e < 4; ++e) {
-                const float2 f = __bfloat1622float2(p2[e]);
-                const f32x2 f2 = pack2(f.x, f.y);
+                const f32x2 f2 = bf16x2_wide(p2[e]);
                 ss2[e & 1] = fma2(f2, f2, ss2[e & 1]);
               }
             }
