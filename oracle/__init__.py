@@ -260,7 +260,7 @@ def compress_layer(K, V, Q, params: Params, cu=None, rbar_in=None) -> Dict[str, 
 # The paper plugs its scores into compressors that only differ in how many rows a layer or a
 # head keeps (Sec. 4.1; related work: PyramidKV layer schedules, SparseMM / HeadKV per-head
 # shares).  These two functions are plain Python on top of `topb`; the paper prints no formula
-# for either policy, so the schedule below is this build's reading (parity unpinned by the
+# for either policy, so the schedule below is the reading taken here (parity unpinned by the
 # paper; pinned by its invariants: total kept, monotone, taper 0 = uniform).
 def select_given(s: np.ndarray, head_budgets, params: Params, cu=None) -> Dict[str, np.ndarray]:
     """Top-b on given scores [H, Ptot] with the rows to keep per (sequence, head) given

@@ -367,7 +367,7 @@ void mixkv_oracle_topb(const float* s, int n, int b, int32_t* idx) {
 }
 
 /* Budgets of one sequence (Algorithm 1: B' = B - W candidates kept per head).
- * Fixed: every head gets min(B - W, P).  Adaptive (this build's reading of the
+ * Fixed: every head gets min(B - W, P).  Adaptive (the reading taken here of the
  * one-sentence AdaKV description): each head is guaranteed f = floor(floor_frac *
  * (B - W)); the remaining H * (B - W - f) slots go to the globally highest scores
  * of the H heads together (ties to the lower (head, position)); head h gets
