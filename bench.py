@@ -455,6 +455,12 @@ def run_mixkv(args):
         "clocks": clocks,
         "gpu_launches": n_stage * args.steps * len(blocks),
     }
+    # the head-wise redundancy the kernels measured on these inputs (Eq. 4), first layer: the
+    # weight that Eq. 5 gives the diversity score of each head
+    sc0 = binding.scores(dev_in[0]["K"][0], dev_in[0]["V"][0], dev_in[0]["Q"][0], pg,
+                         cu_seqlens=cu_list, want_parts=True)
+    torch.cuda.synchronize()
+    line["config"]["rbar_first_layer"] = [round(float(x), 3) for x in sc0["rbar"].flatten().tolist()]
     if per_layer_ms is not None:
         one_us = per_layer_ms / NL * 1e3
         line["one_layer_per_call"] = {
